@@ -1,0 +1,220 @@
+/*
+ * liblsa — C ABI of the LongCat-Sparse-Attention indexer + sparse-attention forward
+ * for NVIDIA B200 (sm_100a).
+ *
+ * The path (one cross-layer group of R attention layers that share one index set):
+ *
+ *   a0  lsa_block_means   sub-block mean keys                       Sec. 3.3, stage 1 (first paragraph)
+ *   a1  coarse page score I_page[t,p]                               Eq. 9
+ *   a2  top-M pages                                                 Eq. 10
+ *   a3  fine token score  I[t,s] on the recalled pages              Eq. 11 (= Eq. 1)
+ *   a4  top-K_sparse outside sink and window                        Eq. 12 with Eq. 6-7
+ *   a5  lsa_convert       index set -> contiguous pieces / physical cache rows   Sec. 3.1 (streaming-aware layout)
+ *   a6  lsa_sparse_attn   attention over sink U window U sparse     Eq. 3, Sec. 4.1.1
+ *   a7  lsa_layer_group   a0..a5 once, a6 for each of the R layers  Sec. 3.2
+ *
+ * Conventions
+ *   - Positions are 0-indexed.  Query t sees keys s <= t.  S = k_sink, W = k_swa, Ksp = k_sparse.
+ *     Candidate range of query t: C(t) = [S, t-W] (empty when t-W < S).  sink = [0, min(S,t+1)),
+ *     window = [max(S, t-W+1), t].
+ *   - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".
+ *     The library allocates no device memory: scratch lives in the workspace given to
+ *     lsa_create (size it with lsa_workspace_bytes).
+ *   - Every call enqueues work on the context's stream and returns without waiting.
+ *   - Return value: LSA_OK or a negative lsa_error.  Nothing throws, aborts or traps.
+ *     A device-side status word (0 = fine) records kernel-detected problems (bounded wait
+ *     expired); read it with lsa_status.
+ *   - bf16 tensors are passed as void*; rows are contiguous unless a leading dimension is given.
+ *     All base pointers must be 16-byte aligned and every row stride a multiple of 16 bytes.
+ *   - Top-K order is total: larger score first, on equal scores the smaller position first;
+ *     +0 and -0 are equal.  Inputs must be finite.  Selected positions are reported ascending.
+ *
+ * Supported shapes (anything else returns LSA_ERR_SHAPE):
+ *   indexer  (H_I, d_I) in {(8,64), (64,128)};  page P in {64,128,256}, sub_block B with P/B in
+ *            {8,16,32};  keep_pages*P <= 4096;  k_sparse <= 4096, multiple of 4
+ *   attention (H, d_qk, d_v) in {(16,128,128), (64,576,512)}
+ *   paged mode needs kv_page == page.
+ */
+#ifndef LSA_H_
+#define LSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define LSA_API __attribute__((visibility("default")))
+#else
+#define LSA_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LSA_OK = 0,
+  LSA_ERR_ARG = -1,        /* null pointer, negative size, inconsistent arguments */
+  LSA_ERR_SHAPE = -2,      /* dimension or alignment the kernels do not support */
+  LSA_ERR_WORKSPACE = -3,  /* workspace missing or smaller than lsa_workspace_bytes says */
+  LSA_ERR_CUDA = -4,       /* a CUDA runtime call failed (see lsa_last_cuda_error) */
+  LSA_ERR_TIMEOUT = -5     /* a bounded device-side wait expired (reported through lsa_status) */
+} lsa_error;
+
+enum { LSA_KEY_BF16 = 0, LSA_KEY_E4M3 = 1 };
+
+typedef struct lsa_ctx lsa_ctx;
+
+/* Plain data; set struct_size = sizeof(lsa_params). */
+typedef struct {
+  uint32_t struct_size;
+  int32_t n_heads_idx;  /* H_I  (Eq. 1) */
+  int32_t d_idx;        /* d_I */
+  int32_t key_dtype;    /* LSA_KEY_BF16, or LSA_KEY_E4M3 = OCP e4m3 codes + one fp32 scale per token */
+  int32_t page;         /* P   (Sec. 3.3) */
+  int32_t sub_block;    /* B,  divides P */
+  int32_t keep_pages;   /* M */
+  int32_t k_sparse;     /* Ksp (Eq. 6) */
+  int32_t k_sink;       /* S */
+  int32_t k_swa;        /* W */
+  int32_t n_heads;      /* H  attention heads; all share one K/V row per token (absorbed MQA, Sec. 2.2) */
+  int32_t d_qk;
+  int32_t d_v;
+  float sm_scale;       /* logits = sm_scale * q.k */
+  int32_t n_layers;     /* R, size of the cross-layer group (Sec. 3.2) */
+  int32_t q_chunk;      /* queries scored per pass of the indexer in lsa_layer_group; 0 = all at once */
+  int32_t hi_enable;    /* 1: two-stage selection (Eq. 9-12); 0: every eligible page is kept (Eq. 7) */
+  int32_t paged;        /* 0: caches are [n_key, d] arrays and queries are consecutive positions (prefill)
+                           1: caches are pools [n_phys_pages*kv_page, d] read through page_table and there is
+                              one query per sequence at position ctx_len[b]-1 (decode) */
+  int32_t kv_page;      /* tokens per physical cache page (paged mode) */
+} lsa_params;
+
+/* ---- context ------------------------------------------------------------------------------ */
+
+/* Create a context bound to `device` and to `cuda_stream` (a cudaStream_t; NULL = legacy default).
+ * `workspace` is caller-owned device memory of `workspace_bytes` bytes, 256-byte aligned, that must
+ * outlive the context; calls on one context must not overlap on the GPU.  Host allocations only. */
+LSA_API int lsa_create(lsa_ctx** ctx, int device, void* cuda_stream, void* workspace, size_t workspace_bytes);
+LSA_API int lsa_destroy(lsa_ctx* ctx);
+
+/* Scratch needed by any call with these parameters for n_query queries (prefill: the largest number
+ * passed to one call; with q_chunk > 0 lsa_layer_group needs only q_chunk of them), caches of at most
+ * n_key_max tokens per sequence and `batch` sequences (paged mode).  Writes *bytes (host). */
+LSA_API int lsa_workspace_bytes(const lsa_params* p, int64_t n_query, int64_t n_key_max, int batch, size_t* bytes);
+
+/* Waits for the stream, then writes the device status word (host int; 0 = fine, LSA_ERR_TIMEOUT...)
+ * and clears it. */
+LSA_API int lsa_status(lsa_ctx* ctx, int* device_status);
+LSA_API const char* lsa_strerror(int err);
+/* Text of the last CUDA error seen by this context (host string owned by the library). */
+LSA_API const char* lsa_last_cuda_error(lsa_ctx* ctx);
+/* Number of kernels this context has launched since creation (host counter). */
+LSA_API int64_t lsa_launch_count(lsa_ctx* ctx);
+
+/* ---- a0: mean-key cache (Sec. 3.3) ---------------------------------------------------------- */
+
+/* kmean[n, :] = mean over the tokens present in sub-block n of the (dequantised) indexer keys, fp32
+ * accumulation, stored bf16 (round to nearest even).
+ *   k_idx    bf16 [n_key, d_I]  or  uint8 e4m3 codes [n_key, d_I] with k_scale fp32 [n_key]
+ *   kmean    bf16 [ceil(n_key/B), d_I]
+ * Paged mode: k_idx / k_scale are pools indexed by physical row and kmean is the twin pool
+ * [n_phys_pages*kv_page/B, d_I]: sub-block j of physical page g is row g*(kv_page/B)+j.  The means of
+ * sequence b's first ctx_len[b] tokens are written (a trailing partial sub-block averages the tokens
+ * present); n_key is ignored; page_table int32 [batch, page_table_stride].
+ * Prefill: page_table = ctx_len = NULL, batch = 1. */
+LSA_API int lsa_block_means(lsa_ctx* ctx, const lsa_params* p, const void* k_idx, const float* k_scale,
+                    int64_t n_key, const int32_t* page_table, int64_t page_table_stride,
+                    const int32_t* ctx_len, int batch, void* kmean);
+
+/* ---- a1-a4: the indexer (Eq. 9-12 with the scoring range of Eq. 7) -------------------------- */
+
+/* For each query: eligible pages E = pages meeting C(t); if hi_enable and |E| > M keep the M pages
+ * with the largest Eq.-9 score, else all of E; score the tokens of the kept pages inside C(t) with
+ * Eq. 1 (fp32 accumulation of bf16 products; e4m3 keys are widened exactly and the per-token scale is
+ * applied to the dot product); keep the Ksp largest.
+ *   q_idx       bf16 [n_query, H_I, d_I]       w  fp32 [n_query, H_I]
+ *   k_idx/k_scale/kmean  as in lsa_block_means
+ *   prefill (paged=0): query row i sits at position q_pos0+i; n_key tokens are cached (>= q_pos0+n_query);
+ *                      page_table = ctx_len = NULL, batch = 1
+ *   decode (paged=1):  n_query = batch; query b sits at ctx_len[b]-1; page_table int32
+ *                      [batch, page_table_stride] maps logical page -> physical page
+ *   sparse_idx  int32 [n_query, Ksp]  ascending positions (logical), padded with -1
+ *   n_sparse    int32 [n_query]
+ *   pages_out   optional int32 [n_query, M] kept pages ascending, -1 padded (NULL to skip)
+ * Scratch: the page-score matrix fp32 [n_query, ceil(n_key_max/P)] in the workspace. */
+LSA_API int lsa_index(lsa_ctx* ctx, const lsa_params* p, const void* q_idx, const float* w, const void* k_idx,
+              const float* k_scale, const void* kmean, int64_t q_pos0, int64_t n_query, int64_t n_key,
+              const int32_t* page_table, int64_t page_table_stride, const int32_t* ctx_len, int batch,
+              int32_t* sparse_idx, int32_t* n_sparse, int32_t* pages_out);
+
+/* The selection step alone (Eq. 2 / 7 / 10 / 12) on caller-given fp32 scores; bit-exact by definition.
+ *   scores    fp32 [n_query, ld_scores], column c of row i is the score of candidate c
+ *   cand_pos  NULL: candidate c is position c;  else int32 [n_query, n_cand] positions, -1 = absent
+ *   apply_range 1: only positions inside C(q_pos0+i) (from k_sink, k_swa) take part; 0: all present
+ *   idx_out   int32 [n_query, k] ascending positions, -1 padded;  n_out int32 [n_query]
+ * n_cand is unlimited (scores are re-read from memory on every radix pass); k <= 8192. */
+LSA_API int lsa_select(lsa_ctx* ctx, const lsa_params* p, const float* scores, int64_t ld_scores,
+               const int32_t* cand_pos, int64_t q_pos0, int64_t n_query, int64_t n_cand, int32_t k,
+               int32_t apply_range, int32_t* idx_out, int32_t* n_out);
+
+/* ---- a5: streaming-aware conversion (Sec. 3.1) ---------------------------------------------- */
+
+/* Lays the index set of each query out as cache rows in the order the attention kernel streams them:
+ * [sink run | sparse rows ascending | window run].  In paged mode each position is translated to its
+ * physical row  page_table[b][pos / kv_page] * kv_page + pos % kv_page, so that the sink and the window
+ * become runs of whole contiguous pages and the R layers of the group share one translation.
+ *   rows_out   int32 [n_query, k_sink + k_sparse + k_swa]   (-1 padded)     n_rows_out int32 [n_query]
+ *   runs_out   optional int32 [n_query, 4] = {first sink row count, sparse count, window count,
+ *              number of maximal runs of consecutive rows in the list}  (NULL to skip) */
+LSA_API int lsa_convert(lsa_ctx* ctx, const lsa_params* p, const int32_t* sparse_idx, const int32_t* n_sparse,
+                int64_t q_pos0, int64_t n_query, const int32_t* page_table, int64_t page_table_stride,
+                const int32_t* ctx_len, int batch, int32_t* rows_out, int32_t* n_rows_out, int32_t* runs_out);
+
+/* ---- a6: sparse attention (Eq. 3) ------------------------------------------------------------ */
+
+/* out[t,h,:] = sum_{s in S_t} softmax_s(sm_scale * q[t,h].k[s]) * v[s,:d_v],  S_t = sink U window U sparse;
+ * bf16 tensor-core products, fp32 softmax and accumulation; one softmax over the whole set.
+ *   q    bf16 [n_query, H, d_qk]
+ *   k    bf16 rows of ld_k elements (>= d_qk);  v bf16 rows of ld_v elements (>= d_v).  MLA latent: v == k.
+ *   sparse_idx / n_sparse  as written by lsa_index (logical positions)
+ *   rows / n_rows  optional output of lsa_convert; when given (required in paged mode) the kernel reads
+ *                  these cache rows instead of rebuilding the set from sparse_idx
+ *   out  bf16 [n_query, H, d_v]      lse  optional fp32 [n_query, H] = log sum_s exp(logit)
+ * Paged mode splits each sequence's rows over several thread blocks; the partial results sit in the
+ * workspace and are merged by their log-sum-exp. */
+LSA_API int lsa_sparse_attn(lsa_ctx* ctx, const lsa_params* p, const void* q, const void* k, const void* v,
+                    int64_t ld_k, int64_t ld_v, const int32_t* sparse_idx, const int32_t* n_sparse,
+                    const int32_t* rows, const int32_t* n_rows, int64_t q_pos0, int64_t n_query,
+                    int64_t n_key, const int32_t* ctx_len, int batch, void* out, float* lse);
+
+/* ---- a7: one cross-layer group (Sec. 3.2) ---------------------------------------------------- */
+
+/* Indexer once (lsa_index, in passes of q_chunk queries when q_chunk > 0), conversion once, then the
+ * attention of the R = n_layers layers one after the other on the context's stream, all with the same
+ * index set.  q/k/v/out/lse are HOST arrays of R device pointers (lse or its entries may be NULL).
+ * kmean must already hold the means (lsa_block_means) — the cache is maintained per sequence, not per
+ * group.  sparse_idx / n_sparse are caller buffers, returned filled for inspection. */
+LSA_API int lsa_layer_group(lsa_ctx* ctx, const lsa_params* p, const void* q_idx, const float* w,
+                    const void* k_idx, const float* k_scale, const void* kmean, int64_t q_pos0,
+                    int64_t n_query, int64_t n_key, const int32_t* page_table, int64_t page_table_stride,
+                    const int32_t* ctx_len, int batch, const void* const* q, const void* const* k,
+                    const void* const* v, int64_t ld_k, int64_t ld_v, void* const* out, float* const* lse,
+                    int32_t* sparse_idx, int32_t* n_sparse);
+
+/* Same group, prefill only, with the per-query tensors in HOST memory (pinned for full speed):
+ * q_idx_host, w_host, q_host[r], out_host[r] are host pointers; caches (k_idx, k_scale, kmean, k[r], v[r])
+ * stay device-resident.  The queries are processed in passes of `stage_queries`; each pass copies its
+ * slice of q_idx, w and q[r] to the device staging buffers, runs the group on it and copies out[r] back;
+ * copies of the next pass overlap the kernels of the current one on two internal streams.
+ * stage[2] are two caller-owned device staging areas of lsa_host_stage_bytes() bytes each. */
+LSA_API int lsa_layer_group_host(lsa_ctx* ctx, const lsa_params* p, const void* q_idx_host, const float* w_host,
+                         const void* k_idx, const float* k_scale, const void* kmean, int64_t n_query,
+                         int64_t n_key, const void* const* q_host, const void* const* k,
+                         const void* const* v, int64_t ld_k, int64_t ld_v, void* const* out_host,
+                         int64_t stage_queries, void* const* stage, size_t stage_bytes);
+LSA_API int lsa_host_stage_bytes(const lsa_params* p, int64_t stage_queries, size_t* bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LSA_H_ */

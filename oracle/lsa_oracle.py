@@ -191,7 +191,7 @@ def select_sparse(t, q_I, w, k_hat, km, *, P, B, M, Ksp, S, W, hi_enable=True):
         pages = E
     cand = np.concatenate([np.arange(max(lo, p * P), min(hi, p * P + P - 1) + 1, dtype=np.int64)
                            for p in pages])
-    I = indexer_scores(q_I, w, np.asarray(k_hat, dtype=np.float64)[cand])
+    I = indexer_scores(q_I, w, np.asarray(k_hat)[cand])
     return top_k(I, cand, Ksp), pages
 
 
@@ -236,8 +236,8 @@ def attend(q, k, v, S_t, sm_scale):
     """
     q = np.asarray(q, dtype=np.float64)
     S_t = np.asarray(S_t, dtype=np.int64)
-    ks = np.asarray(k, dtype=np.float64)[S_t]
-    vs = np.asarray(v, dtype=np.float64)[S_t]
+    ks = np.asarray(k)[S_t].astype(np.float64)     # gather first: the caches may be huge float32 arrays
+    vs = np.asarray(v)[S_t].astype(np.float64)
     z = sm_scale * (q @ ks.T)                 # [H, |S_t|]
     m = z.max(axis=1, keepdims=True)
     e = np.exp(z - m)

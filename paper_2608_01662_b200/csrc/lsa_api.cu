@@ -1,0 +1,447 @@
+// C ABI of liblsa: argument checking, workspace carving and the sequencing of the kernels.
+// Every step of the path runs in the CUDA kernels of lsa_index.cu / lsa_attn.cu; nothing here
+// computes on the host.
+#include "../../include/lsa.h"
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "lsa_internal.h"
+
+struct lsa_ctx {
+  int device;
+  cudaStream_t stream;
+  uint8_t* ws;
+  size_t ws_bytes;
+  int sm_count;
+  int64_t launches;
+  char cuda_msg[256];
+  // lsa_layer_group_host only
+  cudaStream_t copy_in, copy_out;
+  cudaEvent_t ev_in[2], ev_done[2], ev_out[2];
+};
+
+namespace {
+
+constexpr size_t kStatusBytes = 256;
+constexpr int kMaxSplit = 16;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int cuda_fail(lsa_ctx* c, cudaError_t e) {
+  if (c) std::snprintf(c->cuda_msg, sizeof(c->cuda_msg), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+  return LSA_ERR_CUDA;
+}
+
+bool pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_params(const lsa_params* p, bool need_index, bool need_attn) {
+  if (p == nullptr || p->struct_size != sizeof(lsa_params)) return LSA_ERR_ARG;
+  if (p->k_sink < 0 || p->k_swa < 0 || p->k_sparse < 0) return LSA_ERR_ARG;
+  if (p->paged != 0 && p->paged != 1) return LSA_ERR_ARG;
+  if (need_index) {
+    if (p->key_dtype != LSA_KEY_BF16 && p->key_dtype != LSA_KEY_E4M3) return LSA_ERR_ARG;
+    if (p->page <= 0 || p->sub_block <= 0 || p->keep_pages <= 0) return LSA_ERR_ARG;
+    if (!lsa::index_shape_supported(p->n_heads_idx, p->d_idx)) return LSA_ERR_SHAPE;
+    if (p->page != 64 && p->page != 128 && p->page != 256) return LSA_ERR_SHAPE;
+    if (p->page % p->sub_block != 0) return LSA_ERR_SHAPE;
+    const int spp = p->page / p->sub_block;
+    if (spp != 8 && spp != 16 && spp != 32) return LSA_ERR_SHAPE;
+    if (static_cast<int64_t>(p->keep_pages) * p->page > 4096) return LSA_ERR_SHAPE;
+    if (p->k_sparse > 4096 || p->k_sparse % 4 != 0) return LSA_ERR_SHAPE;
+    if (p->paged && p->kv_page != p->page) return LSA_ERR_SHAPE;
+  }
+  if (need_attn) {
+    if (!lsa::attn_shape_supported(p->n_heads, p->d_qk, p->d_v)) return LSA_ERR_SHAPE;
+    if (!(p->sm_scale > 0.f)) return LSA_ERR_ARG;
+    if (p->paged && !pow2(p->kv_page)) return LSA_ERR_SHAPE;
+  }
+  return LSA_OK;
+}
+
+// Workspace map.  All offsets are multiples of 256 bytes.
+struct WsLayout {
+  size_t page_scores, rows, n_rows, part_out, part_lse, total;
+  int ps_ld, rows_ld;
+};
+
+WsLayout ws_layout(const lsa_params* p, int64_t n_query, int64_t n_key_max, int batch) {
+  WsLayout l{};
+  size_t off = kStatusBytes;
+  const int64_t nq = p->paged ? batch : n_query;
+  const int P = p->page > 0 ? p->page : 64;
+  l.ps_ld = static_cast<int>(align_up(static_cast<size_t>((n_key_max + P - 1) / P), 4));
+  l.page_scores = off;
+  off += align_up(static_cast<size_t>(nq) * l.ps_ld * sizeof(float), 256);
+  l.rows_ld = p->k_sink + p->k_sparse + p->k_swa;
+  if (p->paged) {
+    l.rows = off;
+    off += align_up(static_cast<size_t>(batch) * l.rows_ld * sizeof(int32_t), 256);
+    l.n_rows = off;
+    off += align_up(static_cast<size_t>(batch) * sizeof(int32_t), 256);
+    l.part_out = off;
+    off += align_up(static_cast<size_t>(batch) * kMaxSplit * p->n_heads * p->d_v * sizeof(float), 256);
+    l.part_lse = off;
+    off += align_up(static_cast<size_t>(batch) * kMaxSplit * p->n_heads * sizeof(float), 256);
+  }
+  l.total = off;
+  return l;
+}
+
+int* status_word(lsa_ctx* c) { return c->ws ? reinterpret_cast<int*>(c->ws) : nullptr; }
+
+// Number of row splits per sequence in paged (decode) attention: fill the SMs with whole waves.
+int pick_split(int sm_count, int batch, int max_rows) {
+  const int tiles = (max_rows + 63) / 64;
+  int best = 1;
+  double best_eff = 0.0;
+  for (int s = 1; s <= kMaxSplit && s <= tiles; ++s) {
+    if ((tiles + s - 1) / s < 4 && s > 1) break;  // keep at least 4 tiles per block
+    const int blocks = batch * s;
+    const int waves = (blocks + sm_count - 1) / sm_count;
+    const double eff = static_cast<double>(blocks) / (static_cast<double>(waves) * sm_count);
+    if (eff > best_eff + 1e-9) {
+      best_eff = eff;
+      best = s;
+    }
+  }
+  return best;
+}
+
+int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w, const void* k_idx,
+              const float* k_scale, const void* kmean, int64_t q_pos0, int64_t n_query, int64_t n_key,
+              const int32_t* page_table, int64_t pt_stride, const int32_t* ctx_len, int batch,
+              int32_t* sparse_idx, int32_t* n_sparse, int32_t* pages_out) {
+  const int64_t nq = p->paged ? batch : n_query;
+  if (nq == 0) return LSA_OK;
+  const int64_t n_key_max = p->paged ? pt_stride * p->kv_page : n_key;
+  // without the coarse stage every eligible page is scored: the candidate buffer bounds the cache length
+  if (!p->hi_enable && n_key_max > 4096) return LSA_ERR_SHAPE;
+  const int64_t chunk = (!p->paged && p->q_chunk > 0) ? p->q_chunk : nq;
+  const WsLayout l = ws_layout(p, chunk < nq ? chunk : nq, n_key_max, batch);
+  if (c->ws == nullptr || l.total > c->ws_bytes) return LSA_ERR_WORKSPACE;
+  for (int64_t q0 = 0; q0 < nq; q0 += chunk) {
+    const int64_t n = nq - q0 < chunk ? nq - q0 : chunk;
+    lsa::IndexArgs a{};
+    a.HI = p->n_heads_idx; a.DI = p->d_idx; a.key_e4m3 = p->key_dtype == LSA_KEY_E4M3;
+    a.P = p->page; a.B = p->sub_block; a.M = p->keep_pages; a.Ksp = p->k_sparse; a.S = p->k_sink; a.W = p->k_swa;
+    a.hi_enable = p->hi_enable; a.paged = p->paged;
+    a.q_idx = static_cast<const uint8_t*>(q_idx) + q0 * p->n_heads_idx * p->d_idx * 2;
+    a.w = w + q0 * p->n_heads_idx;
+    a.k_idx = k_idx; a.k_scale = k_scale; a.kmean = kmean;
+    a.q_pos0 = q_pos0 + q0; a.n_query = static_cast<int>(n); a.n_key = n_key;
+    a.page_table = page_table; a.pt_stride = pt_stride; a.ctx_len = ctx_len;
+    a.page_scores = reinterpret_cast<float*>(c->ws + l.page_scores); a.ps_ld = l.ps_ld;
+    a.sparse_idx = sparse_idx + q0 * p->k_sparse; a.n_sparse = n_sparse + q0;
+    a.pages_out = pages_out ? pages_out + q0 * p->keep_pages : nullptr;
+    a.status = status_word(c);
+    cudaError_t e = cudaSuccess;
+    if (p->hi_enable) e = lsa::launch_coarse(a, c->stream, &c->launches);
+    if (e == cudaSuccess) e = lsa::launch_fine_select(a, c->stream, &c->launches);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+  }
+  return LSA_OK;
+}
+
+int run_attn(lsa_ctx* c, const lsa_params* p, const void* q, const void* k, const void* v, int64_t ld_k,
+             int64_t ld_v, const int32_t* sparse_idx, const int32_t* n_sparse, const int32_t* rows,
+             const int32_t* n_rows, int64_t q_pos0, int64_t n_query, const int32_t* ctx_len, int batch,
+             void* out, float* lse) {
+  const int64_t nq = p->paged ? batch : n_query;
+  if (nq == 0) return LSA_OK;
+  lsa::AttnArgs a{};
+  a.H = p->n_heads; a.DQK = p->d_qk; a.DV = p->d_v; a.S = p->k_sink; a.W = p->k_swa; a.Ksp = p->k_sparse;
+  a.paged = p->paged; a.sm_scale = p->sm_scale;
+  a.q = q; a.k = k; a.v = v; a.ld_k = ld_k; a.ld_v = ld_v;
+  a.sparse_idx = sparse_idx; a.n_sparse = n_sparse; a.rows = rows; a.n_rows = n_rows;
+  a.rows_ld = p->k_sink + p->k_sparse + p->k_swa;
+  a.q_pos0 = q_pos0; a.n_query = static_cast<int>(nq); a.ctx_len = ctx_len; a.out = out; a.lse = lse;
+  a.n_split = 1; a.status = status_word(c);
+  if (p->paged) {
+    const WsLayout l = ws_layout(p, nq, 0, batch);
+    if (c->ws == nullptr || l.total > c->ws_bytes) return LSA_ERR_WORKSPACE;
+    a.n_split = pick_split(c->sm_count, batch, a.rows_ld);
+    a.part_out = reinterpret_cast<float*>(c->ws + l.part_out);
+    a.part_lse = reinterpret_cast<float*>(c->ws + l.part_lse);
+  }
+  if (a.H == 64 && !(v == k && ld_v == ld_k)) return LSA_ERR_SHAPE;
+  cudaError_t e = lsa::launch_attn(a, c->stream, &c->launches);
+  return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
+}
+
+}  // namespace
+
+extern "C" {
+
+int lsa_create(lsa_ctx** ctx, int device, void* cuda_stream, void* workspace, size_t workspace_bytes) {
+  if (ctx == nullptr) return LSA_ERR_ARG;
+  *ctx = nullptr;
+  if (workspace != nullptr && (reinterpret_cast<uintptr_t>(workspace) & 255u)) return LSA_ERR_ARG;
+  if (workspace != nullptr && workspace_bytes < kStatusBytes) return LSA_ERR_WORKSPACE;
+  cudaError_t e = cudaSetDevice(device);
+  if (e != cudaSuccess) return LSA_ERR_CUDA;
+  lsa_ctx* c = new (std::nothrow) lsa_ctx();
+  if (c == nullptr) return LSA_ERR_ARG;
+  std::memset(c, 0, sizeof(*c));
+  c->device = device;
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  c->ws = static_cast<uint8_t*>(workspace);
+  c->ws_bytes = workspace ? workspace_bytes : 0;
+  e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking);
+  for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+    e = cudaEventCreateWithFlags(&c->ev_in[i], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_done[i], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_out[i], cudaEventDisableTiming);
+  }
+  if (e == cudaSuccess && c->ws) e = cudaMemsetAsync(c->ws, 0, kStatusBytes, c->stream);
+  if (e != cudaSuccess) {
+    delete c;
+    return LSA_ERR_CUDA;
+  }
+  *ctx = c;
+  return LSA_OK;
+}
+
+int lsa_destroy(lsa_ctx* c) {
+  if (c == nullptr) return LSA_ERR_ARG;
+  cudaSetDevice(c->device);
+  for (int i = 0; i < 2; ++i) {
+    if (c->ev_in[i]) cudaEventDestroy(c->ev_in[i]);
+    if (c->ev_done[i]) cudaEventDestroy(c->ev_done[i]);
+    if (c->ev_out[i]) cudaEventDestroy(c->ev_out[i]);
+  }
+  if (c->copy_in) cudaStreamDestroy(c->copy_in);
+  if (c->copy_out) cudaStreamDestroy(c->copy_out);
+  delete c;
+  return LSA_OK;
+}
+
+int lsa_workspace_bytes(const lsa_params* p, int64_t n_query, int64_t n_key_max, int batch, size_t* bytes) {
+  if (bytes == nullptr || n_query < 0 || n_key_max < 0 || batch < 0) return LSA_ERR_ARG;
+  const int r = check_params(p, true, true);
+  if (r != LSA_OK) return r;
+  int64_t nq = n_query;
+  if (!p->paged && p->q_chunk > 0 && p->q_chunk < nq) nq = p->q_chunk;
+  *bytes = ws_layout(p, nq, n_key_max, batch).total;
+  return LSA_OK;
+}
+
+int lsa_status(lsa_ctx* c, int* device_status) {
+  if (c == nullptr || device_status == nullptr) return LSA_ERR_ARG;
+  *device_status = 0;
+  cudaError_t e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e);
+  if (c->ws == nullptr) return LSA_OK;
+  e = cudaMemcpyAsync(device_status, c->ws, sizeof(int), cudaMemcpyDeviceToHost, c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->ws, 0, sizeof(int), c->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+  return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
+}
+
+const char* lsa_strerror(int err) {
+  switch (err) {
+    case LSA_OK: return "ok";
+    case LSA_ERR_ARG: return "invalid argument";
+    case LSA_ERR_SHAPE: return "unsupported shape or alignment";
+    case LSA_ERR_WORKSPACE: return "workspace missing or too small";
+    case LSA_ERR_CUDA: return "CUDA runtime error";
+    case LSA_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown error";
+  }
+}
+
+const char* lsa_last_cuda_error(lsa_ctx* c) { return c ? c->cuda_msg : ""; }
+int64_t lsa_launch_count(lsa_ctx* c) { return c ? c->launches : 0; }
+
+int lsa_block_means(lsa_ctx* c, const lsa_params* p, const void* k_idx, const float* k_scale, int64_t n_key,
+                    const int32_t* page_table, int64_t page_table_stride, const int32_t* ctx_len, int batch,
+                    void* kmean) {
+  if (c == nullptr) return LSA_ERR_ARG;
+  int r = check_params(p, true, false);
+  if (r != LSA_OK) return r;
+  if (k_idx == nullptr || kmean == nullptr || n_key < 0) return LSA_ERR_ARG;
+  if (p->key_dtype == LSA_KEY_E4M3 && k_scale == nullptr) return LSA_ERR_ARG;
+  if (p->paged && (page_table == nullptr || ctx_len == nullptr || batch <= 0 || page_table_stride <= 0)) return LSA_ERR_ARG;
+  if (!aligned16(k_idx) || !aligned16(kmean)) return LSA_ERR_SHAPE;
+  cudaError_t e = lsa::launch_block_means(p->d_idx, p->key_dtype == LSA_KEY_E4M3, p->sub_block, p->kv_page, k_idx,
+                                          k_scale, n_key, p->paged ? page_table : nullptr, page_table_stride,
+                                          ctx_len, batch, kmean, c->stream, &c->launches);
+  return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
+}
+
+int lsa_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w, const void* k_idx,
+              const float* k_scale, const void* kmean, int64_t q_pos0, int64_t n_query, int64_t n_key,
+              const int32_t* page_table, int64_t page_table_stride, const int32_t* ctx_len, int batch,
+              int32_t* sparse_idx, int32_t* n_sparse, int32_t* pages_out) {
+  if (c == nullptr) return LSA_ERR_ARG;
+  int r = check_params(p, true, false);
+  if (r != LSA_OK) return r;
+  if (q_idx == nullptr || w == nullptr || k_idx == nullptr || sparse_idx == nullptr || n_sparse == nullptr) return LSA_ERR_ARG;
+  if (p->hi_enable && kmean == nullptr) return LSA_ERR_ARG;
+  if (p->key_dtype == LSA_KEY_E4M3 && k_scale == nullptr) return LSA_ERR_ARG;
+  if (n_query < 0 || n_key < 0 || q_pos0 < 0) return LSA_ERR_ARG;
+  if (p->paged) {
+    if (page_table == nullptr || ctx_len == nullptr || batch <= 0 || page_table_stride <= 0) return LSA_ERR_ARG;
+  } else if (q_pos0 + n_query > n_key) {
+    return LSA_ERR_ARG;
+  }
+  if (!aligned16(q_idx) || !aligned16(w) || !aligned16(k_idx) || (kmean && !aligned16(kmean))) return LSA_ERR_SHAPE;
+  return run_index(c, p, q_idx, w, k_idx, k_scale, kmean, q_pos0, n_query, n_key, page_table, page_table_stride,
+                   ctx_len, batch, sparse_idx, n_sparse, pages_out);
+}
+
+int lsa_select(lsa_ctx* c, const lsa_params* p, const float* scores, int64_t ld_scores, const int32_t* cand_pos,
+               int64_t q_pos0, int64_t n_query, int64_t n_cand, int32_t k, int32_t apply_range, int32_t* idx_out,
+               int32_t* n_out) {
+  if (c == nullptr || p == nullptr || p->struct_size != sizeof(lsa_params)) return LSA_ERR_ARG;
+  if (scores == nullptr || idx_out == nullptr || n_out == nullptr) return LSA_ERR_ARG;
+  if (n_query < 0 || n_cand < 0 || k < 0 || ld_scores < n_cand || q_pos0 < 0) return LSA_ERR_ARG;
+  if (k > 8192 || n_cand > 0x7fffffff) return LSA_ERR_SHAPE;
+  if (n_query == 0 || k == 0) return LSA_OK;
+  cudaError_t e = lsa::launch_select(scores, ld_scores, cand_pos, q_pos0, static_cast<int>(n_query), n_cand, k,
+                                     apply_range, p->k_sink, p->k_swa, idx_out, n_out, c->stream, &c->launches);
+  return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
+}
+
+int lsa_convert(lsa_ctx* c, const lsa_params* p, const int32_t* sparse_idx, const int32_t* n_sparse, int64_t q_pos0,
+                int64_t n_query, const int32_t* page_table, int64_t page_table_stride, const int32_t* ctx_len,
+                int batch, int32_t* rows_out, int32_t* n_rows_out, int32_t* runs_out) {
+  if (c == nullptr || p == nullptr || p->struct_size != sizeof(lsa_params)) return LSA_ERR_ARG;
+  if (sparse_idx == nullptr || n_sparse == nullptr || rows_out == nullptr || n_rows_out == nullptr) return LSA_ERR_ARG;
+  if (p->paged && (page_table == nullptr || ctx_len == nullptr || batch <= 0 || p->kv_page <= 0)) return LSA_ERR_ARG;
+  const int64_t nq = p->paged ? batch : n_query;
+  if (nq < 0 || q_pos0 < 0) return LSA_ERR_ARG;
+  cudaError_t e = lsa::launch_convert(p->k_sink, p->k_swa, p->k_sparse, p->paged, p->kv_page, sparse_idx, n_sparse,
+                                      q_pos0, static_cast<int>(nq), page_table, page_table_stride, ctx_len, rows_out,
+                                      n_rows_out, runs_out, c->stream, &c->launches);
+  return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
+}
+
+int lsa_sparse_attn(lsa_ctx* c, const lsa_params* p, const void* q, const void* k, const void* v, int64_t ld_k,
+                    int64_t ld_v, const int32_t* sparse_idx, const int32_t* n_sparse, const int32_t* rows,
+                    const int32_t* n_rows, int64_t q_pos0, int64_t n_query, int64_t n_key, const int32_t* ctx_len,
+                    int batch, void* out, float* lse) {
+  if (c == nullptr) return LSA_ERR_ARG;
+  int r = check_params(p, false, true);
+  if (r != LSA_OK) return r;
+  if (q == nullptr || k == nullptr || v == nullptr || out == nullptr) return LSA_ERR_ARG;
+  if (rows == nullptr && (sparse_idx == nullptr || n_sparse == nullptr)) return LSA_ERR_ARG;
+  if (rows != nullptr && n_rows == nullptr) return LSA_ERR_ARG;
+  if (p->paged && (rows == nullptr || ctx_len == nullptr || batch <= 0)) return LSA_ERR_ARG;
+  if (n_query < 0 || q_pos0 < 0 || n_key < 0) return LSA_ERR_ARG;
+  if (ld_k < p->d_qk || ld_v < p->d_v || (ld_k % 8) || (ld_v % 8)) return LSA_ERR_SHAPE;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return LSA_ERR_SHAPE;
+  return run_attn(c, p, q, k, v, ld_k, ld_v, sparse_idx, n_sparse, rows, n_rows, q_pos0, n_query, ctx_len, batch, out, lse);
+}
+
+int lsa_layer_group(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w, const void* k_idx,
+                    const float* k_scale, const void* kmean, int64_t q_pos0, int64_t n_query, int64_t n_key,
+                    const int32_t* page_table, int64_t page_table_stride, const int32_t* ctx_len, int batch,
+                    const void* const* q, const void* const* k, const void* const* v, int64_t ld_k, int64_t ld_v,
+                    void* const* out, float* const* lse, int32_t* sparse_idx, int32_t* n_sparse) {
+  if (c == nullptr) return LSA_ERR_ARG;
+  int r = check_params(p, true, true);
+  if (r != LSA_OK) return r;
+  if (p->n_layers <= 0 || q == nullptr || k == nullptr || v == nullptr || out == nullptr) return LSA_ERR_ARG;
+  for (int i = 0; i < p->n_layers; ++i)
+    if (q[i] == nullptr || k[i] == nullptr || v[i] == nullptr || out[i] == nullptr) return LSA_ERR_ARG;
+  r = lsa_index(c, p, q_idx, w, k_idx, k_scale, kmean, q_pos0, n_query, n_key, page_table, page_table_stride,
+                ctx_len, batch, sparse_idx, n_sparse, nullptr);
+  if (r != LSA_OK) return r;
+  const int32_t* rows = nullptr;
+  const int32_t* n_rows = nullptr;
+  if (p->paged) {
+    const WsLayout l = ws_layout(p, batch, page_table_stride * p->kv_page, batch);
+    if (c->ws == nullptr || l.total > c->ws_bytes) return LSA_ERR_WORKSPACE;
+    int32_t* rows_w = reinterpret_cast<int32_t*>(c->ws + l.rows);
+    int32_t* n_rows_w = reinterpret_cast<int32_t*>(c->ws + l.n_rows);
+    r = lsa_convert(c, p, sparse_idx, n_sparse, q_pos0, n_query, page_table, page_table_stride, ctx_len, batch,
+                    rows_w, n_rows_w, nullptr);
+    if (r != LSA_OK) return r;
+    rows = rows_w;
+    n_rows = n_rows_w;
+  }
+  for (int i = 0; i < p->n_layers; ++i) {
+    r = lsa_sparse_attn(c, p, q[i], k[i], v[i], ld_k, ld_v, sparse_idx, n_sparse, rows, n_rows, q_pos0, n_query,
+                        n_key, ctx_len, batch, out[i], lse ? lse[i] : nullptr);
+    if (r != LSA_OK) return r;
+  }
+  return LSA_OK;
+}
+
+int lsa_host_stage_bytes(const lsa_params* p, int64_t sq, size_t* bytes) {
+  if (bytes == nullptr || sq <= 0) return LSA_ERR_ARG;
+  const int r = check_params(p, true, true);
+  if (r != LSA_OK) return r;
+  if (p->paged || p->n_layers <= 0) return LSA_ERR_ARG;
+  size_t off = 0;
+  off += align_up(static_cast<size_t>(sq) * p->n_heads_idx * p->d_idx * 2, 256);
+  off += align_up(static_cast<size_t>(sq) * p->n_heads_idx * 4, 256);
+  off += p->n_layers * align_up(static_cast<size_t>(sq) * p->n_heads * p->d_qk * 2, 256);
+  off += p->n_layers * align_up(static_cast<size_t>(sq) * p->n_heads * p->d_v * 2, 256);
+  off += align_up(static_cast<size_t>(sq) * p->k_sparse * 4, 256);
+  off += align_up(static_cast<size_t>(sq) * 4, 256);
+  *bytes = off;
+  return LSA_OK;
+}
+
+int lsa_layer_group_host(lsa_ctx* c, const lsa_params* p, const void* q_idx_host, const float* w_host,
+                         const void* k_idx, const float* k_scale, const void* kmean, int64_t n_query, int64_t n_key,
+                         const void* const* q_host, const void* const* k, const void* const* v, int64_t ld_k,
+                         int64_t ld_v, void* const* out_host, int64_t sq, void* const* stage, size_t stage_bytes) {
+  if (c == nullptr) return LSA_ERR_ARG;
+  size_t need = 0;
+  int r = lsa_host_stage_bytes(p, sq, &need);
+  if (r != LSA_OK) return r;
+  if (stage == nullptr || stage[0] == nullptr || stage[1] == nullptr || stage_bytes < need) return LSA_ERR_WORKSPACE;
+  if (q_idx_host == nullptr || w_host == nullptr || q_host == nullptr || out_host == nullptr || n_query < 0) return LSA_ERR_ARG;
+  const int R = p->n_layers;
+  if (R > 16) return LSA_ERR_SHAPE;
+  const size_t b_qi = static_cast<size_t>(p->n_heads_idx) * p->d_idx * 2, b_w = static_cast<size_t>(p->n_heads_idx) * 4;
+  const size_t b_q = static_cast<size_t>(p->n_heads) * p->d_qk * 2, b_o = static_cast<size_t>(p->n_heads) * p->d_v * 2;
+  cudaError_t e = cudaSuccess;
+  const int64_t n_pass = (n_query + sq - 1) / sq;
+  // the caller's earlier work on the context stream must be visible to the copy streams
+  e = cudaEventRecord(c->ev_done[0], c->stream);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(c->copy_in, c->ev_done[0], 0);
+  for (int64_t i = 0; i < n_pass && e == cudaSuccess; ++i) {
+    const int s = static_cast<int>(i & 1);
+    const int64_t q0 = i * sq, n = n_query - q0 < sq ? n_query - q0 : sq;
+    uint8_t* base = static_cast<uint8_t*>(stage[s]);
+    size_t off = 0;
+    uint8_t* d_qi = base + off; off += align_up(static_cast<size_t>(sq) * b_qi, 256);
+    uint8_t* d_w = base + off; off += align_up(static_cast<size_t>(sq) * b_w, 256);
+    const void* d_q[16]; void* d_o[16];
+    for (int l = 0; l < R; ++l) { d_q[l] = base + off; off += align_up(static_cast<size_t>(sq) * b_q, 256); }
+    for (int l = 0; l < R; ++l) { d_o[l] = base + off; off += align_up(static_cast<size_t>(sq) * b_o, 256); }
+    int32_t* d_idx = reinterpret_cast<int32_t*>(base + off); off += align_up(static_cast<size_t>(sq) * p->k_sparse * 4, 256);
+    int32_t* d_n = reinterpret_cast<int32_t*>(base + off);
+    // stage s is free once the copy-out of pass i-2 has drained it
+    if (i >= 2) e = cudaStreamWaitEvent(c->copy_in, c->ev_out[s], 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d_qi, static_cast<const uint8_t*>(q_idx_host) + q0 * b_qi, n * b_qi, cudaMemcpyHostToDevice, c->copy_in);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d_w, reinterpret_cast<const uint8_t*>(w_host) + q0 * b_w, n * b_w, cudaMemcpyHostToDevice, c->copy_in);
+    for (int l = 0; l < R && e == cudaSuccess; ++l)
+      e = cudaMemcpyAsync(const_cast<void*>(d_q[l]), static_cast<const uint8_t*>(q_host[l]) + q0 * b_q, n * b_q, cudaMemcpyHostToDevice, c->copy_in);
+    if (e == cudaSuccess) e = cudaEventRecord(c->ev_in[s], c->copy_in);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(c->stream, c->ev_in[s], 0);
+    if (e != cudaSuccess) break;
+    r = lsa_layer_group(c, p, d_qi, reinterpret_cast<const float*>(d_w), k_idx, k_scale, kmean, q0, n, n_key, nullptr,
+                        0, nullptr, 1, d_q, k, v, ld_k, ld_v, d_o, nullptr, d_idx, d_n);
+    if (r != LSA_OK) return r;
+    e = cudaEventRecord(c->ev_done[s], c->stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(c->copy_out, c->ev_done[s], 0);
+    for (int l = 0; l < R && e == cudaSuccess; ++l)
+      e = cudaMemcpyAsync(static_cast<uint8_t*>(out_host[l]) + q0 * b_o, d_o[l], n * b_o, cudaMemcpyDeviceToHost, c->copy_out);
+    if (e == cudaSuccess) e = cudaEventRecord(c->ev_out[s], c->copy_out);
+  }
+  // the context stream finishes only after every copy-out has
+  for (int s = 0; s < 2 && e == cudaSuccess; ++s)
+    if (n_pass > s) e = cudaStreamWaitEvent(c->stream, c->ev_out[(n_pass - 1 - s) & 1], 0);
+  return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
+}
+
+}  // extern "C"

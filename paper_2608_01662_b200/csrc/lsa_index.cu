@@ -1,0 +1,551 @@
+// Indexer kernels: sub-block mean cache (a0), coarse page scores (a1, Eq. 9), page top-M (a2, Eq. 10),
+// fine token scores on the recalled pages (a3, Eq. 11) and top-K_sparse (a4, Eq. 12), the standalone
+// selection (Eq. 2/7) and the streaming-aware conversion of an index set to cache rows (a5, Sec. 3.1).
+//
+// Scoring tiles put 128 keys (or mean keys) on the M axis of the tensor-core tile and the H_I heads of
+// one query on the N axis, so that the ReLU / head-weight / head-sum epilogue of Eq. 1 runs inside one
+// thread quad and one number per key leaves the tile.
+#include "lsa_internal.h"
+#include "lsa_select.cuh"
+
+namespace lsa {
+
+namespace {
+
+constexpr int kTileRows = 128;   // keys per scoring tile
+constexpr int kThreads = 256;    // 8 warps, 16 tile rows each
+
+// ------------------------------------------------------------------------------------------------
+// a0: mean-key cache
+// ------------------------------------------------------------------------------------------------
+template <bool E4M3>
+__global__ void block_means_kernel(const uint8_t* __restrict__ k_idx, const float* __restrict__ k_scale,
+                                   int64_t n_key, int DI, int B, int kv_page,
+                                   const int32_t* __restrict__ page_table, int64_t pt_stride,
+                                   const int32_t* __restrict__ ctx_len, __nv_bfloat16* __restrict__ kmean) {
+  const int U = DI / 8;  // 8 output dims per thread
+  const int64_t gid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int64_t sub = gid / U;
+  const int u = static_cast<int>(gid % U);
+  int64_t row0, out_row;
+  int cnt;
+  if (page_table != nullptr) {
+    const int b = blockIdx.y;
+    const int64_t n = ctx_len[b];
+    if (sub * B >= n) return;
+    const int64_t pos0 = sub * B;
+    const int64_t phys = page_table[b * pt_stride + pos0 / kv_page];
+    row0 = phys * kv_page + pos0 % kv_page;
+    out_row = phys * (kv_page / B) + (pos0 % kv_page) / B;
+    cnt = static_cast<int>(min64(B, n - pos0));
+  } else {
+    if (sub * B >= n_key) return;
+    row0 = sub * B;
+    out_row = sub;
+    cnt = static_cast<int>(min64(B, n_key - row0));
+  }
+  float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  for (int r = 0; r < cnt; ++r) {
+    const int64_t row = row0 + r;
+    if (E4M3) {
+      const uint2 c = *reinterpret_cast<const uint2*>(k_idx + row * DI + u * 8);
+      const float sc = k_scale[row];
+      const uint32_t w[2] = {c.x, c.y};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        __half2_raw h = __nv_cvt_fp8x2_to_halfraw2(
+            static_cast<__nv_fp8x2_storage_t>((w[j >> 1] >> ((j & 1) * 16)) & 0xffff), __NV_E4M3);
+        const float2 f = __half22float2(*reinterpret_cast<__half2*>(&h));
+        acc[2 * j] += f.x * sc;
+        acc[2 * j + 1] += f.y * sc;
+      }
+    } else {
+      const uint4 c = *reinterpret_cast<const uint4*>(k_idx + (row * DI + u * 8) * 2);
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&c);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 f = __bfloat1622float2(h[j]);
+        acc[2 * j] += f.x;
+        acc[2 * j + 1] += f.y;
+      }
+    }
+  }
+  const float inv = static_cast<float>(cnt);
+  uint4 o;
+  o.x = pack_bf16(acc[0] / inv, acc[1] / inv);
+  o.y = pack_bf16(acc[2] / inv, acc[3] / inv);
+  o.z = pack_bf16(acc[4] / inv, acc[5] / inv);
+  o.w = pack_bf16(acc[6] / inv, acc[7] / inv);
+  *reinterpret_cast<uint4*>(kmean + out_row * DI + u * 8) = o;
+}
+
+// ------------------------------------------------------------------------------------------------
+// shared scoring pieces
+// ------------------------------------------------------------------------------------------------
+
+// Copy one query's indexer heads [HI, DI] bf16 (contiguous) into a swizzled shared tile.
+template <int HI, int DI>
+__device__ __forceinline__ void load_q_async(uint32_t dst, const __nv_bfloat16* src) {
+  constexpr int U = DI / 8;
+  for (int e = threadIdx.x; e < HI * U; e += kThreads)
+    cp_async16(dst + swz<DI * 2>(e / U, e % U), reinterpret_cast<const uint8_t*>(src) + e * 16, 16);
+}
+
+// A fragments of this warp's 16 rows of a [128, DI] swizzled tile.
+template <int DI>
+__device__ __forceinline__ void load_a_frags(uint32_t (&a)[DI / 16][4], uint32_t tile) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int row = 16 * warp + (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+  for (int ks = 0; ks < DI / 16; ++ks) ldmatrix_x4(a[ks], tile + swz<DI * 2>(row, 2 * ks + (lane >> 4)));
+}
+
+// Eq. 1 for the warp's rows g and g+8:  sum_j w[j] * relu(row . q_j).  Every lane of a quad gets
+// the finished sums.
+template <int HI, int DI>
+__device__ __forceinline__ void score_16rows(const uint32_t (&a)[DI / 16][4], uint32_t q_tile,
+                                             const float* __restrict__ ws, float& s_lo, float& s_hi) {
+  constexpr int NT = HI / 8, KS = DI / 16;
+  const int lane = threadIdx.x & 31;
+  float acc[NT][4];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) {
+    if constexpr (NT == 1) {
+      uint32_t b[2];
+      ldmatrix_x2(b, q_tile + swz<DI * 2>(lane & 7, 2 * ks + ((lane >> 3) & 1)));
+      mma_bf16(acc[0], a[ks], b[0], b[1]);
+    } else {
+#pragma unroll
+      for (int nt = 0; nt < NT; nt += 2) {
+        uint32_t b[4];
+        ldmatrix_x4(b, q_tile + swz<DI * 2>(8 * nt + (lane & 7) + (lane >> 4) * 8, 2 * ks + ((lane >> 3) & 1)));
+        mma_bf16(acc[nt], a[ks], b[0], b[1]);
+        mma_bf16(acc[nt + 1], a[ks], b[2], b[3]);
+      }
+    }
+  }
+  const int c2 = (lane & 3) * 2;
+  s_lo = 0.f;
+  s_hi = 0.f;
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    const float w0 = ws[8 * nt + c2], w1 = ws[8 * nt + c2 + 1];
+    s_lo = fmaf(w0, fmaxf(acc[nt][0], 0.f), s_lo);
+    s_lo = fmaf(w1, fmaxf(acc[nt][1], 0.f), s_lo);
+    s_hi = fmaf(w0, fmaxf(acc[nt][2], 0.f), s_hi);
+    s_hi = fmaf(w1, fmaxf(acc[nt][3], 0.f), s_hi);
+  }
+  s_lo += __shfl_xor_sync(0xffffffffu, s_lo, 1);
+  s_hi += __shfl_xor_sync(0xffffffffu, s_hi, 1);
+  s_lo += __shfl_xor_sync(0xffffffffu, s_lo, 2);
+  s_hi += __shfl_xor_sync(0xffffffffu, s_hi, 2);
+}
+
+// ------------------------------------------------------------------------------------------------
+// a1: coarse page scores (Eq. 9).  One block = one tile of 128 mean keys x a group of queries.
+// ------------------------------------------------------------------------------------------------
+constexpr int kCoarseQG = 32;  // prefill queries per block
+
+template <int HI, int DI>
+struct CoarseSmem {
+  alignas(128) uint8_t a[kTileRows * DI * 2];
+  alignas(128) uint8_t q[2][HI * DI * 2];
+  float w[2][HI];
+  float sub[kTileRows];
+};
+
+template <int HI, int DI>
+__global__ void __launch_bounds__(kThreads) coarse_score_kernel(IndexArgs p) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  auto& sm = *reinterpret_cast<CoarseSmem<HI, DI>*>(smem_raw);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int spp = p.P / p.B;          // sub-blocks per page
+  const int ppt = kTileRows / spp;    // pages per tile
+  const int64_t sub0 = static_cast<int64_t>(blockIdx.x) * kTileRows;
+  const int64_t page0 = sub0 / spp;
+
+  int q_begin, q_end;
+  int64_t n_key;
+  const int32_t* pt = nullptr;
+  if (p.paged) {
+    q_begin = blockIdx.y;
+    q_end = q_begin + 1;
+    n_key = p.ctx_len[q_begin];
+    pt = p.page_table + q_begin * p.pt_stride;
+  } else {
+    q_begin = blockIdx.y * kCoarseQG;
+    q_end = min(p.n_query, q_begin + kCoarseQG);
+    n_key = p.n_key;
+  }
+  auto pos_of = [&](int qi) -> int64_t { return p.paged ? n_key - 1 : p.q_pos0 + qi; };
+  // A query needs this tile iff the tile's first page is eligible (page0*P <= t-W) and the coarse
+  // stage runs at all for it (more than M eligible pages).
+  const int64_t t_need = max(page0 * p.P + p.W, (static_cast<int64_t>(p.M) + p.S / p.P) * p.P + p.W);
+  if (pos_of(q_end - 1) < t_need) return;
+  int q_first = q_begin;
+  if (!p.paged && t_need - p.q_pos0 > q_begin) q_first = static_cast<int>(t_need - p.q_pos0);
+
+  // ---- mean-key tile -> shared (zero rows past the end of the cache)
+  const int64_t n_sub = (n_key + p.B - 1) / p.B;
+  {
+    constexpr int U = DI / 8;
+    const uint8_t* km = reinterpret_cast<const uint8_t*>(p.kmean);
+    for (int e = tid; e < kTileRows * U; e += kThreads) {
+      const int r = e / U, u = e % U;
+      const int64_t sub = sub0 + r;
+      int64_t src_row = sub;
+      if (p.paged && sub < n_sub) src_row = static_cast<int64_t>(pt[sub / spp]) * spp + sub % spp;
+      cp_async16(smem_u32(sm.a) + swz<DI * 2>(r, u), km + (sub < n_sub ? src_row : 0) * DI * 2 + u * 16,
+                 sub < n_sub ? 16 : 0);
+    }
+  }
+  const __nv_bfloat16* qg = reinterpret_cast<const __nv_bfloat16*>(p.q_idx);
+  auto prefetch_q = [&](int qi, int buf) {
+    load_q_async<HI, DI>(smem_u32(sm.q[buf]), qg + static_cast<int64_t>(qi) * HI * DI);
+    if (tid < HI / 4) cp_async16(smem_u32(&sm.w[buf][tid * 4]), p.w + static_cast<int64_t>(qi) * HI + tid * 4, 16);
+    cp_async_commit();
+  };
+  prefetch_q(q_first, 0);
+  cp_async_wait<0>();
+  __syncthreads();
+  uint32_t a[DI / 16][4];
+  load_a_frags<DI>(a, smem_u32(sm.a));
+
+  for (int qi = q_first; qi < q_end; ++qi) {
+    const int buf = (qi - q_first) & 1;
+    if (qi + 1 < q_end) prefetch_q(qi + 1, buf ^ 1);
+    float s_lo, s_hi;
+    score_16rows<HI, DI>(a, smem_u32(sm.q[buf]), sm.w[buf], s_lo, s_hi);
+    if ((lane & 3) == 0) {
+      sm.sub[16 * warp + (lane >> 2)] = s_lo;
+      sm.sub[16 * warp + (lane >> 2) + 8] = s_hi;
+    }
+    __syncthreads();
+    if (tid < ppt) {
+      const int64_t page = page0 + tid;
+      const int64_t hi = pos_of(qi) - p.W;
+      if (page * p.P <= hi) {
+        float s = 0.f;
+        for (int j = 0; j < spp; ++j) s += sm.sub[tid * spp + j];
+        p.page_scores[static_cast<int64_t>(qi) * p.ps_ld + page] = s;
+      }
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// a2-a4: per query: top-M pages, fine scores on their tokens, top-K_sparse.
+// ------------------------------------------------------------------------------------------------
+constexpr int kMaxSlots = 4096;  // keep_pages * page
+constexpr int kMaxPages = 64;    // keep_pages
+
+template <int HI, int DI>
+struct FineSmem {
+  alignas(128) uint8_t a[2][kTileRows * DI * 2];
+  alignas(128) uint8_t q[HI * DI * 2];
+  float w[HI];
+  uint32_t keys[kMaxSlots];
+  int32_t pages[kMaxPages];
+  SelectScratch sel;
+};
+
+template <int HI, int DI, bool E4M3>
+__global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  auto& sm = *reinterpret_cast<FineSmem<HI, DI>*>(smem_raw);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int qi = blockIdx.x;
+  int64_t t, n_key;
+  const int32_t* pt = nullptr;
+  if (p.paged) {
+    n_key = p.ctx_len[qi];
+    t = n_key - 1;
+    pt = p.page_table + qi * p.pt_stride;
+  } else {
+    n_key = p.n_key;
+    t = p.q_pos0 + qi;
+  }
+  int32_t* out_idx = p.sparse_idx + static_cast<int64_t>(qi) * p.Ksp;
+  int32_t* out_pages = p.pages_out ? p.pages_out + static_cast<int64_t>(qi) * p.M : nullptr;
+  const int64_t lo = p.S, hi = t - p.W;
+  if (hi < lo) {
+    for (int i = tid; i < p.Ksp; i += kThreads) out_idx[i] = -1;
+    if (out_pages) for (int i = tid; i < p.M; i += kThreads) out_pages[i] = -1;
+    if (tid == 0) p.n_sparse[qi] = 0;
+    return;
+  }
+  const int p0 = static_cast<int>(lo / p.P), p1 = static_cast<int>(hi / p.P);
+  const int nE = p1 - p0 + 1;
+  int nP;
+  if (p.hi_enable && nE > p.M) {
+    const float* ps = p.page_scores + static_cast<int64_t>(qi) * p.ps_ld + p0;
+    nP = block_select_topk([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M,
+                           sm.pages, sm.sel);
+  } else {
+    nP = nE;  // host guarantees nE <= kMaxSlots / P here
+    for (int i = tid; i < nP; i += kThreads) sm.pages[i] = p0 + i;
+  }
+  // ---- query heads and weights -> shared
+  load_q_async<HI, DI>(smem_u32(sm.q), reinterpret_cast<const __nv_bfloat16*>(p.q_idx) + static_cast<int64_t>(qi) * HI * DI);
+  if (tid < HI / 4) cp_async16(smem_u32(&sm.w[tid * 4]), p.w + static_cast<int64_t>(qi) * HI + tid * 4, 16);
+  cp_async_commit();
+  __syncthreads();  // sm.pages visible
+  if (out_pages) for (int i = tid; i < p.M; i += kThreads) out_pages[i] = i < nP ? sm.pages[i] : -1;
+
+  const int n_slots = nP * p.P;
+  const int n_tiles = (n_slots + kTileRows - 1) / kTileRows;
+  const int pshift = 31 - __clz(p.P);
+  auto slot_pos = [&](int c) -> int64_t { return static_cast<int64_t>(sm.pages[c >> pshift]) * p.P + (c & (p.P - 1)); };
+  auto phys_row = [&](int64_t pos) -> int64_t {
+    return p.paged ? static_cast<int64_t>(pt[pos >> pshift]) * p.P + (pos & (p.P - 1)) : pos;
+  };
+  const uint8_t* kbase = reinterpret_cast<const uint8_t*>(p.k_idx);
+
+  // Tile loaders.  bf16 keys go global -> shared asynchronously; e4m3 keys are read into registers one
+  // tile ahead, widened to bf16 and stored.
+  constexpr int U = DI / 8;                           // 16-byte bf16 units per row
+  constexpr int CU = DI / 16;                         // 16-byte code units per row (e4m3)
+  constexpr int kCodePerThread = kTileRows * CU / kThreads;
+  uint4 staged[E4M3 ? kCodePerThread : 1];
+  auto issue_tile = [&](int tile, int buf) {
+    if constexpr (E4M3) {
+#pragma unroll
+      for (int j = 0; j < kCodePerThread; ++j) {
+        const int e = tid + j * kThreads, r = e / CU, u = e % CU;
+        const int c = tile * kTileRows + r;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (c < n_slots) {
+          const int64_t pos = slot_pos(c);
+          if (pos < n_key) v = *reinterpret_cast<const uint4*>(kbase + phys_row(pos) * DI + u * 16);
+        }
+        staged[j] = v;
+      }
+    } else {
+      for (int e = tid; e < kTileRows * U; e += kThreads) {
+        const int r = e / U, u = e % U;
+        const int c = tile * kTileRows + r;
+        bool ok = c < n_slots;
+        int64_t pos = 0;
+        if (ok) {
+          pos = slot_pos(c);
+          ok = pos < n_key;
+        }
+        cp_async16(smem_u32(sm.a[buf]) + swz<DI * 2>(r, u), kbase + (ok ? phys_row(pos) : 0) * DI * 2 + u * 16,
+                   ok ? 16 : 0);
+      }
+      cp_async_commit();
+    }
+  };
+  auto land_tile = [&](int buf) {
+    if constexpr (E4M3) {
+#pragma unroll
+      for (int j = 0; j < kCodePerThread; ++j) {
+        const int e = tid + j * kThreads, r = e / CU, u = e % CU;
+        uint4 lo16, hi16;
+        e4m3x16_to_bf16(staged[j], lo16, hi16);
+        *reinterpret_cast<uint4*>(sm.a[buf] + swz<DI * 2>(r, 2 * u)) = lo16;
+        *reinterpret_cast<uint4*>(sm.a[buf] + swz<DI * 2>(r, 2 * u + 1)) = hi16;
+      }
+    }
+  };
+
+  issue_tile(0, 0);
+  for (int tile = 0; tile < n_tiles; ++tile) {
+    const int buf = tile & 1;
+    land_tile(buf);
+    cp_async_wait<0>();
+    __syncthreads();  // tile `tile` (and, first time, q/w) in shared; buffer buf^1 free
+    if (tile + 1 < n_tiles) issue_tile(tile + 1, buf ^ 1);
+    uint32_t a[DI / 16][4];
+    load_a_frags<DI>(a, smem_u32(sm.a[buf]));
+    float s_lo, s_hi;
+    score_16rows<HI, DI>(a, smem_u32(sm.q), sm.w, s_lo, s_hi);
+    if ((lane & 3) == 0) {
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const int c = tile * kTileRows + 16 * warp + (lane >> 2) + 8 * half;
+        if (c < n_slots) {
+          const int64_t pos = slot_pos(c);
+          uint32_t key = 0;
+          if (pos >= lo && pos <= hi) {
+            float s = half ? s_hi : s_lo;
+            if constexpr (E4M3) s *= p.k_scale[phys_row(pos)];
+            key = score_key(s);
+          }
+          sm.keys[c] = key;
+        }
+      }
+    }
+  }
+  __syncthreads();
+  const int n_sel = block_select_topk([&](int i) { return sm.keys[i]; },
+                                      [&](int i) { return static_cast<int>(slot_pos(i)); }, n_slots, p.Ksp, out_idx,
+                                      sm.sel);
+  if (tid == 0) p.n_sparse[qi] = n_sel;
+}
+
+// ------------------------------------------------------------------------------------------------
+// standalone selection on caller-given scores
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __restrict__ scores, int64_t ld,
+                                                            const int32_t* __restrict__ cand_pos, int64_t q_pos0,
+                                                            int64_t n_cand, int k, int apply_range, int S, int W,
+                                                            int32_t* __restrict__ idx_out, int32_t* __restrict__ n_out) {
+  __shared__ SelectScratch sc;
+  const int qi = blockIdx.x;
+  const float* row = scores + qi * ld;
+  const int32_t* pos = cand_pos ? cand_pos + qi * n_cand : nullptr;
+  const int64_t lo = S, hi = q_pos0 + qi - W;
+  auto id = [&](int i) { return pos ? pos[i] : i; };
+  auto key = [&](int i) -> uint32_t {
+    const int64_t s = id(i);
+    if (s < 0) return 0u;
+    if (apply_range && (s < lo || s > hi)) return 0u;
+    return score_key(row[i]);
+  };
+  const int n = block_select_topk(key, id, static_cast<int>(n_cand), k, idx_out + static_cast<int64_t>(qi) * k, sc);
+  if (threadIdx.x == 0) n_out[qi] = n;
+}
+
+// ------------------------------------------------------------------------------------------------
+// a5: index set -> cache rows  [sink run | sparse ascending | window run]
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) convert_kernel(int S, int W, int Ksp, int paged, int kv_page,
+                                                     const int32_t* __restrict__ sparse_idx,
+                                                     const int32_t* __restrict__ n_sparse, int64_t q_pos0,
+                                                     const int32_t* __restrict__ page_table, int64_t pt_stride,
+                                                     const int32_t* __restrict__ ctx_len,
+                                                     int32_t* __restrict__ rows_out, int32_t* __restrict__ n_rows_out,
+                                                     int32_t* __restrict__ runs_out) {
+  const int qi = blockIdx.x, tid = threadIdx.x;
+  const int64_t t = paged ? ctx_len[qi] - 1 : q_pos0 + qi;
+  const int32_t* pt = paged ? page_table + qi * pt_stride : nullptr;
+  const int n_sink = static_cast<int>(min64(S, t + 1));
+  const int64_t win0 = max64(S, t - W + 1);
+  const int n_win = static_cast<int>(max64(0, t - win0 + 1));
+  const int n_sp = n_sparse[qi];
+  const int n_tot = n_sink + n_sp + n_win;
+  const int ld = S + Ksp + W;
+  int32_t* out = rows_out + static_cast<int64_t>(qi) * ld;
+  auto row_of = [&](int i) -> int32_t {
+    int64_t pos;
+    if (i < n_sink) pos = i;
+    else if (i < n_sink + n_sp) pos = sparse_idx[static_cast<int64_t>(qi) * Ksp + i - n_sink];
+    else pos = win0 + (i - n_sink - n_sp);
+    return static_cast<int32_t>(paged ? static_cast<int64_t>(pt[pos / kv_page]) * kv_page + pos % kv_page : pos);
+  };
+  int breaks = 0;
+  for (int i = tid; i < ld; i += 128) {
+    int32_t r = -1;
+    if (i < n_tot) {
+      r = row_of(i);
+      if (i == 0 || row_of(i - 1) + 1 != r) ++breaks;
+    }
+    out[i] = r;
+  }
+  if (tid == 0) n_rows_out[qi] = n_tot;
+  if (runs_out != nullptr) {
+    __shared__ int sh[4];
+    breaks = __reduce_add_sync(0xffffffffu, breaks);
+    if ((tid & 31) == 0) sh[tid >> 5] = breaks;
+    __syncthreads();
+    if (tid == 0) {
+      int32_t* ro = runs_out + static_cast<int64_t>(qi) * 4;
+      ro[0] = n_sink;
+      ro[1] = n_sp;
+      ro[2] = n_win;
+      ro[3] = sh[0] + sh[1] + sh[2] + sh[3];
+    }
+  }
+}
+
+template <class K>
+cudaError_t set_smem(K kernel, size_t bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+}
+
+}  // namespace
+
+bool index_shape_supported(int HI, int DI) { return (HI == 8 && DI == 64) || (HI == 64 && DI == 128); }
+
+cudaError_t launch_block_means(int DI, int key_e4m3, int B, int kv_page, const void* k_idx, const float* k_scale,
+                               int64_t n_key, const int32_t* page_table, int64_t pt_stride,
+                               const int32_t* ctx_len, int batch, void* kmean, cudaStream_t st, int64_t* n_launch) {
+  const int U = DI / 8;
+  // paged: upper bound on sub-blocks per sequence is pt_stride * kv_page / B
+  const int64_t n_sub = page_table ? pt_stride * kv_page / B : (n_key + B - 1) / B;
+  if (n_sub == 0) return cudaSuccess;
+  const int threads = 256;
+  dim3 grid(static_cast<unsigned>((n_sub * U + threads - 1) / threads), page_table ? batch : 1);
+  auto* kp = reinterpret_cast<const uint8_t*>(k_idx);
+  auto* km = reinterpret_cast<__nv_bfloat16*>(kmean);
+  if (key_e4m3)
+    block_means_kernel<true><<<grid, threads, 0, st>>>(kp, k_scale, n_key, DI, B, kv_page, page_table, pt_stride, ctx_len, km);
+  else
+    block_means_kernel<false><<<grid, threads, 0, st>>>(kp, k_scale, n_key, DI, B, kv_page, page_table, pt_stride, ctx_len, km);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+template <int HI, int DI>
+static cudaError_t launch_coarse_t(const IndexArgs& a, int64_t n_key_max, cudaStream_t st, int64_t* n_launch) {
+  const size_t smem = sizeof(CoarseSmem<HI, DI>);
+  cudaError_t e = set_smem(coarse_score_kernel<HI, DI>, smem);
+  if (e != cudaSuccess) return e;
+  const int64_t n_sub = (n_key_max + a.B - 1) / a.B;
+  dim3 grid(static_cast<unsigned>((n_sub + kTileRows - 1) / kTileRows),
+            a.paged ? a.n_query : (a.n_query + kCoarseQG - 1) / kCoarseQG);
+  coarse_score_kernel<HI, DI><<<grid, kThreads, smem, st>>>(a);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_coarse(const IndexArgs& a, cudaStream_t st, int64_t* n_launch) {
+  // key tiles that any query can need: up to the largest cached length
+  const int64_t n_key_max = a.paged ? a.pt_stride * a.P : a.n_key;
+  if (a.HI == 8 && a.DI == 64) return launch_coarse_t<8, 64>(a, n_key_max, st, n_launch);
+  return launch_coarse_t<64, 128>(a, n_key_max, st, n_launch);
+}
+
+template <int HI, int DI, bool E4M3>
+static cudaError_t launch_fine_t(const IndexArgs& a, cudaStream_t st, int64_t* n_launch) {
+  const size_t smem = sizeof(FineSmem<HI, DI>);
+  cudaError_t e = set_smem(fine_select_kernel<HI, DI, E4M3>, smem);
+  if (e != cudaSuccess) return e;
+  fine_select_kernel<HI, DI, E4M3><<<a.n_query, kThreads, smem, st>>>(a);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_fine_select(const IndexArgs& a, cudaStream_t st, int64_t* n_launch) {
+  if (a.n_query == 0) return cudaSuccess;
+  if (a.HI == 8 && a.DI == 64)
+    return a.key_e4m3 ? launch_fine_t<8, 64, true>(a, st, n_launch) : launch_fine_t<8, 64, false>(a, st, n_launch);
+  return a.key_e4m3 ? launch_fine_t<64, 128, true>(a, st, n_launch) : launch_fine_t<64, 128, false>(a, st, n_launch);
+}
+
+cudaError_t launch_select(const float* scores, int64_t ld, const int32_t* cand_pos, int64_t q_pos0, int n_query,
+                          int64_t n_cand, int k, int apply_range, int S, int W, int32_t* idx_out, int32_t* n_out,
+                          cudaStream_t st, int64_t* n_launch) {
+  if (n_query == 0) return cudaSuccess;
+  select_kernel<<<n_query, kSelThreads, 0, st>>>(scores, ld, cand_pos, q_pos0, n_cand, k, apply_range, S, W, idx_out, n_out);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_convert(int S, int W, int Ksp, int paged, int kv_page, const int32_t* sparse_idx,
+                           const int32_t* n_sparse, int64_t q_pos0, int n_query, const int32_t* page_table,
+                           int64_t pt_stride, const int32_t* ctx_len, int32_t* rows_out, int32_t* n_rows_out,
+                           int32_t* runs_out, cudaStream_t st, int64_t* n_launch) {
+  if (n_query == 0) return cudaSuccess;
+  convert_kernel<<<n_query, 128, 0, st>>>(S, W, Ksp, paged, kv_page, sparse_idx, n_sparse, q_pos0, page_table,
+                                          pt_stride, ctx_len, rows_out, n_rows_out, runs_out);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+}  // namespace lsa

@@ -1,0 +1,72 @@
+// Host-side launcher interface between the C ABI (lsa_api.cu) and the kernel files.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace lsa {
+
+struct IndexArgs {
+  int HI, DI, key_e4m3, P, B, M, Ksp, S, W, hi_enable, paged;
+  const void* q_idx;      // bf16 [n_query, HI, DI]
+  const float* w;         // [n_query, HI]
+  const void* k_idx;      // bf16 or e4m3 codes, rows of DI
+  const float* k_scale;   // per token, e4m3 only
+  const void* kmean;      // bf16 rows of DI
+  int64_t q_pos0;
+  int n_query;
+  int64_t n_key;
+  const int32_t* page_table;
+  int64_t pt_stride;
+  const int32_t* ctx_len;
+  float* page_scores;     // [n_query, ps_ld]
+  int ps_ld;
+  int32_t* sparse_idx;    // [n_query, Ksp]
+  int32_t* n_sparse;
+  int32_t* pages_out;     // optional [n_query, M]
+  int* status;
+};
+
+struct AttnArgs {
+  int H, DQK, DV, S, W, Ksp, paged;
+  float sm_scale;
+  const void* q;          // bf16 [n_query, H, DQK]
+  const void* k;          // bf16 rows of ld_k
+  const void* v;          // bf16 rows of ld_v
+  int64_t ld_k, ld_v;
+  const int32_t* sparse_idx;
+  const int32_t* n_sparse;
+  const int32_t* rows;    // optional [n_query, rows_ld]
+  const int32_t* n_rows;
+  int rows_ld;
+  int64_t q_pos0;
+  int n_query;
+  const int32_t* ctx_len;
+  void* out;              // bf16 [n_query, H, DV]
+  float* lse;             // optional [n_query, H]
+  int n_split;            // >1: partial results in part_out / part_lse, merged afterwards
+  float* part_out;        // fp32 [n_query, n_split, H, DV]
+  float* part_lse;        // fp32 [n_query, n_split, H]
+  int* status;
+};
+
+// Each launcher returns the cudaError_t of its launches and adds the number of kernels it
+// launched to *n_launch.
+cudaError_t launch_block_means(int DI, int key_e4m3, int B, int kv_page, const void* k_idx, const float* k_scale,
+                               int64_t n_key, const int32_t* page_table, int64_t pt_stride,
+                               const int32_t* ctx_len, int batch, void* kmean, cudaStream_t st, int64_t* n_launch);
+cudaError_t launch_coarse(const IndexArgs& a, cudaStream_t st, int64_t* n_launch);
+cudaError_t launch_fine_select(const IndexArgs& a, cudaStream_t st, int64_t* n_launch);
+cudaError_t launch_select(const float* scores, int64_t ld, const int32_t* cand_pos, int64_t q_pos0, int n_query,
+                          int64_t n_cand, int k, int apply_range, int S, int W, int32_t* idx_out, int32_t* n_out,
+                          cudaStream_t st, int64_t* n_launch);
+cudaError_t launch_convert(int S, int W, int Ksp, int paged, int kv_page, const int32_t* sparse_idx,
+                           const int32_t* n_sparse, int64_t q_pos0, int n_query, const int32_t* page_table,
+                           int64_t pt_stride, const int32_t* ctx_len, int32_t* rows_out, int32_t* n_rows_out,
+                           int32_t* runs_out, cudaStream_t st, int64_t* n_launch);
+cudaError_t launch_attn(const AttnArgs& a, cudaStream_t st, int64_t* n_launch);
+
+bool index_shape_supported(int HI, int DI);
+bool attn_shape_supported(int H, int DQK, int DV);
+
+}  // namespace lsa

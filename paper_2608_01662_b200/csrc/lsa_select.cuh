@@ -1,0 +1,149 @@
+// Block-wide exact top-k by radix select, with ordered compaction.
+//
+// Items i = 0..n-1 carry a 32-bit key (larger = better, 0 = absent) and appear in ascending id
+// order.  The k items that are largest under (key descending, i ascending) are written in
+// ascending i.  Four 8-bit histogram passes find the k-th largest key T; everything above T is
+// taken, and of the items equal to T the first (k - #above) in index order.
+#pragma once
+
+#include "lsa_common.cuh"
+
+namespace lsa {
+
+constexpr int kSelThreads = 256;
+constexpr int kSelWarps = kSelThreads / 32;
+
+struct SelectScratch {
+  uint32_t hist[kSelWarps][256];
+  uint32_t warp_gt[kSelWarps];
+  uint32_t warp_eq[kSelWarps];
+  uint32_t prefix;
+  uint32_t remaining;
+  uint32_t n_valid;
+};
+
+// KeyF: uint32_t operator()(int i).   IdF: int operator()(int i).
+// Every thread of the 256-thread block must call this.  Returns the number of items written
+// (min(k, #present)); out[written..k) is filled with -1.
+template <class KeyF, class IdF>
+__device__ int block_select_topk(KeyF key, IdF id, int n, int k, int* out, SelectScratch& sc) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  // ---- how many items are present
+  uint32_t cnt = 0;
+  for (int i = tid; i < n; i += kSelThreads) cnt += key(i) != 0u;
+  cnt = __reduce_add_sync(0xffffffffu, cnt);
+  if (lane == 0) sc.warp_gt[warp] = cnt;
+  __syncthreads();
+  if (tid == 0) {
+    uint32_t s = 0;
+    for (int w = 0; w < kSelWarps; ++w) s += sc.warp_gt[w];
+    sc.n_valid = s;
+  }
+  __syncthreads();
+  const int n_valid = static_cast<int>(sc.n_valid);
+  uint32_t T = 0;      // take keys > T ...
+  int need_eq = 0;     // ... and the first need_eq keys == T
+  if (k <= 0 || n_valid == 0) {
+    for (int i = tid; i < k; i += kSelThreads) out[i] = -1;
+    __syncthreads();
+    return 0;
+  }
+  if (n_valid > k) {
+    uint32_t prefix = 0, mask = 0;
+    uint32_t remaining = static_cast<uint32_t>(k);
+#pragma unroll 1
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      for (int i = tid; i < kSelWarps * 256; i += kSelThreads) (&sc.hist[0][0])[i] = 0;
+      __syncthreads();
+      for (int i = tid; i < n; i += kSelThreads) {
+        const uint32_t kk = key(i);
+        if (kk != 0u && (kk & mask) == prefix) atomicAdd(&sc.hist[warp][(kk >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (warp == 0) {
+        // lane l owns bins 255-8l .. 248-8l (descending); find the bin where the running count
+        // from the top reaches `remaining`
+        uint32_t mine[8], tot = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int b = 255 - 8 * lane - j;
+          uint32_t s = 0;
+#pragma unroll
+          for (int w = 0; w < kSelWarps; ++w) s += sc.hist[w][b];
+          mine[j] = s;
+          tot += s;
+        }
+        uint32_t incl = tot;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
+          if (lane >= d) incl += v;
+        }
+        const uint32_t excl = incl - tot;
+        if (excl < remaining && remaining <= incl) {
+          uint32_t run = excl;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            if (run < remaining && remaining <= run + mine[j]) {
+              sc.prefix = prefix | (static_cast<uint32_t>(255 - 8 * lane - j) << shift);
+              sc.remaining = remaining - run;
+            }
+            run += mine[j];
+          }
+        }
+      }
+      __syncthreads();
+      prefix = sc.prefix;
+      remaining = sc.remaining;
+      mask |= 255u << shift;
+      __syncthreads();
+    }
+    T = prefix;
+    need_eq = static_cast<int>(remaining);
+  }
+
+  // ---- ordered compaction: warp w owns the contiguous index range [w*per, (w+1)*per)
+  const int per = ((n + kSelWarps - 1) / kSelWarps + 31) & ~31;
+  const int begin = warp * per, end = min(n, begin + per);
+  uint32_t gt = 0, eq = 0;
+  for (int i = begin + lane; i < end; i += 32) {
+    const uint32_t kk = key(i);
+    gt += kk > T;
+    eq += (kk == T) & (kk != 0u);
+  }
+  gt = __reduce_add_sync(0xffffffffu, gt);
+  eq = __reduce_add_sync(0xffffffffu, eq);
+  if (lane == 0) {
+    sc.warp_gt[warp] = gt;
+    sc.warp_eq[warp] = eq;
+  }
+  __syncthreads();
+  int gt_before = 0, eq_before = 0;
+  for (int w = 0; w < warp; ++w) {
+    gt_before += static_cast<int>(sc.warp_gt[w]);
+    eq_before += static_cast<int>(sc.warp_eq[w]);
+  }
+  int out_run = gt_before + min(eq_before, need_eq);
+  int eq_run = eq_before;
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  for (int base = begin; base < end; base += 32) {
+    const int i = base + lane;
+    const uint32_t kk = i < end ? key(i) : 0u;
+    const bool is_gt = kk > T;
+    const bool is_eq = (kk == T) && (kk != 0u);
+    const uint32_t eq_mask = __ballot_sync(0xffffffffu, is_eq);
+    const int my_eq_rank = eq_run + __popc(eq_mask & lt_mask);
+    const bool sel = is_gt || (is_eq && my_eq_rank < need_eq);
+    const uint32_t sel_mask = __ballot_sync(0xffffffffu, sel);
+    if (sel) out[out_run + __popc(sel_mask & lt_mask)] = id(i);
+    out_run += __popc(sel_mask);
+    eq_run += __popc(eq_mask);
+  }
+  const int written = min(k, n_valid);
+  for (int i = written + tid; i < k; i += kSelThreads) out[i] = -1;
+  __syncthreads();
+  return written;
+}
+
+}  // namespace lsa

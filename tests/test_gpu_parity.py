@@ -1,0 +1,230 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle (needs a B200)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import lsa_oracle as orc
+from paper_2608_01662_b200 import binding
+from paper_2608_01662_b200.configs import CONFIGS
+from paper_2608_01662_b200.workload import DecodeWorkload, PrefillWorkload
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+SMALL_MLA = CONFIGS["cfg2"].replace(name="mla_small", L=4096, M=16, Ksp=512, W=256, seed=11)
+SMALL_FP8 = CONFIGS["cfg3"].replace(name="fp8_small", L=6000, M=8, Ksp=512, W=384, R=2, seed=12)
+SMALL_DEC = CONFIGS["cfg4"].replace(name="dec_small", batch=6, ctx_lo=1500, ctx_hi=6000, M=16, Ksp=512, R=2, seed=13)
+
+
+def _sel_params(S=0, W=0):
+    return binding.make_params(CONFIGS["cfg1"].replace(S=S, W=W))
+
+
+# ---------------------------------------------------------------- selection alone: bit exact
+@pytest.mark.parametrize("n_cand,k", [(1, 1), (37, 8), (1000, 256), (4096, 2048), (5000, 5000), (70000, 2048), (300, 512)])
+def test_select_is_bit_exact_on_given_scores(cuda_device, n_cand, k):
+    g = torch.Generator(device="cpu").manual_seed(n_cand * 7 + k)
+    n_query = 9
+    scores = torch.randn(n_query, n_cand, generator=g)
+    scores[:, ::5] = torch.round(scores[:, ::5] * 2) / 2          # many exact ties
+    scores[1] = 0.0
+    scores[2, ::2] = -0.0                                          # +0 / -0 are one value
+    scores[3] = -scores[3].abs()
+    params = _sel_params()
+    ctx = binding.Context(params, n_query, n_cand, device=cuda_device)
+    d_scores = scores.to(cuda_device)
+    idx = torch.empty((n_query, k), dtype=torch.int32, device=cuda_device)
+    cnt = torch.empty((n_query,), dtype=torch.int32, device=cuda_device)
+    ctx.select(d_scores, None, 0, k, False, idx, cnt)
+    assert ctx.status() == 0
+    idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+    for i in range(n_query):
+        want = orc.select_fp32(scores[i].numpy(), None, 0, k, apply_range=False)
+        assert cnt[i] == len(want)
+        assert np.array_equal(idx[i, :cnt[i]], want) and (idx[i, cnt[i]:] == -1).all()
+
+
+def test_select_with_positions_range_and_leading_dimension(cuda_device):
+    rng = np.random.default_rng(5)
+    n_query, n_cand, ld, k, S, W, q_pos0 = 16, 700, 768, 100, 4, 64, 500
+    scores = torch.from_numpy(np.round(rng.standard_normal((n_query, ld)), 1).astype(np.float32))
+    params = _sel_params(S, W)
+    ctx = binding.Context(params, n_query, 4096, device=cuda_device)
+    idx = torch.empty((n_query, k), dtype=torch.int32, device=cuda_device)
+    cnt = torch.empty((n_query,), dtype=torch.int32, device=cuda_device)
+    d_scores = scores.to(cuda_device)[:, :n_cand]                 # row stride 768, 700 columns
+    ctx.select(d_scores, None, q_pos0, k, True, idx, cnt)
+    for i in range(n_query):
+        want = orc.select_fp32(scores[i, :n_cand].numpy(), None, q_pos0 + i, k, apply_range=True, S=S, W=W)
+        assert np.array_equal(idx[i, :int(cnt[i])].cpu().numpy(), want)
+    # explicit candidate positions with holes, ascending per row
+    pos = np.sort(rng.permutation(5000)[:n_query * n_cand].reshape(n_query, n_cand), axis=1).astype(np.int32)
+    pos[:, ::9] = -1
+    d_pos = torch.from_numpy(pos).to(cuda_device)
+    d_sc = scores[:, :n_cand].contiguous().to(cuda_device)
+    ctx.select(d_sc, d_pos, 0, k, False, idx, cnt)
+    for i in range(n_query):
+        want = orc.select_fp32(scores[i, :n_cand].numpy(), pos[i], 0, k, apply_range=False)
+        assert np.array_equal(idx[i, :int(cnt[i])].cpu().numpy(), want)
+    assert ctx.status() == 0
+
+
+# ---------------------------------------------------------------- mean cache
+@pytest.mark.parametrize("cfg", [CONFIGS["cfg1"], SMALL_FP8], ids=lambda c: c.name)
+def test_block_means_match_oracle(cuda_device, cfg):
+    wl = PrefillWorkload(cfg, cuda_device)
+    wl.prepare()
+    k_hat = (orc.dequant_keys(pu.to_np(wl.keys["k"]), pu.to_np(wl.keys["scale"])) if "scale" in wl.keys
+             else pu.to_np(wl.keys["k"]).astype(np.float64))
+    want = orc.block_means(k_hat, cfg.B)
+    got = pu.to_np(wl.kmean).astype(np.float64)
+    assert got.shape == want.shape
+    # fp32 accumulation then one rounding vs fp64 then one rounding: equal except rare 1-ulp ties
+    diff = got != want
+    assert diff.mean() < 2e-3
+    assert np.abs(got - want).max() <= np.abs(want).max() * 2.0 ** -7
+
+
+# ---------------------------------------------------------------- whole path, small shapes
+def test_cfg1_every_query(cuda_device):
+    cfg = CONFIGS["cfg1"]
+    wl = PrefillWorkload(cfg, cuda_device)
+    wl.prepare()
+    pages = torch.empty((cfg.L, cfg.M), dtype=torch.int32, device=cuda_device)
+    wl.index(pages)
+    sparse_from_index = wl.sparse_idx.clone()
+    wl.step()
+    assert wl.ctx.status() == 0
+    assert torch.equal(sparse_from_index, wl.sparse_idx)          # the group runs the same indexer
+    m = pu.check_prefill(wl, range(cfg.L), pages=pages)
+    print("cfg1", m.summary())
+    m.assert_ok(pu.TOL_BF16)
+
+
+@pytest.mark.parametrize("cfg", [SMALL_MLA, SMALL_FP8], ids=lambda c: c.name)
+def test_small_mla_prefill(cuda_device, cfg):
+    wl = PrefillWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.step()
+    assert wl.ctx.status() == 0
+    m = pu.check_prefill(wl, pu.boundary_queries(cfg, 0, cfg.L, 60, seed=1))
+    print(cfg.name, m.summary())
+    m.assert_ok(pu.TOL_FP8 if cfg.key_dtype == "e4m3" else pu.TOL_BF16)
+
+
+def test_prefill_query_window_with_offset_matches_whole_run(cuda_device):
+    """Queries [q_pos0, q_pos0+n) scored alone (chunked prefill) give the rows of the full run."""
+    cfg = SMALL_MLA.replace(R=1)
+    full = PrefillWorkload(cfg, cuda_device)
+    full.prepare()
+    full.step()
+    part = PrefillWorkload(cfg, cuda_device, q_pos0=3000, n_query=500)
+    part.prepare()
+    part.step()
+    assert torch.equal(part.sparse_idx, full.sparse_idx[3000:3500])
+    assert torch.equal(part.out[0], full.out[0][3000:3500])
+    # q_chunk splits the indexer passes without changing anything
+    chunked = PrefillWorkload(cfg.replace(q_chunk=1000), cuda_device)
+    chunked.prepare()
+    chunked.step()
+    assert torch.equal(chunked.sparse_idx, full.sparse_idx) and torch.equal(chunked.out[0], full.out[0])
+
+
+def test_runs_are_deterministic(cuda_device):
+    wl = PrefillWorkload(SMALL_FP8, cuda_device)
+    wl.prepare()
+    wl.step()
+    idx0, out0 = wl.sparse_idx.clone(), wl.out[1].clone()
+    for _ in range(3):
+        wl.step()
+        assert torch.equal(idx0, wl.sparse_idx) and torch.equal(out0, wl.out[1])
+
+
+def test_small_paged_decode(cuda_device):
+    cfg = SMALL_DEC
+    wl = DecodeWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.step()
+    assert wl.ctx.status() == 0
+    m = pu.check_decode(wl, range(cfg.batch))
+    print(cfg.name, m.summary())
+    m.assert_ok(pu.TOL_FP8)
+
+
+def test_convert_lists_physical_rows(cuda_device):
+    cfg = SMALL_DEC
+    wl = DecodeWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.index()
+    ld = cfg.S + cfg.Ksp + cfg.W
+    rows = torch.empty((cfg.batch, ld), dtype=torch.int32, device=cuda_device)
+    n_rows = torch.empty((cfg.batch,), dtype=torch.int32, device=cuda_device)
+    runs = torch.empty((cfg.batch, 4), dtype=torch.int32, device=cuda_device)
+    wl.ctx.convert(wl.sparse_idx, wl.n_sparse, 0, cfg.batch, rows, n_rows, runs, wl.page_table, wl.ctx_len)
+    table, ctx = pu.to_np(wl.page_table), pu.to_np(wl.ctx_len)
+    for b in range(cfg.batch):
+        t = int(ctx[b]) - 1
+        n_sp = int(wl.n_sparse[b])
+        S_t = orc.index_set(t, cfg.S, cfg.W, pu.to_np(wl.sparse_idx[b])[:n_sp])
+        want = orc.paged_rows(S_t, table[b], cfg.kv_page)
+        got = pu.to_np(rows[b])
+        assert int(n_rows[b]) == len(want) and np.array_equal(got[:len(want)], want) and (got[len(want):] == -1).all()
+        r = pu.to_np(runs[b])
+        assert list(r[:3]) == [cfg.S, n_sp, cfg.W]
+        assert r[3] == 1 + int((np.diff(want) != 1).sum())
+        # the window is whole-page runs: far fewer breaks than rows
+        assert r[3] <= n_sp + cfg.W // cfg.kv_page + 3
+
+
+# ---------------------------------------------------------------- edge cases and errors
+def test_short_sequences_and_empty_calls(cuda_device):
+    cfg = CONFIGS["cfg1"].replace(L=100, name="short")            # L < S + W: every query sees [0, t]
+    wl = PrefillWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.step()
+    assert int(wl.n_sparse.max()) == 0 and (wl.sparse_idx == -1).all()
+    m = pu.check_prefill(wl, range(cfg.L))
+    m.assert_ok(pu.TOL_BF16)
+    # zero queries: nothing is launched, nothing fails
+    n0 = wl.ctx.launch_count()
+    wl.ctx.index(wl.q_idx, wl.w, wl.keys["k"], None, wl.kmean, 0, 0, cfg.L, wl.sparse_idx, wl.n_sparse)
+    assert wl.ctx.launch_count() == n0 and wl.ctx.status() == 0
+
+
+def test_full_candidate_budget_selects_every_candidate(cuda_device):
+    """Ksp >= number of candidates: S_t = [0, t] and the result is dense causal attention."""
+    cfg = CONFIGS["cfg1"].replace(L=600, Ksp=512, M=8, name="dense")
+    wl = PrefillWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.step()
+    n_sp = pu.to_np(wl.n_sparse)
+    for t in range(cfg.L):
+        assert n_sp[t] == max(0, t - cfg.W - cfg.S + 1)
+    q, k, v = pu.to_np(wl.q[0]).astype(np.float64), pu.to_np(wl.k[0]).astype(np.float64), pu.to_np(wl.v[0]).astype(np.float64)
+    tq = torch.from_numpy(q).permute(1, 0, 2)[None]
+    tk = torch.from_numpy(k)[None, None].expand(1, cfg.H, cfg.L, cfg.d_qk)
+    tv = torch.from_numpy(v)[None, None].expand(1, cfg.H, cfg.L, cfg.d_v)
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True, scale=cfg.sm_scale)[0]
+    got = torch.from_numpy(pu.to_np(wl.out[0])).permute(1, 0, 2).to(torch.float64)
+    assert (got - ref).abs().max() <= 2e-2
+    assert ((got - ref).norm() / ref.norm()) <= 5e-3
+
+
+def test_errors_are_codes_not_crashes(cuda_device):
+    cfg = CONFIGS["cfg1"]
+    bad = binding.make_params(cfg.replace(H_I=12))
+    with pytest.raises(binding.LsaError) as e:
+        binding.workspace_bytes(bad, 10, 100)
+    assert e.value.code == -2
+    wl = PrefillWorkload(cfg.replace(L=256, name="err"), cuda_device)
+    with pytest.raises(binding.LsaError) as e:                     # queries beyond the cache
+        wl.ctx.index(wl.q_idx, wl.w, wl.keys["k"], None, wl.kmean, 200, 100, 256, wl.sparse_idx, wl.n_sparse)
+    assert e.value.code == -1
+    small_ws = binding.Context(wl.params, 1, 64, device=cuda_device)
+    with pytest.raises(binding.LsaError) as e:                     # workspace sized for a smaller problem
+        small_ws.index(wl.q_idx, wl.w, wl.keys["k"], None, wl.kmean, 0, 256, 256, wl.sparse_idx, wl.n_sparse)
+    assert e.value.code == -3
+    assert wl.ctx.status() == 0
