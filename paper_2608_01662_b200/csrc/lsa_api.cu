@@ -67,14 +67,11 @@ struct WsLayout {
   int ps_ld, rows_ld;
 };
 
+// The page-score matrix comes last, so that the offsets of the other pieces do not depend on the cache length.
 WsLayout ws_layout(const lsa_params* p, int64_t n_query, int64_t n_key_max, int batch) {
   WsLayout l{};
   size_t off = kStatusBytes;
   const int64_t nq = p->paged ? batch : n_query;
-  const int P = p->page > 0 ? p->page : 64;
-  l.ps_ld = static_cast<int>(align_up(static_cast<size_t>((n_key_max + P - 1) / P), 4));
-  l.page_scores = off;
-  off += align_up(static_cast<size_t>(nq) * l.ps_ld * sizeof(float), 256);
   l.rows_ld = p->k_sink + p->k_sparse + p->k_swa;
   if (p->paged) {
     l.rows = off;
@@ -86,6 +83,10 @@ WsLayout ws_layout(const lsa_params* p, int64_t n_query, int64_t n_key_max, int 
     l.part_lse = off;
     off += align_up(static_cast<size_t>(batch) * kMaxSplit * p->n_heads * sizeof(float), 256);
   }
+  const int P = p->page > 0 ? p->page : 64;
+  l.ps_ld = static_cast<int>(align_up(static_cast<size_t>((n_key_max + P - 1) / P), 4));
+  l.page_scores = off;
+  off += align_up(static_cast<size_t>(nq) * l.ps_ld * sizeof(float), 256);
   l.total = off;
   return l;
 }

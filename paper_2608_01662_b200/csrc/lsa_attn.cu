@@ -185,12 +185,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) sparse_attn_kernel(AttnArgs p
     for (int nt = 0; nt < NTQ; ++nt) {
       const float p0 = exp2f(s[nt][0] - m_new[0]), p1 = exp2f(s[nt][1] - m_new[0]);
       const float p2 = exp2f(s[nt][2] - m_new[1]), p3 = exp2f(s[nt][3] - m_new[1]);
-      // the sums use the bf16-rounded weights that multiply V, so that rows of P/sum add to one
       const uint32_t lo = pack_bf16(p0, p1), hi = pack_bf16(p2, p3);
-      const float2 flo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&lo));
-      const float2 fhi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&hi));
-      sum[0] += flo.x + flo.y;
-      sum[1] += fhi.x + fhi.y;
+      sum[0] += p0 + p1;  // fp32 sums of the unrounded weights: lse stays exact to fp32
+      sum[1] += p2 + p3;
       const int key = grp * 8 * NTQ + 8 * nt + c2;
       *reinterpret_cast<uint32_t*>(sm.p + swz<kKeys * 2>(16 * mt + g, key >> 3) + (key & 7) * 2) = lo;
       *reinterpret_cast<uint32_t*>(sm.p + swz<kKeys * 2>(16 * mt + g + 8, key >> 3) + (key & 7) * 2) = hi;

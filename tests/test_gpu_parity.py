@@ -61,7 +61,7 @@ def test_select_with_positions_range_and_leading_dimension(cuda_device):
         want = orc.select_fp32(scores[i, :n_cand].numpy(), None, q_pos0 + i, k, apply_range=True, S=S, W=W)
         assert np.array_equal(idx[i, :int(cnt[i])].cpu().numpy(), want)
     # explicit candidate positions with holes, ascending per row
-    pos = np.sort(rng.permutation(5000)[:n_query * n_cand].reshape(n_query, n_cand), axis=1).astype(np.int32)
+    pos = np.stack([np.sort(rng.permutation(5000)[:n_cand]) for _ in range(n_query)]).astype(np.int32)
     pos[:, ::9] = -1
     d_pos = torch.from_numpy(pos).to(cuda_device)
     d_sc = scores[:, :n_cand].contiguous().to(cuda_device)
