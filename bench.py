@@ -1,0 +1,383 @@
+#!/usr/bin/env python
+"""Benchmark of the LSA layer-group forward (indexer + sparse attention, one index set reused by R layers).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg3] [--impl reference]
+
+A step is one lsa_layer_group call over the whole synthetic workload (coarse page scores, page
+top-M, fine scores, top-K_sparse, conversion, R attention layers).  Default workload: cfg3, the 128K
+prefill the headline metric is quoted on.  Prints one JSON line (rank 0).  With N > 1 every rank runs
+its own independent sequence (weak scaling, no data-path collective).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "LSA layer-group tokens/sec (128K prefill)"
+UNIT = "tokens/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="cfg3")
+    ap.add_argument("--impl", default="lsa", choices=["lsa", "reference"])
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--cpu-queries", type=int, default=24)
+    return ap.parse_args()
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons every 200 ms while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            time.sleep(0.25)
+            self.proc.terminate()          # the exact child started above
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# algorithmic work
+# ------------------------------------------------------------------------------------------------
+def attn_rows_per_query(cfg, t):
+    n_sink = min(cfg.S, t + 1)
+    n_win = t - max(cfg.S, t - cfg.W + 1) + 1
+    n_sp = min(cfg.Ksp, max(0, t - cfg.W - cfg.S + 1))
+    return n_sink + max(0, n_win) + n_sp
+
+
+def attn_flops_per_launch(cfg, positions):
+    """2*H*(d_qk+d_v) flops per (query, attended row): QK^T and PV of Eq. 3, one layer."""
+    return float(sum(2 * cfg.H * (cfg.d_qk + cfg.d_v) * attn_rows_per_query(cfg, int(t)) for t in positions))
+
+
+def attn_bytes_per_launch(cfg, positions):
+    """Decode: every attended cache row is read once, plus q and out."""
+    rows = sum(attn_rows_per_query(cfg, int(t)) for t in positions)
+    return float(rows * cfg.d_qk * 2 + len(positions) * cfg.H * (cfg.d_qk + cfg.d_v) * 2)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "tensor_tflops": d["bf16_tflops_sustained"], "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tensor_tflops": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(cfg, wl, n_queries, seed=0):
+    """Times the oracle (as it stands) on n_queries sampled queries of the workload: selection plus the R
+    attention layers.  Returns (queries per second, seconds, threads used)."""
+    import numpy as np
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import parity_util as pu
+    from oracle import reference_run as ref
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([i.get("num_threads", 1) for i in threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    rng = np.random.default_rng(seed)
+    kw = dict(P=cfg.P, B=cfg.B, M=cfg.M, Ksp=cfg.Ksp, S=cfg.S, W=cfg.W)
+    if cfg.mode == "prefill":
+        caches = ref.HostCaches(pu.to_np(wl.keys["k"]), pu.to_np(wl.keys["scale"]) if "scale" in wl.keys else None,
+                                [pu.to_np(k) for k in wl.k], [pu.to_np(v) for v in wl.v], cfg.B, n_key=wl.n_key)
+        qs = [int(x) for x in rng.integers(wl.q_pos0, wl.q_pos0 + wl.n_query, n_queries)]
+        host = [(t, pu.to_np(wl.q_idx[t - wl.q_pos0]), pu.to_np(wl.w[t - wl.q_pos0]),
+                 [pu.to_np(q[t - wl.q_pos0]) for q in wl.q]) for t in qs]
+        t0 = time.perf_counter()
+        for t, qi, w, ql in host:
+            sparse, _ = ref.select_query(t, qi, w, caches, hi_enable=cfg.hi_enable, **kw)
+            ref.attend_query(t, ql, caches, sparse, S=cfg.S, W=cfg.W, sm_scale=cfg.sm_scale, d_v=cfg.d_v)
+        dt = time.perf_counter() - t0
+        return len(host) / dt, dt, threads
+    # decode: whole sequences
+    seqs = [(seed + i) % cfg.batch for i in range(min(n_queries, cfg.batch))]
+    dt = 0.0
+    for b in seqs:
+        caches, t = pu.decode_caches(wl, b)            # host copies: not part of the timed work
+        qi, w, ql = pu.to_np(wl.q_idx[b]), pu.to_np(wl.w[b]), [pu.to_np(q[b]) for q in wl.q]
+        t0 = time.perf_counter()
+        sparse, _ = ref.select_query(t, qi, w, caches, hi_enable=cfg.hi_enable, **kw)
+        ref.attend_query(t, ql, caches, sparse, S=cfg.S, W=cfg.W, sm_scale=cfg.sm_scale, d_v=cfg.d_v)
+        dt += time.perf_counter() - t0
+    return len(seqs) / dt, dt, threads
+
+
+# ------------------------------------------------------------------------------------------------
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    from paper_2608_01662_b200.configs import CONFIGS
+    cfg = CONFIGS[args.config]
+    decode = cfg.mode == "decode"
+    metric = "LSA layer-group decode us/step" if decode else METRIC
+    unit = "us/step" if decode else UNIT
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        run_reference(args, cfg, metric, unit, decode)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2608_01662_b200 import build
+    from paper_2608_01662_b200.workload import make_workload
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+
+    # prefill at cfg5 size keeps only one 16384-query chunk of per-query tensors resident
+    kw = {}
+    if not decode and cfg.q_chunk and cfg.L > 262144:
+        kw = dict(q_pos0=cfg.L - cfg.q_chunk, n_query=cfg.q_chunk)
+    wl = make_workload(cfg, dev, with_lse=False, **kw)
+    wl.prepare()
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        wl.step()
+    barrier()
+    assert wl.ctx.status() == 0
+
+    stream = torch.cuda.current_stream(dev)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wl.ctx.profile_enable(not decode)      # event pairs around each kernel class (see lsa_profile_enable)
+    n0 = wl.ctx.launch_count()
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        ev0.record(stream)
+        for _ in range(args.steps):
+            wl.step()
+        ev1.record(stream)
+        barrier()
+    ms = ev0.elapsed_time(ev1)
+    launches = wl.ctx.launch_count() - n0
+    prof = wl.ctx.profile_read() if not decode else None
+    wl.ctx.profile_enable(False)
+    if decode:
+        # the per-kernel event pairs would perturb a ~100 us step: measure them in a second pass
+        wl.ctx.profile_enable(True)
+        for _ in range(args.steps):
+            wl.step()
+        prof = wl.ctx.profile_read()
+        wl.ctx.profile_enable(False)
+
+    t_ms = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
+    ms_max = float(t_ms.item())
+    ms_per_step = ms_max / args.steps
+    units = wl.units() * world
+    value = ms_per_step * 1e3 if decode else units / (ms_per_step * 1e-3)
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel: sparse attention
+    peaks = measured_peaks()
+    import numpy as np
+    if decode:
+        positions = (wl.ctx_len.cpu().numpy().astype(np.int64) - 1)
+    else:
+        positions = np.arange(wl.q_pos0, wl.q_pos0 + wl.n_query)
+    attn_ms, attn_n = prof["sparse_attn"]
+    roofline = None
+    if attn_n > 0:
+        dur_s = attn_ms / attn_n * 1e-3
+        if decode:
+            a = attn_bytes_per_launch(cfg, positions) / dur_s / 1e9
+            roofline = {"kernel": "sparse_attn_kernel", "bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"],
+                        "unit": "GB/s", "frac": a / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                        "launch_ms": attn_ms / attn_n}
+        else:
+            a = attn_flops_per_launch(cfg, positions) / dur_s / 1e12
+            roofline = {"kernel": "sparse_attn_kernel", "bound": "tensor", "achieved": a,
+                        "peak": peaks["tensor_tflops"], "unit": "TFLOP/s", "frac": a / peaks["tensor_tflops"],
+                        "traffic": None, "peak_source": peaks["source"], "launch_ms": attn_ms / attn_n}
+    kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps}
+               for k, v in prof.items() if v[1] > 0}
+
+    # ---- end to end through the host-buffer entry point (prefill only)
+    e2e = None
+    if not args.no_e2e and not decode and world == 1:
+        e2e = run_e2e(args, cfg, wl, dev)
+
+    cpu = None
+    if not args.no_cpu:
+        v, secs, threads = oracle_sample(cfg, wl, args.cpu_queries)
+        cpu = {"value": (1e6 / v) * cfg.batch if decode else v, "unit": unit, "cores": threads, "kind": "oracle",
+               "sample": f"{args.cpu_queries if not decode else min(args.cpu_queries, cfg.batch)} "
+                         f"{'sequences' if decode else 'uniformly sampled queries'} of the same workload, selection + "
+                         f"{cfg.R} attention layers each, {secs:.1f} s"
+                         + ("; value extrapolated to the batch of %d" % cfg.batch if decode else "")}
+
+    line = {
+        "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": not decode,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "mode": cfg.mode, "L": cfg.L, "batch": cfg.batch, "R": cfg.R,
+                   "indexer_keys": cfg.key_dtype, "P": cfg.P, "B": cfg.B, "M": cfg.M, "K_sparse": cfg.Ksp,
+                   "K_sink": cfg.S, "K_swa": cfg.W, "queries_per_step": wl.units(),
+                   "l2": "inputs larger than L2 (per-layer q and out are GBs); no flush" if not decode
+                         else "KV pools are GBs per layer, far larger than L2; no flush"},
+        "clocks": clocks.summary(), "gpu_launches": int(launches), "kernels": kernels,
+        "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_e2e(args, cfg, wl, dev):
+    """Same metric through lsa_layer_group_host: per-query tensors start in pinned host memory, results
+    end there; the caches stay resident (they are state of the sequence, not inputs of the step)."""
+    import torch
+    from paper_2608_01662_b200 import binding
+    n = wl.n_query
+    q_idx_h = wl.q_idx.cpu().pin_memory()
+    w_h = wl.w.cpu().pin_memory()
+    q_h = [q.cpu().pin_memory() for q in wl.q]
+    out_h = [torch.empty(o.shape, dtype=o.dtype).pin_memory() for o in wl.out]
+    sq = 4096
+    nbytes = binding.host_stage_bytes(wl.params, sq)
+    stage = [torch.empty(nbytes, dtype=torch.uint8, device=dev) for _ in range(2)]
+    h2d = q_idx_h.numel() * 2 + w_h.numel() * 4 + sum(q.numel() * 2 for q in q_h)
+    d2h = sum(o.numel() * 2 for o in out_h)
+
+    def step():
+        wl.ctx.layer_group_host(q_idx_h, w_h, wl.keys["k"], wl.keys.get("scale"), wl.kmean, n, wl.n_key, q_h, wl.k,
+                                wl.v, out_h, sq, stage)
+    step()
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream(dev)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(args.e2e_steps):
+        step()
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / args.e2e_steps
+    # the device-resident run must have produced the same bytes
+    same = all(torch.equal(oh[-64:], o[-64:].cpu()) for oh, o in zip(out_h, wl.out))
+    return {"value": n / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+            "ms_per_step": ms, "steps": args.e2e_steps, "matches_device_run": bool(same),
+            "api": "lsa_layer_group_host, pinned host buffers, 4096-query passes"}
+
+
+def run_reference(args, cfg, metric, unit, decode):
+    """The oracle as the reference arm: each step times it on a bounded sample of the workload."""
+    import torch
+    from paper_2608_01662_b200.workload import make_workload
+    dev = torch.device("cuda:0") if torch.cuda.is_available() else torch.device("cpu")
+    # the sample's inputs are drawn by the same generators; only the sampled queries are scored
+    n_q = 4 if not decode else 1
+    kw = {}
+    if not decode:
+        kw = dict(q_pos0=max(0, cfg.L - 4096), n_query=min(cfg.L, 4096))   # late queries: full-size candidate sets
+    wl = make_workload(cfg, dev, with_lse=False, make_ctx=False, **kw)
+    vals, secs_all, threads = [], 0.0, 1
+    for i in range(max(0, args.warmup) + args.steps):
+        v, secs, threads = oracle_sample(cfg, wl, n_q, seed=i)
+        if i >= args.warmup:
+            vals.append(v)
+            secs_all += secs
+    v = len(vals) / sum(1.0 / x for x in vals)              # total queries / total time
+    value = (1e6 / v) * cfg.batch if decode else v
+    sample = (f"{n_q} sampled late queries per step, selection + {cfg.R} attention layers each" if not decode
+              else "1 sequence per step, extrapolated to the batch")
+    print(json.dumps({
+        "impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": secs_all / max(1, args.steps) * 1e3, "higher_is_better": not decode,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "mode": cfg.mode, "L": cfg.L, "batch": cfg.batch, "R": cfg.R},
+        "cpu_baseline": {"value": value, "unit": unit, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+if __name__ == "__main__":
+    main()

@@ -111,6 +111,15 @@ LSA_API const char* lsa_last_cuda_error(lsa_ctx* ctx);
 /* Number of kernels this context has launched since creation (host counter). */
 LSA_API int64_t lsa_launch_count(lsa_ctx* ctx);
 
+/* Per-kernel timing.  While enabled, every kernel-launching call records a CUDA event pair on the
+ * context's stream around the launches of each kernel class (at most 4096 pairs between reads; later
+ * launches go unrecorded).  lsa_profile_read waits for the stream and writes, per class, the summed
+ * device time in ms and the number of recorded launches (host arrays of LSA_K_COUNT entries), then
+ * starts over.  The first enable creates the events (host resources only). */
+enum { LSA_K_MEANS = 0, LSA_K_COARSE, LSA_K_FINE_SELECT, LSA_K_SELECT, LSA_K_CONVERT, LSA_K_ATTN, LSA_K_MERGE, LSA_K_COUNT };
+LSA_API int lsa_profile_enable(lsa_ctx* ctx, int on);
+LSA_API int lsa_profile_read(lsa_ctx* ctx, double* total_ms, int64_t* launches);
+
 /* ---- a0: mean-key cache (Sec. 3.3) ---------------------------------------------------------- */
 
 /* kmean[n, :] = mean over the tokens present in sub-block n of the (dequantised) indexer keys, fp32

@@ -18,6 +18,7 @@ _LIB = None
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblsa.so")
 
 LSA_KEY_BF16, LSA_KEY_E4M3 = 0, 1
+KERNEL_CLASSES = ("block_means", "coarse_score", "fine_select", "select", "convert", "sparse_attn", "merge_splits")
 
 
 class LsaError(RuntimeError):
@@ -42,6 +43,8 @@ EXPORTS = {
     "lsa_strerror": (c_char_p, [c_int]),
     "lsa_last_cuda_error": (c_char_p, [c_void_p]),
     "lsa_launch_count": (c_int64, [c_void_p]),
+    "lsa_profile_enable": (c_int, [c_void_p, c_int]),
+    "lsa_profile_read": (c_int, [c_void_p, POINTER(ctypes.c_double), POINTER(c_int64)]),
     "lsa_block_means": (c_int, [c_void_p, POINTER(LsaParams), c_void_p, c_void_p, c_int64, c_void_p, c_int64,
                                 c_void_p, c_int, c_void_p]),
     "lsa_index": (c_int, [c_void_p, POINTER(LsaParams), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64,
@@ -150,6 +153,16 @@ class Context:
 
     def launch_count(self) -> int:
         return lib().lsa_launch_count(self.h)
+
+    def profile_enable(self, on: bool):
+        self._chk(lib().lsa_profile_enable(self.h, 1 if on else 0), "lsa_profile_enable")
+
+    def profile_read(self) -> dict:
+        """{kernel class: (total ms, launches)} since the last read."""
+        n = len(KERNEL_CLASSES)
+        ms, cnt = (ctypes.c_double * n)(), (c_int64 * n)()
+        self._chk(lib().lsa_profile_read(self.h, ms, cnt), "lsa_profile_read")
+        return {KERNEL_CLASSES[i]: (ms[i], cnt[i]) for i in range(n)}
 
     def block_means(self, k_idx, k_scale, n_key, kmean, page_table=None, ctx_len=None):
         pt_stride = page_table.shape[1] if page_table is not None else 0

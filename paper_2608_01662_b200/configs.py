@@ -55,6 +55,9 @@ CONFIGS = {
                       R=4, boost_prob=0.05, boost_gain=4.0, **_MLA),
     "cfg4": LsaConfig("cfg4", 3, "decode", 0, 64, 128, "e4m3", 64, 8, 64, 2048, 4, 256,
                       R=4, batch=64, ctx_lo=16384, ctx_hi=131072, kv_page=64, **_MLA),
+    # cfg3 cut to 16K tokens and one layer: small enough for multi-pass ncu captures, still larger than L2
+    "cfg3_16k": LsaConfig("cfg3_16k", 2, "prefill", 16384, 64, 128, "e4m3", 128, 8, 32, 2048, 4, 1024,
+                          R=1, boost_prob=0.05, boost_gain=4.0, **_MLA),
     "cfg5": LsaConfig("cfg5", 4, "prefill", 1048576, 64, 128, "e4m3", 256, 8, 16, 2048, 4, 2048,
                       R=4, q_chunk=16384, **_MLA),
 }

@@ -20,12 +20,32 @@ struct lsa_ctx {
   // lsa_layer_group_host only
   cudaStream_t copy_in, copy_out;
   cudaEvent_t ev_in[2], ev_done[2], ev_out[2];
+  // per-kernel timing (lsa_profile_*): event pairs recorded around the launches of each kernel class
+  int prof_on;
+  int prof_n;
+  cudaEvent_t* prof_ev;   // 2 * kProfPairs events, created on first enable
+  int* prof_cat;
 };
 
 namespace {
 
 constexpr size_t kStatusBytes = 256;
 constexpr int kMaxSplit = 16;
+constexpr int kProfPairs = 4096;
+
+// Runs `launch` (a callable returning cudaError_t), bracketed by an event pair of class `cat` when
+// profiling is on and pairs are left.
+template <class F>
+cudaError_t timed(lsa_ctx* c, int cat, F launch) {
+  const bool rec = c->prof_on && c->prof_ev != nullptr && c->prof_n < kProfPairs;
+  if (rec) cudaEventRecord(c->prof_ev[2 * c->prof_n], c->stream);
+  const cudaError_t e = launch();
+  if (rec) {
+    cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], c->stream);
+    c->prof_cat[c->prof_n++] = cat;
+  }
+  return e;
+}
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -139,8 +159,8 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
     a.pages_out = pages_out ? pages_out + q0 * p->keep_pages : nullptr;
     a.status = status_word(c);
     cudaError_t e = cudaSuccess;
-    if (p->hi_enable) e = lsa::launch_coarse(a, c->stream, &c->launches);
-    if (e == cudaSuccess) e = lsa::launch_fine_select(a, c->stream, &c->launches);
+    if (p->hi_enable) e = timed(c, LSA_K_COARSE, [&] { return lsa::launch_coarse(a, c->stream, &c->launches); });
+    if (e == cudaSuccess) e = timed(c, LSA_K_FINE_SELECT, [&] { return lsa::launch_fine_select(a, c->stream, &c->launches); });
     if (e != cudaSuccess) return cuda_fail(c, e);
   }
   return LSA_OK;
@@ -168,7 +188,8 @@ int run_attn(lsa_ctx* c, const lsa_params* p, const void* q, const void* k, cons
     a.part_lse = reinterpret_cast<float*>(c->ws + l.part_lse);
   }
   if (a.H == 64 && !(v == k && ld_v == ld_k)) return LSA_ERR_SHAPE;
-  cudaError_t e = lsa::launch_attn(a, c->stream, &c->launches);
+  cudaError_t e = timed(c, LSA_K_ATTN, [&] { return lsa::launch_attn(a, c->stream, &c->launches); });
+  if (e == cudaSuccess && a.n_split > 1) e = timed(c, LSA_K_MERGE, [&] { return lsa::launch_merge(a, c->stream, &c->launches); });
   return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
 }
 
@@ -215,6 +236,11 @@ int lsa_destroy(lsa_ctx* c) {
     if (c->ev_done[i]) cudaEventDestroy(c->ev_done[i]);
     if (c->ev_out[i]) cudaEventDestroy(c->ev_out[i]);
   }
+  if (c->prof_ev) {
+    for (int i = 0; i < 2 * kProfPairs; ++i) cudaEventDestroy(c->prof_ev[i]);
+    delete[] c->prof_ev;
+    delete[] c->prof_cat;
+  }
   if (c->copy_in) cudaStreamDestroy(c->copy_in);
   if (c->copy_out) cudaStreamDestroy(c->copy_out);
   delete c;
@@ -256,6 +282,39 @@ const char* lsa_strerror(int err) {
 }
 
 const char* lsa_last_cuda_error(lsa_ctx* c) { return c ? c->cuda_msg : ""; }
+
+int lsa_profile_enable(lsa_ctx* c, int on) {
+  if (c == nullptr) return LSA_ERR_ARG;
+  if (on && c->prof_ev == nullptr) {
+    c->prof_ev = new (std::nothrow) cudaEvent_t[2 * kProfPairs];
+    c->prof_cat = new (std::nothrow) int[kProfPairs];
+    if (c->prof_ev == nullptr || c->prof_cat == nullptr) return LSA_ERR_ARG;
+    for (int i = 0; i < 2 * kProfPairs; ++i) {
+      const cudaError_t e = cudaEventCreate(&c->prof_ev[i]);
+      if (e != cudaSuccess) return cuda_fail(c, e);
+    }
+  }
+  c->prof_on = on ? 1 : 0;
+  c->prof_n = 0;
+  return LSA_OK;
+}
+
+int lsa_profile_read(lsa_ctx* c, double* total_ms, int64_t* launches) {
+  if (c == nullptr || total_ms == nullptr || launches == nullptr) return LSA_ERR_ARG;
+  for (int i = 0; i < LSA_K_COUNT; ++i) {
+    total_ms[i] = 0.0;
+    launches[i] = 0;
+  }
+  cudaError_t e = cudaStreamSynchronize(c->stream);
+  for (int i = 0; i < c->prof_n && e == cudaSuccess; ++i) {
+    float ms = 0.f;
+    e = cudaEventElapsedTime(&ms, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]);
+    total_ms[c->prof_cat[i]] += ms;
+    launches[c->prof_cat[i]] += 1;
+  }
+  c->prof_n = 0;
+  return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
+}
 int64_t lsa_launch_count(lsa_ctx* c) { return c ? c->launches : 0; }
 
 int lsa_block_means(lsa_ctx* c, const lsa_params* p, const void* k_idx, const float* k_scale, int64_t n_key,
@@ -268,9 +327,11 @@ int lsa_block_means(lsa_ctx* c, const lsa_params* p, const void* k_idx, const fl
   if (p->key_dtype == LSA_KEY_E4M3 && k_scale == nullptr) return LSA_ERR_ARG;
   if (p->paged && (page_table == nullptr || ctx_len == nullptr || batch <= 0 || page_table_stride <= 0)) return LSA_ERR_ARG;
   if (!aligned16(k_idx) || !aligned16(kmean)) return LSA_ERR_SHAPE;
-  cudaError_t e = lsa::launch_block_means(p->d_idx, p->key_dtype == LSA_KEY_E4M3, p->sub_block, p->kv_page, k_idx,
-                                          k_scale, n_key, p->paged ? page_table : nullptr, page_table_stride,
-                                          ctx_len, batch, kmean, c->stream, &c->launches);
+  cudaError_t e = timed(c, LSA_K_MEANS, [&] {
+    return lsa::launch_block_means(p->d_idx, p->key_dtype == LSA_KEY_E4M3, p->sub_block, p->kv_page, k_idx, k_scale,
+                                   n_key, p->paged ? page_table : nullptr, page_table_stride, ctx_len, batch, kmean,
+                                   c->stream, &c->launches);
+  });
   return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
 }
 
@@ -303,8 +364,10 @@ int lsa_select(lsa_ctx* c, const lsa_params* p, const float* scores, int64_t ld_
   if (n_query < 0 || n_cand < 0 || k < 0 || ld_scores < n_cand || q_pos0 < 0) return LSA_ERR_ARG;
   if (k > 8192 || n_cand > 0x7fffffff) return LSA_ERR_SHAPE;
   if (n_query == 0 || k == 0) return LSA_OK;
-  cudaError_t e = lsa::launch_select(scores, ld_scores, cand_pos, q_pos0, static_cast<int>(n_query), n_cand, k,
-                                     apply_range, p->k_sink, p->k_swa, idx_out, n_out, c->stream, &c->launches);
+  cudaError_t e = timed(c, LSA_K_SELECT, [&] {
+    return lsa::launch_select(scores, ld_scores, cand_pos, q_pos0, static_cast<int>(n_query), n_cand, k, apply_range,
+                              p->k_sink, p->k_swa, idx_out, n_out, c->stream, &c->launches);
+  });
   return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
 }
 
@@ -316,9 +379,11 @@ int lsa_convert(lsa_ctx* c, const lsa_params* p, const int32_t* sparse_idx, cons
   if (p->paged && (page_table == nullptr || ctx_len == nullptr || batch <= 0 || p->kv_page <= 0)) return LSA_ERR_ARG;
   const int64_t nq = p->paged ? batch : n_query;
   if (nq < 0 || q_pos0 < 0) return LSA_ERR_ARG;
-  cudaError_t e = lsa::launch_convert(p->k_sink, p->k_swa, p->k_sparse, p->paged, p->kv_page, sparse_idx, n_sparse,
-                                      q_pos0, static_cast<int>(nq), page_table, page_table_stride, ctx_len, rows_out,
-                                      n_rows_out, runs_out, c->stream, &c->launches);
+  cudaError_t e = timed(c, LSA_K_CONVERT, [&] {
+    return lsa::launch_convert(p->k_sink, p->k_swa, p->k_sparse, p->paged, p->kv_page, sparse_idx, n_sparse, q_pos0,
+                               static_cast<int>(nq), page_table, page_table_stride, ctx_len, rows_out, n_rows_out,
+                               runs_out, c->stream, &c->launches);
+  });
   return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
 }
 

@@ -299,11 +299,6 @@ cudaError_t launch_attn_t(const AttnArgs& a, cudaStream_t st, int64_t* n_launch)
   dim3 grid(a.n_query, a.n_split);
   kernel<<<grid, kAttnThreads, smem, st>>>(a);
   ++*n_launch;
-  e = cudaGetLastError();
-  if (e != cudaSuccess || a.n_split == 1) return e;
-  merge_splits_kernel<<<dim3(a.n_query, H), 128, 0, st>>>(a.part_out, a.part_lse, a.n_split, H, DV,
-                                                          reinterpret_cast<__nv_bfloat16*>(a.out), a.lse);
-  ++*n_launch;
   return cudaGetLastError();
 }
 
@@ -311,6 +306,14 @@ cudaError_t launch_attn_t(const AttnArgs& a, cudaStream_t st, int64_t* n_launch)
 
 bool attn_shape_supported(int H, int DQK, int DV) {
   return (H == 16 && DQK == 128 && DV == 128) || (H == 64 && DQK == 576 && DV == 512);
+}
+
+cudaError_t launch_merge(const AttnArgs& a, cudaStream_t st, int64_t* n_launch) {
+  if (a.n_query == 0 || a.n_split == 1) return cudaSuccess;
+  merge_splits_kernel<<<dim3(a.n_query, a.H), 128, 0, st>>>(a.part_out, a.part_lse, a.n_split, a.H, a.DV,
+                                                            reinterpret_cast<__nv_bfloat16*>(a.out), a.lse);
+  ++*n_launch;
+  return cudaGetLastError();
 }
 
 cudaError_t launch_attn(const AttnArgs& a, cudaStream_t st, int64_t* n_launch) {

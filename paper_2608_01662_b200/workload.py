@@ -15,7 +15,7 @@ class PrefillWorkload:
     """
 
     def __init__(self, cfg: LsaConfig, device="cuda:0", q_pos0: int = 0, n_query: int | None = None,
-                 n_key: int | None = None, with_lse: bool = True):
+                 n_key: int | None = None, with_lse: bool = True, make_ctx: bool = True):
         assert cfg.mode == "prefill"
         self.cfg, self.device = cfg, torch.device(device)
         self.q_pos0 = q_pos0
@@ -37,7 +37,7 @@ class PrefillWorkload:
         self.kmean = torch.empty((n_sub, cfg.d_I), dtype=torch.bfloat16, device=dev)
         self.sparse_idx = torch.empty((self.n_query, cfg.Ksp), dtype=torch.int32, device=dev)
         self.n_sparse = torch.empty((self.n_query,), dtype=torch.int32, device=dev)
-        self.ctx = binding.Context(self.params, self.n_query, self.n_key, 1, device=dev)
+        self.ctx = binding.Context(self.params, self.n_query, self.n_key, 1, device=dev) if make_ctx else None
 
     def prepare(self):
         """Cache maintenance that happens once per sequence, not per group: the mean-key cache."""
@@ -64,7 +64,7 @@ class PrefillWorkload:
 class DecodeWorkload:
     """cfg.batch sequences with paged caches and one new query token each."""
 
-    def __init__(self, cfg: LsaConfig, device="cuda:0", with_lse: bool = True):
+    def __init__(self, cfg: LsaConfig, device="cuda:0", with_lse: bool = True, make_ctx: bool = True):
         assert cfg.mode == "decode"
         self.cfg, self.device = cfg, torch.device(device)
         dev = self.device
@@ -85,7 +85,7 @@ class DecodeWorkload:
         self.sparse_idx = torch.empty((cfg.batch, cfg.Ksp), dtype=torch.int32, device=dev)
         self.n_sparse = torch.empty((cfg.batch,), dtype=torch.int32, device=dev)
         max_ctx = self.page_table.shape[1] * cfg.kv_page
-        self.ctx = binding.Context(self.params, cfg.batch, max_ctx, cfg.batch, device=dev)
+        self.ctx = binding.Context(self.params, cfg.batch, max_ctx, cfg.batch, device=dev) if make_ctx else None
 
     def prepare(self):
         self.ctx.block_means(self.keys["k"], self.keys.get("scale"), 0, self.kmean, self.page_table, self.ctx_len)

@@ -105,23 +105,31 @@ def check_prefill(wl, queries, check_attention=True, pages=None) -> Metrics:
     return m
 
 
+def decode_caches(wl, b, pools=None):
+    """Logical caches of sequence b of a DecodeWorkload: (HostCaches, query position)."""
+    cfg = wl.cfg
+    if pools is None:
+        pools = (to_np(wl.ctx_len), to_np(wl.page_table), to_np(wl.keys["k"]),
+                 to_np(wl.keys["scale"]) if "scale" in wl.keys else None)
+    ctx, table, k_pool, s_pool = pools
+    n = int(ctx[b])
+    # gather this sequence's K/V rows on the tensors' device (plumbing), widen on the host
+    rows = torch.from_numpy(orc.paged_rows(np.arange(n), table[b], cfg.kv_page)).to(wl.k[0].device)
+    k_l = [to_np(k[rows]) for k in wl.k]
+    caches = ref.HostCaches(k_pool, s_pool, [], [], cfg.B, n_key=n, page_table_row=table[b], kv_page=cfg.kv_page)
+    caches.k = k_l
+    caches.v = [k[:, :cfg.d_v] for k in k_l] if cfg.mla else [to_np(v[rows]) for v in wl.v]
+    return caches, n - 1
+
+
 def check_decode(wl, seqs, check_attention=True) -> Metrics:
     cfg = wl.cfg
     m = Metrics()
     kw = dict(P=cfg.P, B=cfg.B, M=cfg.M, Ksp=cfg.Ksp, S=cfg.S, W=cfg.W)
-    ctx = to_np(wl.ctx_len)
-    table = to_np(wl.page_table)
-    k_pool = to_np(wl.keys["k"])
-    s_pool = to_np(wl.keys["scale"]) if "scale" in wl.keys else None
+    pools = (to_np(wl.ctx_len), to_np(wl.page_table), to_np(wl.keys["k"]),
+             to_np(wl.keys["scale"]) if "scale" in wl.keys else None)
     for b in seqs:
-        n = int(ctx[b])
-        t = n - 1
-        # gather this sequence's K/V rows on the device (plumbing), widen on the host
-        rows = torch.from_numpy(orc.paged_rows(np.arange(n), table[b], cfg.kv_page)).to(wl.device)
-        k_l = [to_np(k[rows]) for k in wl.k]
-        caches = ref.HostCaches(k_pool, s_pool, [], [], cfg.B, n_key=n, page_table_row=table[b], kv_page=cfg.kv_page)
-        caches.k = k_l
-        caches.v = [k[:, :cfg.d_v] for k in k_l] if cfg.mla else [to_np(v[rows]) for v in wl.v]
+        caches, t = decode_caches(wl, b, pools)
         n_sp = int(wl.n_sparse[b])
         gpu_sparse = to_np(wl.sparse_idx[b])
         check_invariants(cfg, t, gpu_sparse, n_sp)
