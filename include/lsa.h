@@ -57,7 +57,8 @@ typedef enum {
   LSA_ERR_SHAPE = -2,      /* dimension or alignment the kernels do not support */
   LSA_ERR_WORKSPACE = -3,  /* workspace missing or smaller than lsa_workspace_bytes says */
   LSA_ERR_CUDA = -4,       /* a CUDA runtime call failed (see lsa_last_cuda_error) */
-  LSA_ERR_TIMEOUT = -5     /* a bounded device-side wait expired (reported through lsa_status) */
+  LSA_ERR_TIMEOUT = -5,    /* a bounded device-side wait expired (reported through lsa_status) */
+  LSA_ERR_CAPACITY = -6    /* the call needs more scratch than a fixed-capacity entry point owns */
 } lsa_error;
 
 enum { LSA_KEY_BF16 = 0, LSA_KEY_E4M3 = 1 };
@@ -155,6 +156,35 @@ LSA_API int lsa_index(lsa_ctx* ctx, const lsa_params* p, const void* q_idx, cons
               const float* k_scale, const void* kmean, int64_t q_pos0, int64_t n_query, int64_t n_key,
               const int32_t* page_table, int64_t page_table_stride, const int32_t* ctx_len, int batch,
               int32_t* sparse_idx, int32_t* n_sparse, int32_t* pages_out);
+
+/* lsa_index for callers that can give the library no scratch memory.  (The paper has no counterpart:
+ * this is a packaging variant of the prefill indexer above, same kernels, same results.)
+ *
+ * Who needs it: code that runs where device memory can no longer be obtained — inside a serving engine
+ * that reserved the whole GPU for its own pools at start-up, from a plugin or callback that is handed
+ * tensors but no allocator, or on a latency-critical path where an allocation (and the device-wide
+ * synchronisation it may imply) is not acceptable.  Such callers cannot size and pass the workspace that
+ * lsa_create / lsa_index expect.  Here the only scratch of the indexer, the page-score matrix
+ * fp32 [n_query, ceil(n_key/P) rounded up to a multiple of 4], sits in a fixed array of
+ * LSA_STATIC_SCRATCH_BYTES inside the library image; every GPU that loads the library holds those bytes
+ * until the process exits.  The call takes no lsa_ctx, allocates nothing on host or device and calls no
+ * allocating routine.
+ *
+ * Arguments as lsa_index with paged = 0 (contiguous caches, query row i at position q_pos0+i); `device`
+ * is the CUDA device of all pointers, `cuda_stream` the stream to enqueue on.  No pages_out.
+ * Limits and behaviour:
+ *   - n_query * (ceil(n_key/P) rounded up to 4) * 4 bytes must not exceed LSA_STATIC_SCRATCH_BYTES, else
+ *     LSA_ERR_CAPACITY and nothing is launched; split the queries over several calls.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
+ *     device made current); make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, which keeps the previous call's contents.  Nothing in it
+ *     has to start at zero (the fine stage reads only entries the coarse stage of the same call wrote).
+ *     Two calls whose kernels overlap on the GPU — different streams, or different host threads — race on
+ *     it: order them on one stream or with events. */
+#define LSA_STATIC_SCRATCH_BYTES (8u << 20)
+LSA_API int lsa_index_static(int device, void* cuda_stream, const lsa_params* p, const void* q_idx, const float* w,
+                             const void* k_idx, const float* k_scale, const void* kmean, int64_t q_pos0,
+                             int64_t n_query, int64_t n_key, int32_t* sparse_idx, int32_t* n_sparse);
 
 /* The selection step alone (Eq. 2 / 7 / 10 / 12) on caller-given fp32 scores; bit-exact by definition.
  *   scores    fp32 [n_query, ld_scores], column c of row i is the score of candidate c

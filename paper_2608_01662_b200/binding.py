@@ -49,6 +49,8 @@ EXPORTS = {
                                 c_void_p, c_int, c_void_p]),
     "lsa_index": (c_int, [c_void_p, POINTER(LsaParams), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64,
                           c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int, c_void_p, c_void_p, c_void_p]),
+    "lsa_index_static": (c_int, [c_int, c_void_p, POINTER(LsaParams), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                 c_int64, c_int64, c_int64, c_void_p, c_void_p]),
     "lsa_select": (c_int, [c_void_p, POINTER(LsaParams), c_void_p, c_int64, c_void_p, c_int64, c_int64, c_int64,
                            c_int32, c_int32, c_void_p, c_void_p]),
     "lsa_convert": (c_int, [c_void_p, POINTER(LsaParams), c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_int64,
@@ -117,6 +119,20 @@ def host_stage_bytes(params: LsaParams, stage_queries: int) -> int:
     if r != 0:
         raise LsaError(r, "lsa_host_stage_bytes")
     return out.value
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def index_static(params: LsaParams, q_idx, w, k_idx, k_scale, kmean, q_pos0, n_query, n_key, sparse_idx, n_sparse,
+                 stream=None):
+    """lsa_index_static: the prefill indexer with its scratch inside the library (no context, no workspace)."""
+    dev = q_idx.device
+    stream = stream if stream is not None else torch.cuda.current_stream(dev)
+    r = lib().lsa_index_static(dev.index or 0, c_void_p(stream.cuda_stream), ctypes.byref(params), _p(q_idx), _p(w),
+                               _p(k_idx), _p(k_scale), _p(kmean), q_pos0, n_query, n_key, _p(sparse_idx), _p(n_sparse))
+    if r != 0:
+        raise LsaError(r, "lsa_index_static")
 
 
 class Context:

@@ -277,6 +277,7 @@ const char* lsa_strerror(int err) {
     case LSA_ERR_WORKSPACE: return "workspace missing or too small";
     case LSA_ERR_CUDA: return "CUDA runtime error";
     case LSA_ERR_TIMEOUT: return "device-side wait timed out";
+    case LSA_ERR_CAPACITY: return "request exceeds the fixed scratch capacity of this entry point";
     default: return "unknown error";
   }
 }
