@@ -36,6 +36,9 @@ def parse_args():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-queries", type=int, default=24)
+    ap.add_argument("--phase", default="group", choices=["group", "index"],
+                    help="group: whole lsa_layer_group step; index: indexer only (no attention tensors are allocated; for profiling)")
+    ap.add_argument("--coarse-groups", type=int, default=0, help="override LSA_TUNE_COARSE_GROUPS (1 or 2)")
     return ap.parse_args()
 
 
@@ -204,8 +207,15 @@ def main():
     kw = {}
     if not decode and cfg.q_chunk and cfg.L > 262144:
         kw = dict(q_pos0=cfg.L - cfg.q_chunk, n_query=cfg.q_chunk)
+    if args.phase == "index":
+        cfg = cfg.replace(R=0)
+        args.no_e2e = True
     wl = make_workload(cfg, dev, with_lse=False, **kw)
+    if args.phase == "index":
+        wl.step = wl.index
     wl.prepare()
+    if args.coarse_groups:
+        wl.ctx.tune(0, args.coarse_groups)
     torch.cuda.synchronize()
 
     def barrier():

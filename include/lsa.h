@@ -112,6 +112,11 @@ LSA_API const char* lsa_last_cuda_error(lsa_ctx* ctx);
 /* Number of kernels this context has launched since creation (host counter). */
 LSA_API int64_t lsa_launch_count(lsa_ctx* ctx);
 
+/* Launch-shape knobs; results never depend on them.
+ *   LSA_TUNE_COARSE_GROUPS  4-query groups held per thread block of the coarse-score kernel (1 or 2; default 1) */
+enum { LSA_TUNE_COARSE_GROUPS = 0, LSA_TUNE_COUNT };
+LSA_API int lsa_tune(lsa_ctx* ctx, int knob, int value);
+
 /* Per-kernel timing.  While enabled, every kernel-launching call records a CUDA event pair on the
  * context's stream around the launches of each kernel class (at most 4096 pairs between reads; later
  * launches go unrecorded).  lsa_profile_read waits for the stream and writes, per class, the summed

@@ -43,6 +43,7 @@ EXPORTS = {
     "lsa_strerror": (c_char_p, [c_int]),
     "lsa_last_cuda_error": (c_char_p, [c_void_p]),
     "lsa_launch_count": (c_int64, [c_void_p]),
+    "lsa_tune": (c_int, [c_void_p, c_int, c_int]),
     "lsa_profile_enable": (c_int, [c_void_p, c_int]),
     "lsa_profile_read": (c_int, [c_void_p, POINTER(ctypes.c_double), POINTER(c_int64)]),
     "lsa_block_means": (c_int, [c_void_p, POINTER(LsaParams), c_void_p, c_void_p, c_int64, c_void_p, c_int64,
@@ -169,6 +170,9 @@ class Context:
 
     def launch_count(self) -> int:
         return lib().lsa_launch_count(self.h)
+
+    def tune(self, knob: int, value: int):
+        self._chk(lib().lsa_tune(self.h, knob, value), "lsa_tune")
 
     def profile_enable(self, on: bool):
         self._chk(lib().lsa_profile_enable(self.h, 1 if on else 0), "lsa_profile_enable")

@@ -21,6 +21,7 @@ struct lsa_ctx {
   cudaStream_t copy_in, copy_out;
   cudaEvent_t ev_in[2], ev_done[2], ev_out[2];
   // per-kernel timing (lsa_profile_*): event pairs recorded around the launches of each kernel class
+  int tune[LSA_TUNE_COUNT];
   int prof_on;
   int prof_n;
   cudaEvent_t* prof_ev;   // 2 * kProfPairs events, created on first enable
@@ -159,7 +160,11 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
     a.pages_out = pages_out ? pages_out + q0 * p->keep_pages : nullptr;
     a.status = status_word(c);
     cudaError_t e = cudaSuccess;
-    if (p->hi_enable) e = timed(c, LSA_K_COARSE, [&] { return lsa::launch_coarse(a, c->stream, &c->launches); });
+    if (p->hi_enable)
+      e = timed(c, LSA_K_COARSE, [&] {
+        return lsa::coarse_tc_supported(a) ? lsa::launch_coarse_tc(a, c->tune[LSA_TUNE_COARSE_GROUPS], c->stream, &c->launches)
+                                           : lsa::launch_coarse(a, c->stream, &c->launches);
+      });
     if (e == cudaSuccess) e = timed(c, LSA_K_FINE_SELECT, [&] { return lsa::launch_fine_select(a, c->stream, &c->launches); });
     if (e != cudaSuccess) return cuda_fail(c, e);
   }
@@ -211,6 +216,7 @@ int lsa_create(lsa_ctx** ctx, int device, void* cuda_stream, void* workspace, si
   c->stream = static_cast<cudaStream_t>(cuda_stream);
   c->ws = static_cast<uint8_t*>(workspace);
   c->ws_bytes = workspace ? workspace_bytes : 0;
+  c->tune[LSA_TUNE_COARSE_GROUPS] = 1;
   e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking);
@@ -283,6 +289,13 @@ const char* lsa_strerror(int err) {
 }
 
 const char* lsa_last_cuda_error(lsa_ctx* c) { return c ? c->cuda_msg : ""; }
+
+int lsa_tune(lsa_ctx* c, int knob, int value) {
+  if (c == nullptr || knob < 0 || knob >= LSA_TUNE_COUNT) return LSA_ERR_ARG;
+  if (knob == LSA_TUNE_COARSE_GROUPS && value != 1 && value != 2) return LSA_ERR_ARG;
+  c->tune[knob] = value;
+  return LSA_OK;
+}
 
 int lsa_profile_enable(lsa_ctx* c, int on) {
   if (c == nullptr) return LSA_ERR_ARG;

@@ -56,6 +56,9 @@ cudaError_t launch_block_means(int DI, int key_e4m3, int B, int kv_page, const v
                                int64_t n_key, const int32_t* page_table, int64_t pt_stride,
                                const int32_t* ctx_len, int batch, void* kmean, cudaStream_t st, int64_t* n_launch);
 cudaError_t launch_coarse(const IndexArgs& a, cudaStream_t st, int64_t* n_launch);
+// tcgen05 version of the coarse stage (contiguous caches, H_I = 64, d_I = 128); groups = 4-query groups per block
+bool coarse_tc_supported(const IndexArgs& a);
+cudaError_t launch_coarse_tc(const IndexArgs& a, int groups, cudaStream_t st, int64_t* n_launch);
 cudaError_t launch_fine_select(const IndexArgs& a, cudaStream_t st, int64_t* n_launch);
 cudaError_t launch_select(const float* scores, int64_t ld, const int32_t* cand_pos, int64_t q_pos0, int n_query,
                           int64_t n_cand, int k, int apply_range, int S, int W, int32_t* idx_out, int32_t* n_out,
