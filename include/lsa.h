@@ -113,7 +113,7 @@ LSA_API const char* lsa_last_cuda_error(lsa_ctx* ctx);
 LSA_API int64_t lsa_launch_count(lsa_ctx* ctx);
 
 /* Launch-shape knobs; results never depend on them.
- *   LSA_TUNE_COARSE_GROUPS  4-query groups held per thread block of the coarse-score kernel (1 or 2; default 1) */
+ *   LSA_TUNE_COARSE_GROUPS  4-query groups held per thread block of the coarse-score kernel (1 or 2; default 2) */
 enum { LSA_TUNE_COARSE_GROUPS = 0, LSA_TUNE_COUNT };
 LSA_API int lsa_tune(lsa_ctx* ctx, int knob, int value);
 

@@ -216,7 +216,7 @@ int lsa_create(lsa_ctx** ctx, int device, void* cuda_stream, void* workspace, si
   c->stream = static_cast<cudaStream_t>(cuda_stream);
   c->ws = static_cast<uint8_t*>(workspace);
   c->ws_bytes = workspace ? workspace_bytes : 0;
-  c->tune[LSA_TUNE_COARSE_GROUPS] = 1;
+  c->tune[LSA_TUNE_COARSE_GROUPS] = 2;
   e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking);

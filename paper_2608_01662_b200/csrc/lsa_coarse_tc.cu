@@ -9,7 +9,7 @@
 //
 //   warp 0      TMA producer: mean-key tiles (and the query groups once) -> 128B-swizzled shared tiles
 //   warp 1      issues tcgen05.mma (M128 N256 K16, bf16 -> fp32) into one of two 256-column TMEM accumulators
-//   warps 2-9   epilogue: tcgen05.ld of the finished accumulator, ReLU * w, sum over heads in-thread (one
+//   warps 2-17  epilogue: tcgen05.ld of the finished accumulator, ReLU * w, sum over heads in-thread (one
 //               thread = one mean key), sum over the sub-blocks of a page by warp shuffles, store
 //
 // so the epilogue of unit u overlaps the MMAs of unit u+1.  Heavy (late) query blocks are launched first.
@@ -27,7 +27,7 @@ constexpr int kAtomBytesA = kTileM * 128;   // one 64-dim column block of an A t
 constexpr int kAtomBytesB = kGroupQ * kHI * 128;
 constexpr int kTileBytesA = 2 * kAtomBytesA;  // d_I = 128 = two 64-dim column blocks
 constexpr int kGroupBytesB = 2 * kAtomBytesB;
-constexpr int kEpiWarps = 8;
+constexpr int kEpiWarps = 16;               // 4 per TMEM lane quarter: one per query of the group
 constexpr int kThreadsTc = 32 * (2 + kEpiWarps);
 constexpr uint32_t kTmemCols = 512;
 
@@ -76,7 +76,7 @@ coarse_score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     tc::mbar_init(smem_u32(&sm.q_full), 1);
     for (int b = 0; b < 2; ++b) {
       tc::mbar_init(smem_u32(&sm.acc_full[b]), 1);
-      tc::mbar_init(smem_u32(&sm.acc_empty[b]), kEpiWarps);
+      tc::mbar_init(smem_u32(&sm.acc_empty[b]), kEpiWarps / 2);
     }
     tc::fence_mbar_init();
   }
@@ -134,48 +134,72 @@ coarse_score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
     }
   } else {
     // ================= epilogue =================
+    // Two sets of 8 warps: set 0 drains accumulator 0 (even units), set 1 accumulator 1 (odd units), so a warp
+    // has two unit periods for its load -> math -> reduce -> store chain.  Within a set, warp (quarter, half)
+    // owns TMEM lanes 32*quarter.. and the head columns of queries 2*half, 2*half+1 of the group.
     const int ew = warp - 2;
-    const int quarter = warp & 3;           // TMEM lanes 32*quarter .. +31 belong to this warp
-    const int half = ew >> 2;               // which two of the group's four queries
+    const int set = ew >> 3;
+    const int quarter = warp & 3;
+    const int half = (ew >> 2) & 1;
     const int row = 32 * quarter + lane;    // mean key within the tile
     bool ok = true;
-    for (int u = 0; u < n_units && ok; ++u) {
-      const int k = u / NG, g = u % NG, buf = u & 1;
-      ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.acc_full[buf]), (u >> 1) & 1, p.status));
+    for (int u = set; u < n_units && ok; u += 2) {
+      const int k = u / NG, g = u % NG;
+      ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.acc_full[set]), (u >> 1) & 1, p.status));
       if (!ok) break;
       tc::fence_after_sync();
       const int64_t sub = static_cast<int64_t>(k) * kTileM + row;
       const int64_t page = sub / spp;
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + set * 256 + half * 2 * kHI;
+      const int ql0 = g * kGroupQ + half * 2;
+      float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
+      {
+        uint32_t v[64];
+        tc::tmem_ld64(taddr, v);
+        tc::tmem_ld_wait();
+        const float4* w4 = reinterpret_cast<const float4*>(&sm.w[ql0][0]);
 #pragma unroll
-      for (int qq = 0; qq < 2; ++qq) {
-        const int ql = g * kGroupQ + half * 2 + qq;     // query within the block
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + buf * 256 + (half * 2 + qq) * kHI;
-        float acc = 0.f;
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t v[32];
-          tc::tmem_ld32(taddr + c * 32, v);
-          tc::tmem_ld_wait();
-          const float4* w4 = reinterpret_cast<const float4*>(&sm.w[ql][c * 32]);
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float4 ww = w4[j];
-            acc = fmaf(ww.x, fmaxf(__uint_as_float(v[4 * j + 0]), 0.f), acc);
-            acc = fmaf(ww.y, fmaxf(__uint_as_float(v[4 * j + 1]), 0.f), acc);
-            acc = fmaf(ww.z, fmaxf(__uint_as_float(v[4 * j + 2]), 0.f), acc);
-            acc = fmaf(ww.w, fmaxf(__uint_as_float(v[4 * j + 3]), 0.f), acc);
-          }
-        }
-        // sum over the sub-blocks of a page: spp (8, 16 or 32) adjacent lanes
-        for (int off = spp >> 1; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-        if ((lane & (spp - 1)) == 0 && ql < nq) {
-          const int64_t t = p.q_pos0 + q0 + ql;
-          if (page * p.P <= t - p.W) p.page_scores[static_cast<int64_t>(q0 + ql) * p.ps_ld + page] = acc;
+        for (int j = 0; j < 16; ++j) {
+          const float4 ww = w4[j];
+          a0 = fmaf(ww.x, fmaxf(__uint_as_float(v[4 * j + 0]), 0.f), a0);
+          a1 = fmaf(ww.y, fmaxf(__uint_as_float(v[4 * j + 1]), 0.f), a1);
+          a0 = fmaf(ww.z, fmaxf(__uint_as_float(v[4 * j + 2]), 0.f), a0);
+          a1 = fmaf(ww.w, fmaxf(__uint_as_float(v[4 * j + 3]), 0.f), a1);
         }
       }
-      tc::fence_before_sync();
-      __syncwarp();
-      if (lane == 0) tc::mbar_arrive(smem_u32(&sm.acc_empty[buf]));
+      {
+        uint32_t v[64];
+        tc::tmem_ld64(taddr + kHI, v);
+        tc::tmem_ld_wait();
+        // the rest of the accumulator is in registers: hand the TMEM buffer back before the arithmetic
+        tc::fence_before_sync();
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(smem_u32(&sm.acc_empty[set]));
+        const float4* w4 = reinterpret_cast<const float4*>(&sm.w[ql0 + 1][0]);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const float4 ww = w4[j];
+          b0 = fmaf(ww.x, fmaxf(__uint_as_float(v[4 * j + 0]), 0.f), b0);
+          b1 = fmaf(ww.y, fmaxf(__uint_as_float(v[4 * j + 1]), 0.f), b1);
+          b0 = fmaf(ww.z, fmaxf(__uint_as_float(v[4 * j + 2]), 0.f), b0);
+          b1 = fmaf(ww.w, fmaxf(__uint_as_float(v[4 * j + 3]), 0.f), b1);
+        }
+      }
+      float acc0 = a0 + a1, acc1 = b0 + b1;
+      // sum over the sub-blocks of a page: spp (8, 16 or 32) adjacent lanes
+      for (int off = spp >> 1; off > 0; off >>= 1) {
+        acc0 += __shfl_xor_sync(0xffffffffu, acc0, off);
+        acc1 += __shfl_xor_sync(0xffffffffu, acc1, off);
+      }
+      if ((lane & (spp - 1)) == 0) {
+#pragma unroll
+        for (int qq = 0; qq < 2; ++qq) {
+          const int ql = ql0 + qq;
+          const int64_t t = p.q_pos0 + q0 + ql;
+          if (ql < nq && page * p.P <= t - p.W)
+            p.page_scores[static_cast<int64_t>(q0 + ql) * p.ps_ld + page] = qq ? acc1 : acc0;
+        }
+      }
     }
   }
   tc::fence_before_sync();
