@@ -38,6 +38,7 @@ def parse_args():
     ap.add_argument("--cpu-queries", type=int, default=24)
     ap.add_argument("--phase", default="group", choices=["group", "index"],
                     help="group: whole lsa_layer_group step; index: indexer only (no attention tensors are allocated; for profiling)")
+    ap.add_argument("--attn-tc", type=int, default=-1, help="override LSA_TUNE_ATTN_TC (0 or 1)")
     ap.add_argument("--coarse-groups", type=int, default=0, help="override LSA_TUNE_COARSE_GROUPS (1 or 2)")
     return ap.parse_args()
 
@@ -216,6 +217,8 @@ def main():
     wl.prepare()
     if args.coarse_groups:
         wl.ctx.tune(0, args.coarse_groups)
+    if args.attn_tc >= 0:
+        wl.ctx.tune(1, args.attn_tc)
     torch.cuda.synchronize()
 
     def barrier():

@@ -193,7 +193,10 @@ int run_attn(lsa_ctx* c, const lsa_params* p, const void* q, const void* k, cons
     a.part_lse = reinterpret_cast<float*>(c->ws + l.part_lse);
   }
   if (a.H == 64 && !(v == k && ld_v == ld_k)) return LSA_ERR_SHAPE;
-  cudaError_t e = timed(c, LSA_K_ATTN, [&] { return lsa::launch_attn(a, c->stream, &c->launches); });
+  cudaError_t e = timed(c, LSA_K_ATTN, [&] {
+    return (c->tune[LSA_TUNE_ATTN_TC] && lsa::attn_tc_supported(a)) ? lsa::launch_attn_tc(a, c->stream, &c->launches)
+                                                                  : lsa::launch_attn(a, c->stream, &c->launches);
+  });
   if (e == cudaSuccess && a.n_split > 1) e = timed(c, LSA_K_MERGE, [&] { return lsa::launch_merge(a, c->stream, &c->launches); });
   return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
 }
@@ -217,6 +220,7 @@ int lsa_create(lsa_ctx** ctx, int device, void* cuda_stream, void* workspace, si
   c->ws = static_cast<uint8_t*>(workspace);
   c->ws_bytes = workspace ? workspace_bytes : 0;
   c->tune[LSA_TUNE_COARSE_GROUPS] = 2;
+  c->tune[LSA_TUNE_ATTN_TC] = 1;
   e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking);

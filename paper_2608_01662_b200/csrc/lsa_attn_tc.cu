@@ -1,0 +1,348 @@
+// a6 on the 5th-generation tensor cores: sparse attention (Eq. 3) for the MLA latent shape
+// (H = 64 heads, d_qk = 576, d_v = 512, the value is the first 512 dims of the key row).
+//
+// One thread block = one query (or one split of one sequence's rows in decode).  Its 64 heads are the M = 64
+// rows of every MMA; the attended cache rows stream through two 64-key shared tiles:
+//
+//   warps 5-8   gather: rows [sink | sparse | window] -> 128B-swizzled K-major tiles with coalesced 16-byte
+//               cp.async (two warps per tile buffer), completion through an mbarrier
+//   warp 4      issues tcgen05.mma:  S = Q K^T   (M64 N64 K16 x 36, both operands K-major)
+//                                    O += P V    (M64 N256 K16 x 8; V is the same shared tile read MN-major,
+//                                                 so each cache row is fetched once)
+//   warps 0-3   softmax: tcgen05.ld S (one row per thread), running max with lazy rescaling of O, exp2, row
+//               sums in fp32, P as bf16 -> shared A operand; at the end O / l -> bf16
+//
+// Tensor-memory map (512 columns allocated): O[:, 0:256] in lanes 0-15 of each 32-lane quarter and O[:, 256:512]
+// in lanes 16-31 (two interleaved M = 64 accumulators), columns 0-255; S double-buffered in columns 256-383.
+// QK^T of tile i+1 is issued before P V of tile i, so the tensor pipe works while the softmax of tile i runs.
+#include "lsa_internal.h"
+#include "lsa_tc.cuh"
+
+namespace lsa {
+
+namespace {
+
+constexpr int kH = 64, kDQK = 576, kDV = 512;
+constexpr int kTileKeys = 64;
+constexpr int kAtoms = kDQK / 64;            // 9 column blocks of 64 dims (128 bytes) per row
+constexpr int kAtomBytes = 64 * 128;         // 64 rows x 128 bytes
+constexpr int kSoftmaxWarps = 4, kLoadWarps = 4;
+constexpr int kThreadsAttnTc = 32 * (kSoftmaxWarps + 1 + kLoadWarps);
+constexpr uint32_t kTmemColsAttn = 512;
+constexpr uint32_t kColS = 256;              // first column of the S buffers
+constexpr float kLog2eTc = 1.4426950408889634f;
+constexpr float kRescaleGap = 8.f;           // rescale O only when the row max grows by more than 2^8
+
+struct AttnTcSmem {
+  alignas(1024) uint8_t q[kAtoms][kAtomBytes];
+  alignas(1024) uint8_t k[2][kAtoms][kAtomBytes];
+  alignas(1024) uint8_t p[kAtomBytes];
+  alignas(8) uint64_t q_full, k_full[2], k_empty[2], s_full[2], s_free[2], p_ready, pv_done;
+  uint32_t tmem_slot;
+};
+
+__global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnArgs p) {
+  extern __shared__ uint8_t smem_raw[];
+  AttnTcSmem& sm = *reinterpret_cast<AttnTcSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int qi = blockIdx.x, split = blockIdx.y;
+
+  // ---- this query's row list (same conventions as the mma.sync kernel)
+  const int64_t t = p.paged ? static_cast<int64_t>(p.ctx_len[qi]) - 1 : p.q_pos0 + qi;
+  int n_sink = 0, n_sp = 0, n_tot;
+  int64_t win0 = 0;
+  const int32_t* rows = nullptr;
+  if (p.rows != nullptr) {
+    rows = p.rows + static_cast<int64_t>(qi) * p.rows_ld;
+    n_tot = p.n_rows[qi];
+  } else {
+    n_sink = static_cast<int>(min64(p.S, t + 1));
+    win0 = max64(p.S, t - p.W + 1);
+    n_sp = p.n_sparse[qi];
+    n_tot = n_sink + n_sp + static_cast<int>(max64(0, t - win0 + 1));
+  }
+  const int32_t* sp = p.sparse_idx ? p.sparse_idx + static_cast<int64_t>(qi) * p.Ksp : nullptr;
+  auto row_of = [&](int i) -> int32_t {
+    if (i >= n_tot) return -1;
+    if (rows) return rows[i];
+    if (i < n_sink) return i;
+    if (i < n_sink + n_sp) return sp[i - n_sink];
+    return static_cast<int32_t>(win0 + (i - n_sink - n_sp));
+  };
+  const int tiles_all = (n_tot + kTileKeys - 1) / kTileKeys;
+  const int tiles_per = (tiles_all + p.n_split - 1) / p.n_split;
+  const int tile_begin = split * tiles_per;
+  const int n_tiles = max(0, min(tiles_all, tile_begin + tiles_per) - tile_begin);
+
+  // ---- set-up
+  if (tid == 0) {
+    tc::mbar_init(smem_u32(&sm.q_full), 32 * kLoadWarps);
+    for (int b = 0; b < 2; ++b) {
+      tc::mbar_init(smem_u32(&sm.k_full[b]), 32 * kLoadWarps / 2);
+      tc::mbar_init(smem_u32(&sm.k_empty[b]), 1);
+      tc::mbar_init(smem_u32(&sm.s_full[b]), 1);
+      tc::mbar_init(smem_u32(&sm.s_free[b]), kSoftmaxWarps);
+    }
+    tc::mbar_init(smem_u32(&sm.p_ready), kSoftmaxWarps);
+    tc::mbar_init(smem_u32(&sm.pv_done), 1);
+    tc::fence_mbar_init();
+  }
+  if (warp == kSoftmaxWarps) {
+    tc::tmem_alloc(smem_u32(&sm.tmem_slot), kTmemColsAttn);
+    tc::tmem_relinquish();
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tmem_base = sm.tmem_slot;
+
+  if (warp > kSoftmaxWarps) {
+    // ================= gather warps =================
+    const int lt = tid - 32 * (kSoftmaxWarps + 1);   // 0..127
+    {
+      // Q: 64 rows of 1152 contiguous bytes
+      const uint8_t* qg = reinterpret_cast<const uint8_t*>(p.q) + static_cast<int64_t>(qi) * kH * kDQK * 2;
+      for (int e = lt; e < kH * 72; e += 32 * kLoadWarps) {
+        const int r = e / 72, c = e % 72;
+        cp_async16(smem_u32(sm.q[c >> 3]) + r * 128 + (((c & 7) ^ (r & 7)) << 4), qg + e * 16, 16);
+      }
+      cp_async_commit();
+      cp_async_wait<0>();
+      tc::fence_proxy_async();
+      tc::mbar_arrive(smem_u32(&sm.q_full));
+    }
+    // Two groups of two warps, one group per tile buffer; warp `wg` of a group gathers rows 32*wg .. +31 of its
+    // tiles.  Lane l looks up the cache row of key 32*wg + l once; the row number is then broadcast and the 72
+    // 16-byte chunks of that row are copied by consecutive lanes (coalesced 512-byte requests).
+    const int grp = lt >> 6, wg = (lt >> 5) & 1;
+    const uint8_t* kg = reinterpret_cast<const uint8_t*>(p.k);
+    for (int i = grp; i < n_tiles; i += 2) {
+      if (!__all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.k_empty[grp]), ((i >> 1) & 1) ^ 1, p.status))) break;
+      const int32_t my_row = row_of((tile_begin + i) * kTileKeys + 32 * wg + lane);
+#pragma unroll 4
+      for (int rr = 0; rr < 32; ++rr) {
+        const int32_t row = __shfl_sync(0xffffffffu, my_row, rr);
+        const int r = 32 * wg + rr;
+        const uint8_t* src = kg + static_cast<int64_t>(row >= 0 ? row : 0) * p.ld_k * 2;
+        const int nb = row >= 0 ? 16 : 0;
+#pragma unroll
+        for (int c = lane; c < 72; c += 32)
+          cp_async16(smem_u32(sm.k[grp][c >> 3]) + r * 128 + (((c & 7) ^ (r & 7)) << 4), src + c * 16, nb);
+      }
+      cp_async_commit();
+      cp_async_wait<0>();
+      tc::fence_proxy_async();
+      tc::mbar_arrive(smem_u32(&sm.k_full[grp]));
+    }
+  } else if (warp == kSoftmaxWarps) {
+    // ================= MMA issuer =================
+    if (lane == 0 && n_tiles > 0) {
+      constexpr uint32_t idesc_qk = tc::idesc_bf16(kH, kTileKeys, 0, 0);
+      constexpr uint32_t idesc_pv = tc::idesc_bf16(kH, 256, 0, 1);   // B = V read MN-major
+      bool ok = tc::mbar_wait(smem_u32(&sm.q_full), 0, p.status);
+      auto issue_pv = [&](int j) {   // O += P_j V_j
+        const int b = j & 1;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const uint32_t d = tmem_base + (static_cast<uint32_t>(16 * half) << 16);
+#pragma unroll
+          for (int kk = 0; kk < kTileKeys / 16; ++kk) {
+            const uint64_t da = tc::smem_desc_sw128(smem_u32(sm.p) + kk * 32, 16, 1024);
+            const uint64_t db = tc::smem_desc_sw128(smem_u32(sm.k[b][4 * half]) + kk * 2048, kAtomBytes, 1024);
+            tc::umma_ss(d, da, db, idesc_pv, (j > 0) || (kk > 0));
+          }
+        }
+        tc::umma_commit(smem_u32(&sm.k_empty[b]));
+        tc::umma_commit(smem_u32(&sm.pv_done));
+      };
+      for (int i = 0; i < n_tiles && ok; ++i) {
+        const int b = i & 1;
+        ok = tc::mbar_wait(smem_u32(&sm.k_full[b]), (i >> 1) & 1, p.status) &&
+             tc::mbar_wait(smem_u32(&sm.s_free[b]), ((i >> 1) & 1) ^ 1, p.status);
+        if (!ok) break;
+        tc::fence_after_sync();
+        const uint32_t d = tmem_base + kColS + b * kTileKeys;
+#pragma unroll
+        for (int a = 0; a < kAtoms; ++a) {
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+            const uint64_t da = tc::smem_desc_sw128(smem_u32(sm.q[a]) + kk * 32, 16, 1024);
+            const uint64_t db = tc::smem_desc_sw128(smem_u32(sm.k[b][a]) + kk * 32, 16, 1024);
+            tc::umma_ss(d, da, db, idesc_qk, (a | kk) != 0);
+          }
+        }
+        tc::umma_commit(smem_u32(&sm.s_full[b]));
+        if (i > 0) {
+          ok = tc::mbar_wait(smem_u32(&sm.p_ready), (i - 1) & 1, p.status);
+          if (!ok) break;
+          tc::fence_after_sync();
+          issue_pv(i - 1);
+        }
+      }
+      if (ok && tc::mbar_wait(smem_u32(&sm.p_ready), (n_tiles - 1) & 1, p.status)) {
+        tc::fence_after_sync();
+        issue_pv(n_tiles - 1);
+      }
+    }
+  } else {
+    // ================= softmax warps =================
+    const int quarter = warp;                 // TMEM lanes 32*warp .. +31
+    const int r16 = lane & 15, hi = lane >> 4;
+    const int row = 16 * quarter + r16;       // head; lanes 16-31 shadow lanes 0-15 and own O[:, 256:512]
+    const float zs = p.sm_scale * kLog2eTc;
+    float m_used = -INFINITY, l_run = 0.f;
+    bool ok = true;
+    const uint32_t lane_addr = static_cast<uint32_t>(32 * quarter) << 16;
+    for (int i = 0; i < n_tiles && ok; ++i) {
+      const int b = i & 1;
+      ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.s_full[b]), (i >> 1) & 1, p.status));
+      if (!ok) break;
+      tc::fence_after_sync();
+      uint32_t v[64];
+      tc::tmem_ld64(tmem_base + lane_addr + kColS + b * kTileKeys, v);
+      tc::tmem_ld_wait();
+      tc::fence_before_sync();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(smem_u32(&sm.s_free[b]));
+      // logits in log2 units, ragged tail masked
+      const int n_valid = min(kTileKeys, n_tot - (tile_begin + i) * kTileKeys);
+      float mx = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 64; ++j) {
+        const float z = j < n_valid ? __uint_as_float(v[j]) * zs : -INFINITY;
+        v[j] = __float_as_uint(z);
+        mx = fmaxf(mx, z);
+      }
+      // running max, moved only when it grows by more than kRescaleGap (O and l are then rescaled)
+      float alpha = 1.f;
+      bool grow = false;
+      if (hi == 0) {
+        if (i == 0) {
+          m_used = mx;
+        } else if (mx > m_used + kRescaleGap) {
+          grow = true;
+          alpha = exp2f(m_used - mx);
+          m_used = mx;
+        }
+      }
+      const bool any_grow = __any_sync(0xffffffffu, grow);
+      bool waited_pv = false;
+      if (any_grow) {
+        // O may be touched only between P V of tile i-1 (done) and P V of tile i (not yet released)
+        ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done), (i - 1) & 1, p.status));
+        if (!ok) break;
+        waited_pv = true;
+        tc::fence_after_sync();
+        const float a_row = __shfl_sync(0xffffffffu, alpha, r16);   // lanes 16-31 take their row's factor
+        if (__any_sync(0xffffffffu, a_row != 1.f)) {
+#pragma unroll 1
+          for (int c = 0; c < 256; c += 64) {
+            uint32_t o[64];
+            tc::tmem_ld64(tmem_base + lane_addr + c, o);
+            tc::tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 64; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * a_row);
+            tc::tmem_st64(tmem_base + lane_addr + c, o);
+          }
+          tc::tmem_st_wait();
+        }
+        l_run *= alpha;
+        tc::fence_before_sync();
+      }
+      // P = exp2(z - m), fp32 row sum, bf16 pack
+      uint32_t pk[32];
+      float sum = 0.f;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const float p0 = exp2f(__uint_as_float(v[2 * j]) - m_used);
+        const float p1 = exp2f(__uint_as_float(v[2 * j + 1]) - m_used);
+        sum += p0 + p1;
+        pk[j] = pack_bf16(p0, p1);
+      }
+      l_run += sum;
+      // the P tile is free once P V of the previous tile has read it
+      if (i > 0 && !waited_pv) {
+        ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done), (i - 1) & 1, p.status));
+        if (!ok) break;
+      }
+      if (hi == 0) {
+        uint8_t* prow = sm.p + row * 128;
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+        tc::fence_proxy_async();
+      }
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(smem_u32(&sm.p_ready));
+    }
+    // ---- epilogue: O / l
+    const float l_row = __shfl_sync(0xffffffffu, l_run, r16);
+    const float m_row = __shfl_sync(0xffffffffu, m_used, r16);
+    bool have_o = ok && n_tiles > 0;
+    if (have_o) have_o = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done), (n_tiles - 1) & 1, p.status));
+    tc::fence_after_sync();
+    const float inv = (have_o && l_row > 0.f) ? 1.f / l_row : 0.f;
+    const int d0 = hi * 256;
+    __nv_bfloat16* out = nullptr;
+    float* pout = nullptr;
+    if (p.n_split == 1) out = reinterpret_cast<__nv_bfloat16*>(p.out) + (static_cast<int64_t>(qi) * kH + row) * kDV + d0;
+    else pout = p.part_out + ((static_cast<int64_t>(qi) * p.n_split + split) * kH + row) * kDV + d0;
+#pragma unroll 1
+    for (int c = 0; c < 256; c += 64) {
+      uint32_t o[64];
+      if (have_o) {
+        tc::tmem_ld64(tmem_base + lane_addr + c, o);
+        tc::tmem_ld_wait();
+      } else {
+#pragma unroll
+        for (int j = 0; j < 64; ++j) o[j] = 0u;
+      }
+      if (out != nullptr) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          uint4 w4;
+          w4.x = pack_bf16(__uint_as_float(o[8 * j + 0]) * inv, __uint_as_float(o[8 * j + 1]) * inv);
+          w4.y = pack_bf16(__uint_as_float(o[8 * j + 2]) * inv, __uint_as_float(o[8 * j + 3]) * inv);
+          w4.z = pack_bf16(__uint_as_float(o[8 * j + 4]) * inv, __uint_as_float(o[8 * j + 5]) * inv);
+          w4.w = pack_bf16(__uint_as_float(o[8 * j + 6]) * inv, __uint_as_float(o[8 * j + 7]) * inv);
+          *reinterpret_cast<uint4*>(out + c + 8 * j) = w4;
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          *reinterpret_cast<float4*>(pout + c + 4 * j) =
+              make_float4(__uint_as_float(o[4 * j]) * inv, __uint_as_float(o[4 * j + 1]) * inv,
+                          __uint_as_float(o[4 * j + 2]) * inv, __uint_as_float(o[4 * j + 3]) * inv);
+      }
+    }
+    if (hi == 0) {
+      const float lse2 = (have_o && l_row > 0.f) ? m_row + log2f(l_row) : -INFINITY;   // log2 domain
+      if (p.n_split == 1) {
+        if (p.lse != nullptr) p.lse[static_cast<int64_t>(qi) * kH + row] = lse2 / kLog2eTc;
+      } else {
+        p.part_lse[(static_cast<int64_t>(qi) * p.n_split + split) * kH + row] = lse2;
+      }
+    }
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+  if (warp == kSoftmaxWarps) tc::tmem_dealloc(tmem_base, kTmemColsAttn);
+}
+
+}  // namespace
+
+bool attn_tc_supported(const AttnArgs& a) {
+  return a.H == kH && a.DQK == kDQK && a.DV == kDV && a.v == a.k && a.ld_v == a.ld_k;
+}
+
+cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t st, int64_t* n_launch) {
+  if (a.n_query == 0) return cudaSuccess;
+  const size_t smem = sizeof(AttnTcSmem) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(sparse_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  sparse_attn_tc_kernel<<<dim3(a.n_query, a.n_split), kThreadsAttnTc, smem, st>>>(a);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+}  // namespace lsa

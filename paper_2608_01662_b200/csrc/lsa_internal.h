@@ -68,6 +68,9 @@ cudaError_t launch_convert(int S, int W, int Ksp, int paged, int kv_page, const 
                            int64_t pt_stride, const int32_t* ctx_len, int32_t* rows_out, int32_t* n_rows_out,
                            int32_t* runs_out, cudaStream_t st, int64_t* n_launch);
 cudaError_t launch_attn(const AttnArgs& a, cudaStream_t st, int64_t* n_launch);
+// tcgen05 version of the attention kernel (MLA latent shape only)
+bool attn_tc_supported(const AttnArgs& a);
+cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t st, int64_t* n_launch);
 cudaError_t launch_merge(const AttnArgs& a, cudaStream_t st, int64_t* n_launch);
 
 bool index_shape_supported(int HI, int DI);
