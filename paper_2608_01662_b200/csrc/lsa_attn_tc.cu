@@ -2,19 +2,23 @@
 // (H = 64 heads, d_qk = 576, d_v = 512, the value is the first 512 dims of the key row).
 //
 // One thread block = one query (or one split of one sequence's rows in decode).  Its 64 heads are the M = 64
-// rows of every MMA; the attended cache rows stream through two 64-key shared tiles:
+// rows of every MMA; the attended cache rows stream through two 64-key shared tiles, each made of two 32-key
+// halves:
 //
-//   warps 5-8   gather: rows [sink | sparse | window] -> 128B-swizzled K-major tiles with coalesced 16-byte
-//               cp.async (two warps per tile buffer), completion through an mbarrier
-//   warp 4      issues tcgen05.mma:  S = Q K^T   (M64 N64 K16 x 36, both operands K-major)
+//   warps 5-8   gather: rows [sink | sparse | window] -> 128B-swizzled K-major half-tiles with coalesced 16-byte
+//               cp.async (one warp per half-tile), completion through an mbarrier
+//   warp 4      issues tcgen05.mma:  S = Q K^T   (M64 N32 K16 x 36 per half; both operands K-major)
 //                                    O += P V    (M64 N256 K16 x 8; V is the same shared tile read MN-major,
 //                                                 so each cache row is fetched once)
-//   warps 0-3   softmax: tcgen05.ld S (one row per thread), running max with lazy rescaling of O, exp2, row
-//               sums in fp32, P as bf16 -> shared A operand; at the end O / l -> bf16
+//               and takes whichever of "next Q K^T" / "next P V" is ready, so the tensor pipe keeps working
+//               while a softmax or a gather is in flight
+//   warps 0-3   softmax: tcgen05.ld S, running max with lazy rescaling of O, exp2, fp32 row sums, P as bf16 ->
+//               shared A operand; at the end O / l -> bf16
 //
-// Tensor-memory map (512 columns allocated): O[:, 0:256] in lanes 0-15 of each 32-lane quarter and O[:, 256:512]
-// in lanes 16-31 (two interleaved M = 64 accumulators), columns 0-255; S double-buffered in columns 256-383.
-// QK^T of tile i+1 is issued before P V of tile i, so the tensor pipe works while the softmax of tile i runs.
+// An M = 64 accumulator occupies 16 of the 32 lanes of each TMEM quarter, so two of them share a column range:
+//   columns   0-255   O[:, 0:256] in lanes 0-15, O[:, 256:512] in lanes 16-31
+//   columns 256-319   S buffers 0 and 1 (32 columns each): keys 0-31 of the tile in lanes 0-15, keys 32-63 in
+//                     lanes 16-31, so that lanes l and l+16 of a softmax warp share one head row
 #include "lsa_internal.h"
 #include "lsa_tc.cuh"
 
@@ -26,6 +30,8 @@ constexpr int kH = 64, kDQK = 576, kDV = 512;
 constexpr int kTileKeys = 64;
 constexpr int kAtoms = kDQK / 64;            // 9 column blocks of 64 dims (128 bytes) per row
 constexpr int kAtomBytes = 64 * 128;         // 64 rows x 128 bytes
+constexpr int kHalfKeys = 32;
+constexpr int kHalfAtomBytes = kHalfKeys * 128;
 constexpr int kSoftmaxWarps = 4, kLoadWarps = 4;
 constexpr int kThreadsAttnTc = 32 * (kSoftmaxWarps + 1 + kLoadWarps);
 constexpr uint32_t kTmemColsAttn = 512;
@@ -35,7 +41,7 @@ constexpr float kRescaleGap = 8.f;           // rescale O only when the row max 
 
 struct AttnTcSmem {
   alignas(1024) uint8_t q[kAtoms][kAtomBytes];
-  alignas(1024) uint8_t k[2][kAtoms][kAtomBytes];
+  alignas(1024) uint8_t k[2][2][kAtoms][kHalfAtomBytes];   // [tile buffer][half][column block][32 rows x 128 B]
   alignas(1024) uint8_t p[kAtomBytes];
   alignas(8) uint64_t q_full, k_full[2], k_empty[2], s_full[2], s_free[2], p_ready, pv_done;
   uint32_t tmem_slot;
@@ -116,81 +122,104 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     // 16-byte chunks of that row are copied by consecutive lanes (coalesced 512-byte requests).
     const int grp = lt >> 6, wg = (lt >> 5) & 1;
     const uint8_t* kg = reinterpret_cast<const uint8_t*>(p.k);
+    int32_t my_row = grp < n_tiles ? row_of((tile_begin + grp) * kTileKeys + kHalfKeys * wg + lane) : -1;
     for (int i = grp; i < n_tiles; i += 2) {
+      // row numbers of this warp's next half-tile are fetched before the wait, off the critical path
+      const int32_t next_row = i + 2 < n_tiles ? row_of((tile_begin + i + 2) * kTileKeys + kHalfKeys * wg + lane) : -1;
       if (!__all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.k_empty[grp]), ((i >> 1) & 1) ^ 1, p.status))) break;
-      const int32_t my_row = row_of((tile_begin + i) * kTileKeys + 32 * wg + lane);
 #pragma unroll 4
-      for (int rr = 0; rr < 32; ++rr) {
+      for (int rr = 0; rr < kHalfKeys; ++rr) {
         const int32_t row = __shfl_sync(0xffffffffu, my_row, rr);
-        const int r = 32 * wg + rr;
         const uint8_t* src = kg + static_cast<int64_t>(row >= 0 ? row : 0) * p.ld_k * 2;
         const int nb = row >= 0 ? 16 : 0;
 #pragma unroll
         for (int c = lane; c < 72; c += 32)
-          cp_async16(smem_u32(sm.k[grp][c >> 3]) + r * 128 + (((c & 7) ^ (r & 7)) << 4), src + c * 16, nb);
+          cp_async16(smem_u32(sm.k[grp][wg][c >> 3]) + rr * 128 + (((c & 7) ^ (rr & 7)) << 4), src + c * 16, nb);
       }
       cp_async_commit();
       cp_async_wait<0>();
       tc::fence_proxy_async();
       tc::mbar_arrive(smem_u32(&sm.k_full[grp]));
+      my_row = next_row;
     }
   } else if (warp == kSoftmaxWarps) {
     // ================= MMA issuer =================
     if (lane == 0 && n_tiles > 0) {
-      constexpr uint32_t idesc_qk = tc::idesc_bf16(kH, kTileKeys, 0, 0);
+      constexpr uint32_t idesc_qk = tc::idesc_bf16(kH, kHalfKeys, 0, 0);
       constexpr uint32_t idesc_pv = tc::idesc_bf16(kH, 256, 0, 1);   // B = V read MN-major
       bool ok = tc::mbar_wait(smem_u32(&sm.q_full), 0, p.status);
-      auto issue_pv = [&](int j) {   // O += P_j V_j
-        const int b = j & 1;
+      // Descriptors are built once; inside the loops only the start-address word moves (one add per operand):
+      // a single thread has to issue ~80 MMAs per tile, so its instruction count per MMA matters.
+      const uint64_t dq0 = tc::smem_desc_sw128(smem_u32(sm.q), 16, 1024);
+      const uint64_t dp0 = tc::smem_desc_sw128(smem_u32(sm.p), 16, 1024);
+      const uint64_t dk0 = tc::smem_desc_sw128(smem_u32(sm.k), 16, 1024);              // K-major view (Q K^T)
+      const uint64_t dv0 = tc::smem_desc_sw128(smem_u32(sm.k), kHalfAtomBytes, 1024);  // MN-major view (P V)
+      constexpr uint32_t kBufBytes = 2 * kAtoms * kHalfAtomBytes, kHalfBytes = kAtoms * kHalfAtomBytes;
+      auto issue_qk = [&](int i) {   // S_i = Q K_i^T, keys 0-31 -> lanes 0-15, keys 32-63 -> lanes 16-31
+        const int b = i & 1;
+        tc::fence_after_sync();
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
-          const uint32_t d = tmem_base + (static_cast<uint32_t>(16 * half) << 16);
+          const uint32_t d = tmem_base + (static_cast<uint32_t>(16 * half) << 16) + kColS + b * kHalfKeys;
+          const uint64_t dkb = tc::desc_advance(dk0, b * kBufBytes + half * kHalfBytes);
 #pragma unroll
-          for (int kk = 0; kk < kTileKeys / 16; ++kk) {
-            const uint64_t da = tc::smem_desc_sw128(smem_u32(sm.p) + kk * 32, 16, 1024);
-            const uint64_t db = tc::smem_desc_sw128(smem_u32(sm.k[b][4 * half]) + kk * 2048, kAtomBytes, 1024);
-            tc::umma_ss(d, da, db, idesc_pv, (j > 0) || (kk > 0));
+          for (int a = 0; a < kAtoms; ++a) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              tc::umma_ss(d, tc::desc_advance(dq0, a * kAtomBytes + kk * 32), tc::desc_advance(dkb, a * kHalfAtomBytes + kk * 32),
+                          idesc_qk, (a | kk) != 0);
           }
+        }
+        tc::umma_commit(smem_u32(&sm.s_full[b]));
+      };
+      auto issue_pv = [&](int j) {   // O += P_j V_j
+        const int b = j & 1;
+        tc::fence_after_sync();
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {          // value dims 256*half .. +255
+          const uint32_t d = tmem_base + (static_cast<uint32_t>(16 * half) << 16);
+          const uint64_t dvb = tc::desc_advance(dv0, b * kBufBytes + 4 * half * kHalfAtomBytes);
+#pragma unroll
+          for (int kk = 0; kk < kTileKeys / 16; ++kk)   // keys 16*kk .. +15: half-tile kk/2, rows 16*(kk%2) ..
+            tc::umma_ss(d, tc::desc_advance(dp0, kk * 32), tc::desc_advance(dvb, (kk >> 1) * kHalfBytes + (kk & 1) * 2048),
+                        idesc_pv, (j > 0) || (kk > 0));
         }
         tc::umma_commit(smem_u32(&sm.k_empty[b]));
         tc::umma_commit(smem_u32(&sm.pv_done));
       };
-      for (int i = 0; i < n_tiles && ok; ++i) {
-        const int b = i & 1;
-        ok = tc::mbar_wait(smem_u32(&sm.k_full[b]), (i >> 1) & 1, p.status) &&
-             tc::mbar_wait(smem_u32(&sm.s_free[b]), ((i >> 1) & 1) ^ 1, p.status);
-        if (!ok) break;
-        tc::fence_after_sync();
-        const uint32_t d = tmem_base + kColS + b * kTileKeys;
-#pragma unroll
-        for (int a = 0; a < kAtoms; ++a) {
-#pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {
-            const uint64_t da = tc::smem_desc_sw128(smem_u32(sm.q[a]) + kk * 32, 16, 1024);
-            const uint64_t db = tc::smem_desc_sw128(smem_u32(sm.k[b][a]) + kk * 32, 16, 1024);
-            tc::umma_ss(d, da, db, idesc_qk, (a | kk) != 0);
+      // Two in-order queues, "next Q K^T" (at most one tile ahead of the softmax it feeds) and "next P V".
+      int qk_next = 0, pv_next = 0;
+      const long long t_start = clock64();
+      uint32_t spins = 0;
+      while (ok && pv_next < n_tiles) {
+        bool did = false;
+        if (qk_next < n_tiles && qk_next <= pv_next + 1) {
+          const int b = qk_next & 1;
+          if (tc::mbar_test(smem_u32(&sm.k_full[b]), (qk_next >> 1) & 1) &&
+              tc::mbar_test(smem_u32(&sm.s_free[b]), ((qk_next >> 1) & 1) ^ 1)) {
+            issue_qk(qk_next++);
+            did = true;
           }
         }
-        tc::umma_commit(smem_u32(&sm.s_full[b]));
-        if (i > 0) {
-          ok = tc::mbar_wait(smem_u32(&sm.p_ready), (i - 1) & 1, p.status);
-          if (!ok) break;
-          tc::fence_after_sync();
-          issue_pv(i - 1);
+        if (!did && pv_next < qk_next && tc::mbar_test(smem_u32(&sm.p_ready), pv_next & 1)) {
+          issue_pv(pv_next++);
+          did = true;
         }
-      }
-      if (ok && tc::mbar_wait(smem_u32(&sm.p_ready), (n_tiles - 1) & 1, p.status)) {
-        tc::fence_after_sync();
-        issue_pv(n_tiles - 1);
+        if (did) {
+          spins = 0;
+        } else if ((++spins & 1023u) == 0 && clock64() - t_start > tc::kWaitCycles * 8) {
+          report_status(p.status, kDevTimeout);   // bounded: nothing became ready for seconds
+          ok = false;
+        }
       }
     }
   } else {
     // ================= softmax warps =================
     const int quarter = warp;                 // TMEM lanes 32*warp .. +31
     const int r16 = lane & 15, hi = lane >> 4;
-    const int row = 16 * quarter + r16;       // head; lanes 16-31 shadow lanes 0-15 and own O[:, 256:512]
+    const int row = 16 * quarter + r16;       // head; lanes l and l+16 share it: keys 0-31 / 32-63, O dims 0-255 / 256-511
     const float zs = p.sm_scale * kLog2eTc;
-    float m_used = -INFINITY, l_run = 0.f;
+    float m_used = -INFINITY, l_run = 0.f;    // m_used is kept identical in both lanes of a row; l_run is a partial sum
     bool ok = true;
     const uint32_t lane_addr = static_cast<uint32_t>(32 * quarter) << 16;
     for (int i = 0; i < n_tiles && ok; ++i) {
@@ -198,62 +227,55 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.s_full[b]), (i >> 1) & 1, p.status));
       if (!ok) break;
       tc::fence_after_sync();
-      uint32_t v[64];
-      tc::tmem_ld64(tmem_base + lane_addr + kColS + b * kTileKeys, v);
+      uint32_t v[32];
+      tc::tmem_ld32(tmem_base + lane_addr + kColS + b * kHalfKeys, v);
       tc::tmem_ld_wait();
       tc::fence_before_sync();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(smem_u32(&sm.s_free[b]));
       // logits in log2 units, ragged tail masked
-      const int n_valid = min(kTileKeys, n_tot - (tile_begin + i) * kTileKeys);
+      const int n_valid = n_tot - (tile_begin + i) * kTileKeys - kHalfKeys * hi;   // keys of this lane's half that exist
       float mx = -INFINITY;
 #pragma unroll
-      for (int j = 0; j < 64; ++j) {
+      for (int j = 0; j < 32; ++j) {
         const float z = j < n_valid ? __uint_as_float(v[j]) * zs : -INFINITY;
         v[j] = __float_as_uint(z);
         mx = fmaxf(mx, z);
       }
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
       // running max, moved only when it grows by more than kRescaleGap (O and l are then rescaled)
       float alpha = 1.f;
-      bool grow = false;
-      if (hi == 0) {
-        if (i == 0) {
-          m_used = mx;
-        } else if (mx > m_used + kRescaleGap) {
-          grow = true;
-          alpha = exp2f(m_used - mx);
-          m_used = mx;
-        }
+      if (i == 0) {
+        m_used = mx;
+      } else if (mx > m_used + kRescaleGap) {
+        alpha = exp2f(m_used - mx);
+        m_used = mx;
       }
-      const bool any_grow = __any_sync(0xffffffffu, grow);
       bool waited_pv = false;
-      if (any_grow) {
+      if (__any_sync(0xffffffffu, alpha != 1.f)) {
         // O may be touched only between P V of tile i-1 (done) and P V of tile i (not yet released)
         ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done), (i - 1) & 1, p.status));
         if (!ok) break;
         waited_pv = true;
         tc::fence_after_sync();
-        const float a_row = __shfl_sync(0xffffffffu, alpha, r16);   // lanes 16-31 take their row's factor
-        if (__any_sync(0xffffffffu, a_row != 1.f)) {
 #pragma unroll 1
-          for (int c = 0; c < 256; c += 64) {
-            uint32_t o[64];
-            tc::tmem_ld64(tmem_base + lane_addr + c, o);
-            tc::tmem_ld_wait();
+        for (int c = 0; c < 256; c += 64) {
+          uint32_t o[64];
+          tc::tmem_ld64(tmem_base + lane_addr + c, o);
+          tc::tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 64; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * a_row);
-            tc::tmem_st64(tmem_base + lane_addr + c, o);
-          }
-          tc::tmem_st_wait();
+          for (int j = 0; j < 64; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+          tc::tmem_st64(tmem_base + lane_addr + c, o);
         }
+        tc::tmem_st_wait();
         l_run *= alpha;
         tc::fence_before_sync();
       }
       // P = exp2(z - m), fp32 row sum, bf16 pack
-      uint32_t pk[32];
+      uint32_t pk[16];
       float sum = 0.f;
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
+      for (int j = 0; j < 16; ++j) {
         const float p0 = exp2f(__uint_as_float(v[2 * j]) - m_used);
         const float p1 = exp2f(__uint_as_float(v[2 * j + 1]) - m_used);
         sum += p0 + p1;
@@ -265,19 +287,19 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
         ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done), (i - 1) & 1, p.status));
         if (!ok) break;
       }
-      if (hi == 0) {
-        uint8_t* prow = sm.p + row * 128;
+      {
+        uint8_t* prow = sm.p + row * 128;    // keys 32*hi .. +31 of this row: 16-byte chunks 4*hi .. 4*hi+3
 #pragma unroll
-        for (int c = 0; c < 8; ++c)
-          *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+        for (int c = 0; c < 4; ++c)
+          *reinterpret_cast<uint4*>(prow + (((4 * hi + c) ^ (row & 7)) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
         tc::fence_proxy_async();
       }
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(smem_u32(&sm.p_ready));
     }
     // ---- epilogue: O / l
-    const float l_row = __shfl_sync(0xffffffffu, l_run, r16);
-    const float m_row = __shfl_sync(0xffffffffu, m_used, r16);
+    const float l_row = l_run + __shfl_xor_sync(0xffffffffu, l_run, 16);
+    const float m_row = m_used;
     bool have_o = ok && n_tiles > 0;
     if (have_o) have_o = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done), (n_tiles - 1) & 1, p.status));
     tc::fence_after_sync();

@@ -31,6 +31,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Non-blocking probe of a phase.
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 // Waits for the phase of the given parity, for at most ~2^31 cycles (about a second).  On expiry the
 // status word gets kDevTimeout and false is returned; the caller leaves its loop and the kernel ends
 // normally.
@@ -139,6 +151,13 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo,
   d |= 1ull << 46;  // descriptor version of this architecture
   d |= 2ull << 61;  // 128-byte swizzle
   return d;
+}
+
+// The same descriptor moved by `bytes` inside shared memory: the start-address field holds address >> 4 in
+// the low 14 bits and never carries out (shared memory is < 256 KB), so one 32-bit add on the low word does it.
+__device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t bytes) {
+  const uint32_t lo = static_cast<uint32_t>(desc) + (bytes >> 4);
+  return (desc & 0xffffffff00000000ull) | lo;
 }
 
 // Instruction descriptor: bf16 x bf16 -> fp32, dense.  a_mn / b_mn = 1 for an MN-major operand.
