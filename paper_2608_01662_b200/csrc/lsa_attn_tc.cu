@@ -2,23 +2,25 @@
 // (H = 64 heads, d_qk = 576, d_v = 512, the value is the first 512 dims of the key row).
 //
 // One thread block = one query (or one split of one sequence's rows in decode).  Its 64 heads are the M = 64
-// rows of every MMA; the attended cache rows stream through two 64-key shared tiles, each made of two 32-key
-// halves:
+// rows of every MMA; the attended cache rows stream through two 64-key shared tiles:
 //
-//   warps 5-8   gather: rows [sink | sparse | window] -> 128B-swizzled K-major half-tiles with coalesced 16-byte
-//               cp.async (one warp per half-tile), completion through an mbarrier
-//   warp 4      issues tcgen05.mma:  S = Q K^T   (M64 N32 K16 x 36 per half; both operands K-major)
-//                                    O += P V    (M64 N256 K16 x 8; V is the same shared tile read MN-major,
-//                                                 so each cache row is fetched once)
-//               and takes whichever of "next Q K^T" / "next P V" is ready, so the tensor pipe keeps working
-//               while a softmax or a gather is in flight
-//   warps 0-3   softmax: tcgen05.ld S, running max with lazy rescaling of O, exp2, fp32 row sums, P as bf16 ->
-//               shared A operand; at the end O / l -> bf16
+//   warps 5-8   gather: rows [sink | sparse | window] -> 128B-swizzled K-major tiles with coalesced 16-byte
+//               cp.async (two warps per tile buffer), completion through an mbarrier
+//   warp 4      one thread issues every tcgen05.mma.  Back-to-back MMAs into one accumulator run far below
+//               the pipe's rate at these small shapes, so each product is cut into two independent
+//               accumulation chains that alternate instruction by instruction:
+//                 S = Q K^T   two partial sums of 18 K-steps each (M64 N64 K16)
+//                 O += P V    value dims 0-255 and 256-511 (M64 N256 K16 x 4 each); V is the key tile read
+//                             MN-major, so each cache row is fetched once
+//               The thread takes whichever of "next Q K^T" / "next P V" is ready.
+//   warps 0-3   softmax: tcgen05.ld of both partial sums, add, running max with lazy rescaling of O, exp2,
+//               fp32 row sums, P as bf16 -> shared A operand; at the end O / l -> bf16
 //
 // An M = 64 accumulator occupies 16 of the 32 lanes of each TMEM quarter, so two of them share a column range:
 //   columns   0-255   O[:, 0:256] in lanes 0-15, O[:, 256:512] in lanes 16-31
-//   columns 256-319   S buffers 0 and 1 (32 columns each): keys 0-31 of the tile in lanes 0-15, keys 32-63 in
-//                     lanes 16-31, so that lanes l and l+16 of a softmax warp share one head row
+//   columns 256-383   S buffers 0 and 1 (64 columns each): the first chain's partial sum in lanes 0-15, the second's in
+//                     lanes 16-31.  Lanes l and l+16 of a softmax warp share head row l: they swap halves, so
+//                     lane l finishes keys 0-31 and lane l+16 keys 32-63 of the tile.
 #include "lsa_internal.h"
 #include "lsa_tc.cuh"
 
@@ -31,9 +33,9 @@ constexpr int kTileKeys = 64;
 constexpr int kAtoms = kDQK / 64;            // 9 column blocks of 64 dims (128 bytes) per row
 constexpr int kAtomBytes = 64 * 128;         // 64 rows x 128 bytes
 constexpr int kHalfKeys = 32;
-constexpr int kHalfAtomBytes = kHalfKeys * 128;
-constexpr int kSoftmaxWarps = 4, kLoadWarps = 4;
-constexpr int kThreadsAttnTc = 32 * (kSoftmaxWarps + 1 + kLoadWarps);
+
+constexpr int kSoftmaxWarps = 4, kMmaWarps = 1, kLoadWarps = 4;
+constexpr int kThreadsAttnTc = 32 * (kSoftmaxWarps + kMmaWarps + kLoadWarps);
 constexpr uint32_t kTmemColsAttn = 512;
 constexpr uint32_t kColS = 256;              // first column of the S buffers
 constexpr float kLog2eTc = 1.4426950408889634f;
@@ -41,7 +43,7 @@ constexpr float kRescaleGap = 8.f;           // rescale O only when the row max 
 
 struct AttnTcSmem {
   alignas(1024) uint8_t q[kAtoms][kAtomBytes];
-  alignas(1024) uint8_t k[2][2][kAtoms][kHalfAtomBytes];   // [tile buffer][half][column block][32 rows x 128 B]
+  alignas(1024) uint8_t k[2][kAtoms][kAtomBytes];   // [tile buffer][column block][64 rows x 128 B]
   alignas(1024) uint8_t p[kAtomBytes];
   alignas(8) uint64_t q_full, k_full[2], k_empty[2], s_full[2], s_free[2], p_ready, pv_done;
   uint32_t tmem_slot;
@@ -80,17 +82,19 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
   const int tile_begin = split * tiles_per;
   const int n_tiles = max(0, min(tiles_all, tile_begin + tiles_per) - tile_begin);
 
+  if (tc::status_raised(p.status)) return;   // an earlier block of this launch gave up on a wait
+
   // ---- set-up
   if (tid == 0) {
     tc::mbar_init(smem_u32(&sm.q_full), 32 * kLoadWarps);
     for (int b = 0; b < 2; ++b) {
       tc::mbar_init(smem_u32(&sm.k_full[b]), 32 * kLoadWarps / 2);
-      tc::mbar_init(smem_u32(&sm.k_empty[b]), 1);
-      tc::mbar_init(smem_u32(&sm.s_full[b]), 1);
+      tc::mbar_init(smem_u32(&sm.k_empty[b]), kMmaWarps);
+      tc::mbar_init(smem_u32(&sm.s_full[b]), kMmaWarps);
       tc::mbar_init(smem_u32(&sm.s_free[b]), kSoftmaxWarps);
     }
     tc::mbar_init(smem_u32(&sm.p_ready), kSoftmaxWarps);
-    tc::mbar_init(smem_u32(&sm.pv_done), 1);
+    tc::mbar_init(smem_u32(&sm.pv_done), kMmaWarps);
     tc::fence_mbar_init();
   }
   if (warp == kSoftmaxWarps) {
@@ -102,9 +106,9 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
   tc::fence_after_sync();
   const uint32_t tmem_base = sm.tmem_slot;
 
-  if (warp > kSoftmaxWarps) {
+  if (warp >= kSoftmaxWarps + kMmaWarps) {
     // ================= gather warps =================
-    const int lt = tid - 32 * (kSoftmaxWarps + 1);   // 0..127
+    const int lt = tid - 32 * (kSoftmaxWarps + kMmaWarps);   // 0..127
     {
       // Q: 64 rows of 1152 contiguous bytes
       const uint8_t* qg = reinterpret_cast<const uint8_t*>(p.q) + static_cast<int64_t>(qi) * kH * kDQK * 2;
@@ -134,7 +138,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
         const int nb = row >= 0 ? 16 : 0;
 #pragma unroll
         for (int c = lane; c < 72; c += 32)
-          cp_async16(smem_u32(sm.k[grp][wg][c >> 3]) + rr * 128 + (((c & 7) ^ (rr & 7)) << 4), src + c * 16, nb);
+          cp_async16(smem_u32(sm.k[grp][c >> 3]) + (kHalfKeys * wg + rr) * 128 + (((c & 7) ^ (rr & 7)) << 4), src + c * 16, nb);
       }
       cp_async_commit();
       cp_async_wait<0>();
@@ -145,51 +149,50 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
   } else if (warp == kSoftmaxWarps) {
     // ================= MMA issuer =================
     if (lane == 0 && n_tiles > 0) {
-      constexpr uint32_t idesc_qk = tc::idesc_bf16(kH, kHalfKeys, 0, 0);
+      constexpr uint32_t idesc_qk = tc::idesc_bf16(kH, kTileKeys, 0, 0);
       constexpr uint32_t idesc_pv = tc::idesc_bf16(kH, 256, 0, 1);   // B = V read MN-major
       bool ok = tc::mbar_wait(smem_u32(&sm.q_full), 0, p.status);
-      // Descriptors are built once; inside the loops only the start-address word moves (one add per operand):
-      // a single thread has to issue ~80 MMAs per tile, so its instruction count per MMA matters.
+      // Descriptors are built once; inside the loops only the start-address word moves (one add per operand).
+      constexpr uint32_t kBufBytes = kAtoms * kAtomBytes;
+      constexpr int kChain = kAtoms * 4 / 2;   // 18 of the 36 K-steps of 16 dims per accumulation chain
       const uint64_t dq0 = tc::smem_desc_sw128(smem_u32(sm.q), 16, 1024);
       const uint64_t dp0 = tc::smem_desc_sw128(smem_u32(sm.p), 16, 1024);
-      const uint64_t dk0 = tc::smem_desc_sw128(smem_u32(sm.k), 16, 1024);              // K-major view (Q K^T)
-      const uint64_t dv0 = tc::smem_desc_sw128(smem_u32(sm.k), kHalfAtomBytes, 1024);  // MN-major view (P V)
-      constexpr uint32_t kBufBytes = 2 * kAtoms * kHalfAtomBytes, kHalfBytes = kAtoms * kHalfAtomBytes;
-      auto issue_qk = [&](int i) {   // S_i = Q K_i^T, keys 0-31 -> lanes 0-15, keys 32-63 -> lanes 16-31
+      const uint64_t dk0 = tc::smem_desc_sw128(smem_u32(sm.k), 16, 1024);           // K-major view (Q K^T)
+      const uint64_t dv0 = tc::smem_desc_sw128(smem_u32(sm.k), kAtomBytes, 1024);   // MN-major view (P V)
+      constexpr uint32_t kLane16 = 16u << 16;
+      auto issue_qk = [&](int i) {   // S_i = Q K_i^T as two partial sums (chains alternate, MMA by MMA)
         const int b = i & 1;
         tc::fence_after_sync();
+        const uint32_t d = tmem_base + kColS + b * kTileKeys;
+        const uint64_t dkb = tc::desc_advance(dk0, b * kBufBytes);
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const uint32_t d = tmem_base + (static_cast<uint32_t>(16 * half) << 16) + kColS + b * kHalfKeys;
-          const uint64_t dkb = tc::desc_advance(dk0, b * kBufBytes + half * kHalfBytes);
+        for (int s = 0; s < kChain; ++s) {
 #pragma unroll
-          for (int a = 0; a < kAtoms; ++a) {
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              tc::umma_ss(d, tc::desc_advance(dq0, a * kAtomBytes + kk * 32), tc::desc_advance(dkb, a * kHalfAtomBytes + kk * 32),
-                          idesc_qk, (a | kk) != 0);
+          for (int x = 0; x < 2; ++x) {
+            const int ks = x * kChain + s;                    // K-step: column block ks/4, 32-byte slice ks%4
+            const uint32_t off = (ks >> 2) * kAtomBytes + (ks & 3) * 32;
+            tc::umma_ss(d + x * kLane16, tc::desc_advance(dq0, off), tc::desc_advance(dkb, off), idesc_qk, s != 0);
           }
         }
         tc::umma_commit(smem_u32(&sm.s_full[b]));
       };
-      auto issue_pv = [&](int j) {   // O += P_j V_j
+      auto issue_pv = [&](int j) {   // O += P_j V_j, value dims 0-255 and 256-511 alternate
         const int b = j & 1;
         tc::fence_after_sync();
+        const uint64_t dvb = tc::desc_advance(dv0, b * kBufBytes);
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {          // value dims 256*half .. +255
-          const uint32_t d = tmem_base + (static_cast<uint32_t>(16 * half) << 16);
-          const uint64_t dvb = tc::desc_advance(dv0, b * kBufBytes + 4 * half * kHalfAtomBytes);
+        for (int kk = 0; kk < kTileKeys / 16; ++kk) {   // keys 16*kk .. +15
 #pragma unroll
-          for (int kk = 0; kk < kTileKeys / 16; ++kk)   // keys 16*kk .. +15: half-tile kk/2, rows 16*(kk%2) ..
-            tc::umma_ss(d, tc::desc_advance(dp0, kk * 32), tc::desc_advance(dvb, (kk >> 1) * kHalfBytes + (kk & 1) * 2048),
-                        idesc_pv, (j > 0) || (kk > 0));
+          for (int x = 0; x < 2; ++x)
+            tc::umma_ss(tmem_base + x * kLane16, tc::desc_advance(dp0, kk * 32),
+                        tc::desc_advance(dvb, 4 * x * kAtomBytes + kk * 2048), idesc_pv, (j > 0) || (kk > 0));
         }
         tc::umma_commit(smem_u32(&sm.k_empty[b]));
         tc::umma_commit(smem_u32(&sm.pv_done));
       };
       // Two in-order queues, "next Q K^T" (at most one tile ahead of the softmax it feeds) and "next P V".
       int qk_next = 0, pv_next = 0;
-      const long long t_start = clock64();
+      long long t_idle = clock64();
       uint32_t spins = 0;
       while (ok && pv_next < n_tiles) {
         bool did = false;
@@ -207,9 +210,14 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
         }
         if (did) {
           spins = 0;
-        } else if ((++spins & 1023u) == 0 && clock64() - t_start > tc::kWaitCycles * 8) {
-          report_status(p.status, kDevTimeout);   // bounded: nothing became ready for seconds
-          ok = false;
+          t_idle = clock64();
+        } else if ((++spins & 255u) == 0) {
+          if (tc::status_raised(p.status)) {
+            ok = false;
+          } else if (clock64() - t_idle > tc::kWaitCycles) {
+            report_status(p.status, kDevTimeout);   // bounded: nothing became ready for about a second
+            ok = false;
+          }
         }
       }
     }
@@ -228,11 +236,22 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       if (!ok) break;
       tc::fence_after_sync();
       uint32_t v[32];
-      tc::tmem_ld32(tmem_base + lane_addr + kColS + b * kHalfKeys, v);
-      tc::tmem_ld_wait();
+      {
+        // this lane holds one chain's partial sums for all 64 keys; its partner lane (l ^ 16) the other's.
+        // Lane l keeps keys 0-31, lane l+16 keys 32-63: send the half the partner finishes, add the one it sends.
+        uint32_t s64[64];
+        tc::tmem_ld64(tmem_base + lane_addr + kColS + b * kTileKeys, s64);
+        tc::tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float give = __uint_as_float(hi ? s64[j] : s64[32 + j]);
+          const float keep = __uint_as_float(hi ? s64[32 + j] : s64[j]);
+          v[j] = __float_as_uint(keep + __shfl_xor_sync(0xffffffffu, give, 16));
+        }
+      }
       tc::fence_before_sync();
       __syncwarp();
-      if (lane == 0) tc::mbar_arrive(smem_u32(&sm.s_free[b]));
+      if (lane == 0) tc::mbar_arrive(smem_u32(&sm.s_free[b]));   // S buffer b may be overwritten
       // logits in log2 units, ragged tail masked
       const int n_valid = n_tot - (tile_begin + i) * kTileKeys - kHalfKeys * hi;   // keys of this lane's half that exist
       float mx = -INFINITY;

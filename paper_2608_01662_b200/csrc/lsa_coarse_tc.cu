@@ -58,6 +58,7 @@ coarse_score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
   const int64_t t_max = p.q_pos0 + q0 + nq - 1;
   const int64_t t_need = (static_cast<int64_t>(p.M) + p.S / p.P) * p.P + p.W;  // first query with more than M eligible pages
   if (t_max < t_need) return;
+  if (tc::status_raised(p.status)) return;   // an earlier block of this launch gave up on a wait
   const int64_t hi_max = t_max - p.W;
   const int spp = p.P / p.B;
   const int n_tiles = static_cast<int>(hi_max / (static_cast<int64_t>(kTileM) * p.B)) + 1;

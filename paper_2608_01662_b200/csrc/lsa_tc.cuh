@@ -45,17 +45,25 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
 }
 // Waits for the phase of the given parity, for at most ~2^31 cycles (about a second).  On expiry the
 // status word gets kDevTimeout and false is returned; the caller leaves its loop and the kernel ends
-// normally.
+// normally; every other wait of the grid then ends within a few hundred polls, and blocks that start later
+// return at once (see status_raised), so a failed launch costs about a second in total.
 constexpr long long kWaitCycles = 1ll << 31;
+__device__ __forceinline__ bool status_raised(const int* status) {
+  return status != nullptr && *reinterpret_cast<const volatile int*>(status) != 0;
+}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
 #pragma unroll 1
   for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 0 && clock64() - t0 > kWaitCycles) {
-      report_status(status, kDevTimeout);
-      return false;
+    if ((i & 255u) == 0) {
+      // once any wait anywhere in the grid has given up, everybody stops waiting
+      if (status_raised(status)) return false;
+      if (clock64() - t0 > kWaitCycles) {
+        report_status(status, kDevTimeout);
+        return false;
+      }
     }
   }
 }
