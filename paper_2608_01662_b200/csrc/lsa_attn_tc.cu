@@ -34,7 +34,7 @@ constexpr int kAtoms = kDQK / 64;            // 9 column blocks of 64 dims (128 
 constexpr int kAtomBytes = 64 * 128;         // 64 rows x 128 bytes
 constexpr int kHalfKeys = 32;
 
-constexpr int kSoftmaxWarps = 4, kMmaWarps = 1, kLoadWarps = 4;
+constexpr int kSoftmaxWarps = 4, kMmaWarps = 2, kLoadWarps = 4;
 constexpr int kThreadsAttnTc = 32 * (kSoftmaxWarps + kMmaWarps + kLoadWarps);
 constexpr uint32_t kTmemColsAttn = 512;
 constexpr uint32_t kColS = 256;              // first column of the S buffers
@@ -146,8 +146,9 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       tc::mbar_arrive(smem_u32(&sm.k_full[grp]));
       my_row = next_row;
     }
-  } else if (warp == kSoftmaxWarps) {
-    // ================= MMA issuer =================
+  } else if (warp >= kSoftmaxWarps) {
+    // ================= MMA issuers =================
+    const int x = warp - kSoftmaxWarps;   // accumulation chain of this issuer
     if (lane == 0 && n_tiles > 0) {
       constexpr uint32_t idesc_qk = tc::idesc_bf16(kH, kTileKeys, 0, 0);
       constexpr uint32_t idesc_pv = tc::idesc_bf16(kH, 256, 0, 1);   // B = V read MN-major
@@ -167,12 +168,9 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
         const uint64_t dkb = tc::desc_advance(dk0, b * kBufBytes);
 #pragma unroll
         for (int s = 0; s < kChain; ++s) {
-#pragma unroll
-          for (int x = 0; x < 2; ++x) {
-            const int ks = x * kChain + s;                    // K-step: column block ks/4, 32-byte slice ks%4
-            const uint32_t off = (ks >> 2) * kAtomBytes + (ks & 3) * 32;
-            tc::umma_ss(d + x * kLane16, tc::desc_advance(dq0, off), tc::desc_advance(dkb, off), idesc_qk, s != 0);
-          }
+          const int ks = x * kChain + s;                    // K-step: column block ks/4, 32-byte slice ks%4
+          const uint32_t off = (ks >> 2) * kAtomBytes + (ks & 3) * 32;
+          tc::umma_ss(d + x * kLane16, tc::desc_advance(dq0, off), tc::desc_advance(dkb, off), idesc_qk, s != 0);
         }
         tc::umma_commit(smem_u32(&sm.s_full[b]));
       };
@@ -181,12 +179,9 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
         tc::fence_after_sync();
         const uint64_t dvb = tc::desc_advance(dv0, b * kBufBytes);
 #pragma unroll
-        for (int kk = 0; kk < kTileKeys / 16; ++kk) {   // keys 16*kk .. +15
-#pragma unroll
-          for (int x = 0; x < 2; ++x)
-            tc::umma_ss(tmem_base + x * kLane16, tc::desc_advance(dp0, kk * 32),
-                        tc::desc_advance(dvb, 4 * x * kAtomBytes + kk * 2048), idesc_pv, (j > 0) || (kk > 0));
-        }
+        for (int kk = 0; kk < kTileKeys / 16; ++kk)   // keys 16*kk .. +15
+          tc::umma_ss(tmem_base + x * kLane16, tc::desc_advance(dp0, kk * 32),
+                      tc::desc_advance(dvb, 4 * x * kAtomBytes + kk * 2048), idesc_pv, (j > 0) || (kk > 0));
         tc::umma_commit(smem_u32(&sm.k_empty[b]));
         tc::umma_commit(smem_u32(&sm.pv_done));
       };
