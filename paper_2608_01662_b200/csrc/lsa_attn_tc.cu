@@ -14,13 +14,15 @@
 //                             MN-major, so each cache row is fetched once
 //               The thread takes whichever of "next Q K^T" / "next P V" is ready.
 //   warps 0-3   softmax: tcgen05.ld of both partial sums, add, running max with lazy rescaling of O, exp2,
-//               fp32 row sums, P as bf16 -> shared A operand; at the end O / l -> bf16
+//               fp32 row sums, P as bf16 -> tensor memory (A operand of P V); at the end O / l -> bf16
 //
 // An M = 64 accumulator occupies 16 of the 32 lanes of each TMEM quarter, so two of them share a column range:
 //   columns   0-255   O[:, 0:256] in lanes 0-15, O[:, 256:512] in lanes 16-31
 //   columns 256-383   S buffers 0 and 1 (64 columns each): the first chain's partial sum in lanes 0-15, the second's in
 //                     lanes 16-31.  Lanes l and l+16 of a softmax warp share head row l: they swap halves, so
 //                     lane l finishes keys 0-31 and lane l+16 keys 32-63 of the tile.
+//   columns 384-447   P buffers 0 and 1 (32 columns = 64 bf16 each), one copy per lane half, because an MMA reads
+//                     its TMEM operand from the lanes its accumulator lives in
 #include "lsa_internal.h"
 #include "lsa_tc.cuh"
 
@@ -37,15 +39,15 @@ constexpr int kHalfKeys = 32;
 constexpr int kSoftmaxWarps = 4, kMmaWarps = 2, kLoadWarps = 4;
 constexpr int kThreadsAttnTc = 32 * (kSoftmaxWarps + kMmaWarps + kLoadWarps);
 constexpr uint32_t kTmemColsAttn = 512;
-constexpr uint32_t kColS = 256;              // first column of the S buffers
+constexpr uint32_t kColS = 256;              // first column of the S buffers (2 x 64 columns)
+constexpr uint32_t kColP = 384;              // first column of the P buffers (2 x 32 columns of packed bf16)
 constexpr float kLog2eTc = 1.4426950408889634f;
 constexpr float kRescaleGap = 8.f;           // rescale O only when the row max grows by more than 2^8
 
 struct AttnTcSmem {
   alignas(1024) uint8_t q[kAtoms][kAtomBytes];
   alignas(1024) uint8_t k[2][kAtoms][kAtomBytes];   // [tile buffer][column block][64 rows x 128 B]
-  alignas(1024) uint8_t p[kAtomBytes];
-  alignas(8) uint64_t q_full, k_full[2], k_empty[2], s_full[2], s_free[2], p_ready, pv_done;
+  alignas(8) uint64_t q_full, k_full[2], k_empty[2], s_full[2], s_free[2], p_ready, pv_done[2];
   uint32_t tmem_slot;
 };
 
@@ -94,7 +96,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       tc::mbar_init(smem_u32(&sm.s_free[b]), kSoftmaxWarps);
     }
     tc::mbar_init(smem_u32(&sm.p_ready), kSoftmaxWarps);
-    tc::mbar_init(smem_u32(&sm.pv_done), kMmaWarps);
+    for (int b = 0; b < 2; ++b) tc::mbar_init(smem_u32(&sm.pv_done[b]), kMmaWarps);
     tc::fence_mbar_init();
   }
   if (warp == kSoftmaxWarps) {
@@ -157,7 +159,6 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       constexpr uint32_t kBufBytes = kAtoms * kAtomBytes;
       constexpr int kChain = kAtoms * 4 / 2;   // 18 of the 36 K-steps of 16 dims per accumulation chain
       const uint64_t dq0 = tc::smem_desc_sw128(smem_u32(sm.q), 16, 1024);
-      const uint64_t dp0 = tc::smem_desc_sw128(smem_u32(sm.p), 16, 1024);
       const uint64_t dk0 = tc::smem_desc_sw128(smem_u32(sm.k), 16, 1024);           // K-major view (Q K^T)
       const uint64_t dv0 = tc::smem_desc_sw128(smem_u32(sm.k), kAtomBytes, 1024);   // MN-major view (P V)
       constexpr uint32_t kLane16 = 16u << 16;
@@ -180,10 +181,10 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
         const uint64_t dvb = tc::desc_advance(dv0, b * kBufBytes);
 #pragma unroll
         for (int kk = 0; kk < kTileKeys / 16; ++kk)   // keys 16*kk .. +15
-          tc::umma_ss(tmem_base + x * kLane16, tc::desc_advance(dp0, kk * 32),
+          tc::umma_ts(tmem_base + x * kLane16, tmem_base + x * kLane16 + kColP + b * 32 + kk * 8,
                       tc::desc_advance(dvb, 4 * x * kAtomBytes + kk * 2048), idesc_pv, (j > 0) || (kk > 0));
         tc::umma_commit(smem_u32(&sm.k_empty[b]));
-        tc::umma_commit(smem_u32(&sm.pv_done));
+        tc::umma_commit(smem_u32(&sm.pv_done[b]));
       };
       // Two in-order queues, "next Q K^T" (at most one tile ahead of the softmax it feeds) and "next P V".
       int qk_next = 0, pv_next = 0;
@@ -265,12 +266,10 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
         alpha = exp2f(m_used - mx);
         m_used = mx;
       }
-      bool waited_pv = false;
       if (__any_sync(0xffffffffu, alpha != 1.f)) {
         // O may be touched only between P V of tile i-1 (done) and P V of tile i (not yet released)
-        ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done), (i - 1) & 1, p.status));
+        ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done[(i - 1) & 1]), ((i - 1) >> 1) & 1, p.status));
         if (!ok) break;
-        waited_pv = true;
         tc::fence_after_sync();
 #pragma unroll 1
         for (int c = 0; c < 256; c += 64) {
@@ -296,17 +295,25 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
         pk[j] = pack_bf16(p0, p1);
       }
       l_run += sum;
-      // the P tile is free once P V of the previous tile has read it
-      if (i > 0 && !waited_pv) {
-        ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done), (i - 1) & 1, p.status));
+      // P buffer b was last read by P V of tile i-2
+      if (i >= 2) {
+        ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done[b]), ((i >> 1) & 1) ^ 1, p.status));
         if (!ok) break;
+        tc::fence_after_sync();
       }
       {
-        uint8_t* prow = sm.p + row * 128;    // keys 32*hi .. +31 of this row: 16-byte chunks 4*hi .. 4*hi+3
+        // The A operand of P V sits in tensor memory, in the lanes of the accumulator it feeds: both lanes of a
+        // row need all 64 keys, so the two halves are swapped in, then written as 32 columns of packed bf16.
+        uint32_t full[32];
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-          *reinterpret_cast<uint4*>(prow + (((4 * hi + c) ^ (row & 7)) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-        tc::fence_proxy_async();
+        for (int j = 0; j < 16; ++j) {
+          const uint32_t other = __shfl_xor_sync(0xffffffffu, pk[j], 16);
+          full[j] = hi ? other : pk[j];
+          full[16 + j] = hi ? pk[j] : other;
+        }
+        tc::tmem_st32(tmem_base + lane_addr + kColP + b * 32, full);
+        tc::tmem_st_wait();
+        tc::fence_before_sync();
       }
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(smem_u32(&sm.p_ready));
@@ -315,7 +322,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     const float l_row = l_run + __shfl_xor_sync(0xffffffffu, l_run, 16);
     const float m_row = m_used;
     bool have_o = ok && n_tiles > 0;
-    if (have_o) have_o = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done), (n_tiles - 1) & 1, p.status));
+    if (have_o) have_o = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done[(n_tiles - 1) & 1]), ((n_tiles - 1) >> 1) & 1, p.status));
     tc::fence_after_sync();
     const float inv = (have_o && l_row > 0.f) ? 1.f / l_row : 0.f;
     const int d0 = hi * 256;
