@@ -36,18 +36,18 @@ constexpr int kAtoms = kDQK / 64;            // 9 column blocks of 64 dims (128 
 constexpr int kAtomBytes = 64 * 128;         // 64 rows x 128 bytes
 constexpr int kHalfKeys = 32;
 
-constexpr int kSoftmaxWarps = 4, kMmaWarps = 2, kLoadWarps = 4;
+constexpr int kSoftmaxWarps = 4, kMmaWarps = 4, kLoadWarps = 4;
 constexpr int kThreadsAttnTc = 32 * (kSoftmaxWarps + kMmaWarps + kLoadWarps);
 constexpr uint32_t kTmemColsAttn = 512;
-constexpr uint32_t kColS = 256;              // first column of the S buffers (2 x 64 columns)
-constexpr uint32_t kColP = 384;              // first column of the P buffers (2 x 32 columns of packed bf16)
+constexpr uint32_t kColS = 256;              // two S buffers of 128 columns: two column sets of 64 partial sums
+constexpr uint32_t kSBuf = 128;
 constexpr float kLog2eTc = 1.4426950408889634f;
 constexpr float kRescaleGap = 8.f;           // rescale O only when the row max grows by more than 2^8
 
 struct AttnTcSmem {
   alignas(1024) uint8_t q[kAtoms][kAtomBytes];
   alignas(1024) uint8_t k[2][kAtoms][kAtomBytes];   // [tile buffer][column block][64 rows x 128 B]
-  alignas(8) uint64_t q_full, k_full[2], k_empty[2], s_full[2], s_free[2], p_ready, pv_done[2];
+  alignas(8) uint64_t q_full, k_full[2], k_empty[2], s_full[2], p_ready, pv_done[2];
   uint32_t tmem_slot;
 };
 
@@ -93,7 +93,6 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       tc::mbar_init(smem_u32(&sm.k_full[b]), 32 * kLoadWarps / 2);
       tc::mbar_init(smem_u32(&sm.k_empty[b]), kMmaWarps);
       tc::mbar_init(smem_u32(&sm.s_full[b]), kMmaWarps);
-      tc::mbar_init(smem_u32(&sm.s_free[b]), kSoftmaxWarps);
     }
     tc::mbar_init(smem_u32(&sm.p_ready), kSoftmaxWarps);
     for (int b = 0; b < 2; ++b) tc::mbar_init(smem_u32(&sm.pv_done[b]), kMmaWarps);
@@ -150,39 +149,44 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     }
   } else if (warp >= kSoftmaxWarps) {
     // ================= MMA issuers =================
-    const int x = warp - kSoftmaxWarps;   // accumulation chain of this issuer
+    const int x = warp - kSoftmaxWarps;   // 0..3: accumulation chain of this issuer
     if (lane == 0 && n_tiles > 0) {
       constexpr uint32_t idesc_qk = tc::idesc_bf16(kH, kTileKeys, 0, 0);
-      constexpr uint32_t idesc_pv = tc::idesc_bf16(kH, 256, 0, 1);   // B = V read MN-major
+      constexpr uint32_t idesc_pv = tc::idesc_bf16(kH, 128, 0, 1);   // B = V read MN-major
       bool ok = tc::mbar_wait(smem_u32(&sm.q_full), 0, p.status);
       // Descriptors are built once; inside the loops only the start-address word moves (one add per operand).
       constexpr uint32_t kBufBytes = kAtoms * kAtomBytes;
-      constexpr int kChain = kAtoms * 4 / 2;   // 18 of the 36 K-steps of 16 dims per accumulation chain
+      constexpr int kChain = kAtoms * 4 / kMmaWarps;   // 9 of the 36 K-steps of 16 dims per accumulation chain
       const uint64_t dq0 = tc::smem_desc_sw128(smem_u32(sm.q), 16, 1024);
       const uint64_t dk0 = tc::smem_desc_sw128(smem_u32(sm.k), 16, 1024);           // K-major view (Q K^T)
-      const uint64_t dv0 = tc::smem_desc_sw128(smem_u32(sm.k), kAtomBytes, 1024);   // MN-major view (P V)
+      const uint64_t dv0 = tc::desc_advance(tc::smem_desc_sw128(smem_u32(sm.k), kAtomBytes, 1024), 2 * x * kAtomBytes);  // MN-major view (P V)
       constexpr uint32_t kLane16 = 16u << 16;
-      auto issue_qk = [&](int i) {   // S_i = Q K_i^T as two partial sums (chains alternate, MMA by MMA)
+      // Q K^T: partial sum x goes to lane half x&1, column set x>>1 of the S buffer
+      const uint32_t s_dst = tmem_base + (x & 1) * kLane16 + kColS + (x >> 1) * kTileKeys;
+      // P V: value dims 128x .. 128x+127 = columns 128*(x&1) .. of the accumulator in lane half x>>1; P is read
+      // from the same lane half
+      const uint32_t o_dst = tmem_base + (x >> 1) * kLane16 + (x & 1) * 128;
+      const uint32_t p_src = tmem_base + (x >> 1) * kLane16 + kColS;
+      auto issue_qk = [&](int i) {   // partial S_i over this issuer's K-steps
         const int b = i & 1;
         tc::fence_after_sync();
-        const uint32_t d = tmem_base + kColS + b * kTileKeys;
+        const uint32_t d = s_dst + b * kSBuf;
         const uint64_t dkb = tc::desc_advance(dk0, b * kBufBytes);
 #pragma unroll
         for (int s = 0; s < kChain; ++s) {
           const int ks = x * kChain + s;                    // K-step: column block ks/4, 32-byte slice ks%4
           const uint32_t off = (ks >> 2) * kAtomBytes + (ks & 3) * 32;
-          tc::umma_ss(d + x * kLane16, tc::desc_advance(dq0, off), tc::desc_advance(dkb, off), idesc_qk, s != 0);
+          tc::umma_ss(d, tc::desc_advance(dq0, off), tc::desc_advance(dkb, off), idesc_qk, s != 0);
         }
         tc::umma_commit(smem_u32(&sm.s_full[b]));
       };
-      auto issue_pv = [&](int j) {   // O += P_j V_j, value dims 0-255 and 256-511 alternate
+      auto issue_pv = [&](int j) {   // O[:, 128x : 128x+128] += P_j V_j
         const int b = j & 1;
         tc::fence_after_sync();
         const uint64_t dvb = tc::desc_advance(dv0, b * kBufBytes);
 #pragma unroll
         for (int kk = 0; kk < kTileKeys / 16; ++kk)   // keys 16*kk .. +15
-          tc::umma_ts(tmem_base + x * kLane16, tmem_base + x * kLane16 + kColP + b * 32 + kk * 8,
-                      tc::desc_advance(dvb, 4 * x * kAtomBytes + kk * 2048), idesc_pv, (j > 0) || (kk > 0));
+          tc::umma_ts(o_dst, p_src + b * kSBuf + kk * 8, tc::desc_advance(dvb, kk * 2048), idesc_pv, (j > 0) || (kk > 0));
         tc::umma_commit(smem_u32(&sm.k_empty[b]));
         tc::umma_commit(smem_u32(&sm.pv_done[b]));
       };
@@ -194,8 +198,9 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
         bool did = false;
         if (qk_next < n_tiles && qk_next <= pv_next + 1) {
           const int b = qk_next & 1;
+          // S buffer b also holds P of tile qk_next-2: it is free once that tile's P V has completed
           if (tc::mbar_test(smem_u32(&sm.k_full[b]), (qk_next >> 1) & 1) &&
-              tc::mbar_test(smem_u32(&sm.s_free[b]), ((qk_next >> 1) & 1) ^ 1)) {
+              tc::mbar_test(smem_u32(&sm.pv_done[b]), ((qk_next >> 1) & 1) ^ 1)) {
             issue_qk(qk_next++);
             did = true;
           }
@@ -231,13 +236,21 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.s_full[b]), (i >> 1) & 1, p.status));
       if (!ok) break;
       tc::fence_after_sync();
+      const uint32_t s_addr = tmem_base + lane_addr + kColS + b * kSBuf;
       uint32_t v[32];
       {
-        // this lane holds one chain's partial sums for all 64 keys; its partner lane (l ^ 16) the other's.
-        // Lane l keeps keys 0-31, lane l+16 keys 32-63: send the half the partner finishes, add the one it sends.
+        // This lane holds two chains' partial sums for all 64 keys (column sets 0 and 1); its partner lane (l ^ 16)
+        // the other two.  Lane l keeps keys 0-31, lane l+16 keys 32-63: add the own pair, send the half the
+        // partner finishes, add the one it sends.
         uint32_t s64[64];
-        tc::tmem_ld64(tmem_base + lane_addr + kColS + b * kTileKeys, s64);
-        tc::tmem_ld_wait();
+        {
+          uint32_t t64[64];
+          tc::tmem_ld64(s_addr, s64);
+          tc::tmem_ld64(s_addr + kTileKeys, t64);
+          tc::tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 64; ++j) s64[j] = __float_as_uint(__uint_as_float(s64[j]) + __uint_as_float(t64[j]));
+        }
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           const float give = __uint_as_float(hi ? s64[j] : s64[32 + j]);
@@ -245,9 +258,6 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
           v[j] = __float_as_uint(keep + __shfl_xor_sync(0xffffffffu, give, 16));
         }
       }
-      tc::fence_before_sync();
-      __syncwarp();
-      if (lane == 0) tc::mbar_arrive(smem_u32(&sm.s_free[b]));   // S buffer b may be overwritten
       // logits in log2 units, ragged tail masked
       const int n_valid = n_tot - (tile_begin + i) * kTileKeys - kHalfKeys * hi;   // keys of this lane's half that exist
       float mx = -INFINITY;
@@ -295,12 +305,6 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
         pk[j] = pack_bf16(p0, p1);
       }
       l_run += sum;
-      // P buffer b was last read by P V of tile i-2
-      if (i >= 2) {
-        ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done[b]), ((i >> 1) & 1) ^ 1, p.status));
-        if (!ok) break;
-        tc::fence_after_sync();
-      }
       {
         // The A operand of P V sits in tensor memory, in the lanes of the accumulator it feeds: both lanes of a
         // row need all 64 keys, so the two halves are swapped in, then written as 32 columns of packed bf16.
@@ -311,7 +315,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
           full[j] = hi ? other : pk[j];
           full[16 + j] = hi ? pk[j] : other;
         }
-        tc::tmem_st32(tmem_base + lane_addr + kColP + b * 32, full);
+        tc::tmem_st32(s_addr, full);   // over the first 32 columns of the S buffer this lane has just read
         tc::tmem_st_wait();
         tc::fence_before_sync();
       }
