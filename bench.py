@@ -194,6 +194,7 @@ def main():
     import torch.distributed as dist
     from paper_2608_01662_b200 import build
     from paper_2608_01662_b200.workload import make_workload
+    from paper_2608_01662_b200.distributed import job_throughput, max_over_ranks
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
@@ -254,13 +255,8 @@ def main():
         prof = wl.ctx.profile_read()
         wl.ctx.profile_enable(False)
 
-    t_ms = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
-    ms_max = float(t_ms.item())
-    ms_per_step = ms_max / args.steps
-    units = wl.units() * world
-    value = ms_per_step * 1e3 if decode else units / (ms_per_step * 1e-3)
+    ms_per_step = max_over_ranks(ms, dev) / args.steps          # the slowest rank bounds the job
+    value = ms_per_step * 1e3 if decode else job_throughput(wl.units(), world, ms_per_step)
 
     if rank != 0:
         if world > 1:
