@@ -114,18 +114,18 @@ WsLayout ws_layout(const lsa_params* p, int64_t n_query, int64_t n_key_max, int 
 
 int* status_word(lsa_ctx* c) { return c->ws ? reinterpret_cast<int*>(c->ws) : nullptr; }
 
-// Number of row splits per sequence in paged (decode) attention: fill the SMs with whole waves.
+// Number of row splits per sequence in paged (decode) attention.  Blocks run one per SM in waves; a block costs its
+// share of the 64-key units plus a fixed part (Q load, tensor-memory set-up, fp32 partial output), taken as six
+// units' worth.  The split count with the smallest estimate wins; ties go to fewer splits (less merging).
 int pick_split(int sm_count, int batch, int max_rows) {
-  const int tiles = (max_rows + 63) / 64;
+  const int units = (max_rows + 63) / 64;
   int best = 1;
-  double best_eff = 0.0;
-  for (int s = 1; s <= kMaxSplit && s <= tiles; ++s) {
-    if ((tiles + s - 1) / s < 4 && s > 1) break;  // keep at least 4 tiles per block
-    const int blocks = batch * s;
-    const int waves = (blocks + sm_count - 1) / sm_count;
-    const double eff = static_cast<double>(blocks) / (static_cast<double>(waves) * sm_count);
-    if (eff > best_eff + 1e-9) {
-      best_eff = eff;
+  long best_cost = -1;
+  for (int s = 1; s <= kMaxSplit && s <= units; ++s) {
+    const long waves = (static_cast<long>(batch) * s + sm_count - 1) / sm_count;
+    const long cost = waves * ((units + s - 1) / s + 6);
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost;
       best = s;
     }
   }

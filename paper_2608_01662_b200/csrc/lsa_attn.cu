@@ -273,19 +273,34 @@ __global__ void __launch_bounds__(kAttnThreads, 1) sparse_attn_kernel(AttnArgs p
 __global__ void merge_splits_kernel(const float* __restrict__ part_out, const float* __restrict__ part_lse,
                                     int n_split, int H, int DV, __nv_bfloat16* __restrict__ out,
                                     float* __restrict__ lse) {
+  constexpr int kMaxSplit = 16;
   const int qi = blockIdx.x, h = blockIdx.y;
   const float* pl = part_lse + static_cast<int64_t>(qi) * n_split * H + h;
+  float wgt[kMaxSplit];
   float m = -INFINITY;
-  for (int s = 0; s < n_split; ++s) m = fmaxf(m, pl[s * H]);
+  for (int s = 0; s < n_split; ++s) {
+    wgt[s] = pl[s * H];
+    m = fmaxf(m, wgt[s]);
+  }
   float den = 0.f;
-  for (int s = 0; s < n_split; ++s) den += exp2f(pl[s * H] - m);
-  for (int d = threadIdx.x; d < DV; d += blockDim.x) {
-    float acc = 0.f;
+  for (int s = 0; s < n_split; ++s) {
+    wgt[s] = exp2f(wgt[s] - m);
+    den += wgt[s];
+  }
+  const float inv = den > 0.f ? 1.f / den : 0.f;
+  for (int d = threadIdx.x * 4; d < DV; d += blockDim.x * 4) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int s = 0; s < n_split; ++s) {
-      const float wgt = exp2f(pl[s * H] - m) / den;
-      if (wgt > 0.f) acc += wgt * part_out[((static_cast<int64_t>(qi) * n_split + s) * H + h) * DV + d];
+      const float w = wgt[s] * inv;
+      if (w > 0.f) {
+        const float4 v = *reinterpret_cast<const float4*>(part_out + ((static_cast<int64_t>(qi) * n_split + s) * H + h) * DV + d);
+        acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+      }
     }
-    out[(static_cast<int64_t>(qi) * H + h) * DV + d] = __float2bfloat16(acc);
+    uint2 o;
+    o.x = pack_bf16(acc.x, acc.y);
+    o.y = pack_bf16(acc.z, acc.w);
+    *reinterpret_cast<uint2*>(out + (static_cast<int64_t>(qi) * H + h) * DV + d) = o;
   }
   if (lse != nullptr && threadIdx.x == 0) lse[static_cast<int64_t>(qi) * H + h] = (m + log2f(den)) / kLog2e;
 }
