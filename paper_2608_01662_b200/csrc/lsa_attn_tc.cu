@@ -5,7 +5,7 @@
 // rows of every MMA; the attended cache rows stream through two 64-key shared tiles:
 //
 //   warps 5-8   gather: rows [sink | sparse | window] -> 128B-swizzled K-major tiles with coalesced 16-byte
-//               cp.async (two warps per tile buffer), completion through an mbarrier
+//               cp.async (all four warps on each tile), completion through an mbarrier
 //   warp 4      one thread issues every tcgen05.mma.  Back-to-back MMAs into one accumulator run far below
 //               the pipe's rate at these small shapes, so each product is cut into two independent
 //               accumulation chains that alternate instruction by instruction:
@@ -90,7 +90,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
   if (tid == 0) {
     tc::mbar_init(smem_u32(&sm.q_full), 32 * kLoadWarps);
     for (int b = 0; b < 2; ++b) {
-      tc::mbar_init(smem_u32(&sm.k_full[b]), 32 * kLoadWarps / 2);
+      tc::mbar_init(smem_u32(&sm.k_full[b]), 32 * kLoadWarps);
       tc::mbar_init(smem_u32(&sm.k_empty[b]), kMmaWarps);
       tc::mbar_init(smem_u32(&sm.s_full[b]), kMmaWarps);
     }
@@ -122,29 +122,34 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       tc::fence_proxy_async();
       tc::mbar_arrive(smem_u32(&sm.q_full));
     }
-    // Two groups of two warps, one group per tile buffer; warp `wg` of a group gathers rows 32*wg .. +31 of its
-    // tiles.  Lane l looks up the cache row of key 32*wg + l once; the row number is then broadcast and the 72
-    // 16-byte chunks of that row are copied by consecutive lanes (coalesced 512-byte requests).
-    const int grp = lt >> 6, wg = (lt >> 5) & 1;
+    // Every gather warp works on every tile: warp w copies rows 16w .. 16w+15, so a freed buffer is refilled by all
+    // four warps at once.  Lanes 0-15 look up the cache row of their key once; the row number is then broadcast
+    // and the 72 16-byte chunks of that row are copied by consecutive lanes (coalesced 512-byte requests).
+    const int lw = lt >> 5;
+    constexpr int kRowsPerWarp = kTileKeys / kLoadWarps;
     const uint8_t* kg = reinterpret_cast<const uint8_t*>(p.k);
-    int32_t my_row = grp < n_tiles ? row_of((tile_begin + grp) * kTileKeys + kHalfKeys * wg + lane) : -1;
-    for (int i = grp; i < n_tiles; i += 2) {
-      // row numbers of this warp's next half-tile are fetched before the wait, off the critical path
-      const int32_t next_row = i + 2 < n_tiles ? row_of((tile_begin + i + 2) * kTileKeys + kHalfKeys * wg + lane) : -1;
-      if (!__all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.k_empty[grp]), ((i >> 1) & 1) ^ 1, p.status))) break;
+    auto my_key_row = [&](int i) -> int32_t {
+      return (i < n_tiles && lane < kRowsPerWarp) ? row_of((tile_begin + i) * kTileKeys + kRowsPerWarp * lw + lane) : -1;
+    };
+    int32_t my_row = my_key_row(0);
+    for (int i = 0; i < n_tiles; ++i) {
+      const int b = i & 1;
+      const int32_t next_row = my_key_row(i + 1);   // fetched before the wait: off the critical path
+      if (!__all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.k_empty[b]), ((i >> 1) & 1) ^ 1, p.status))) break;
 #pragma unroll 4
-      for (int rr = 0; rr < kHalfKeys; ++rr) {
+      for (int rr = 0; rr < kRowsPerWarp; ++rr) {
         const int32_t row = __shfl_sync(0xffffffffu, my_row, rr);
+        const int r = kRowsPerWarp * lw + rr;
         const uint8_t* src = kg + static_cast<int64_t>(row >= 0 ? row : 0) * p.ld_k * 2;
         const int nb = row >= 0 ? 16 : 0;
 #pragma unroll
         for (int c = lane; c < 72; c += 32)
-          cp_async16(smem_u32(sm.k[grp][c >> 3]) + (kHalfKeys * wg + rr) * 128 + (((c & 7) ^ (rr & 7)) << 4), src + c * 16, nb);
+          cp_async16(smem_u32(sm.k[b][c >> 3]) + r * 128 + (((c & 7) ^ (r & 7)) << 4), src + c * 16, nb);
       }
       cp_async_commit();
       cp_async_wait<0>();
       tc::fence_proxy_async();
-      tc::mbar_arrive(smem_u32(&sm.k_full[grp]));
+      tc::mbar_arrive(smem_u32(&sm.k_full[b]));
       my_row = next_row;
     }
   } else if (warp >= kSoftmaxWarps) {
