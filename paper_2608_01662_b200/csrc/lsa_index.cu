@@ -249,6 +249,7 @@ struct FineSmem {
   alignas(128) uint8_t q[HI * DI * 2];
   float w[HI];
   uint32_t keys[kMaxSlots];
+  float scale[2][kTileRows];   // per-token key scales of the tile in flight (e4m3 keys)
   int32_t pages[kMaxPages];
   SelectScratch sel;
 };
@@ -283,8 +284,16 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
   int nP;
   if (p.hi_enable && nE > p.M) {
     const float* ps = p.page_scores + static_cast<int64_t>(qi) * p.ps_ld + p0;
-    nP = block_select_topk([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M,
-                           sm.pages, sm.sel);
+    if (nE <= kMaxSlots) {
+      // one pass over the page scores (L2) into the candidate buffer, which is idle until the fine stage;
+      // the six passes of the radix select then run out of shared memory
+      for (int i = tid; i < nE; i += kThreads) sm.keys[i] = score_key(ps[i]);
+      __syncthreads();
+      nP = block_select_topk([&](int i) { return sm.keys[i]; }, [&](int i) { return p0 + i; }, nE, p.M, sm.pages, sm.sel);
+    } else {
+      nP = block_select_topk([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M,
+                             sm.pages, sm.sel);
+    }
   } else {
     nP = nE;  // host guarantees nE <= kMaxSlots / P here
     for (int i = tid; i < nP; i += kThreads) sm.pages[i] = p0 + i;
@@ -311,8 +320,17 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
   constexpr int CU = DI / 16;                         // 16-byte code units per row (e4m3)
   constexpr int kCodePerThread = kTileRows * CU / kThreads;
   uint4 staged[E4M3 ? kCodePerThread : 1];
+  float staged_scale = 0.f;
   auto issue_tile = [&](int tile, int buf) {
     if constexpr (E4M3) {
+      if (tid < kTileRows) {   // this row's scale travels with the tile instead of being fetched after the MMAs
+        const int c = tile * kTileRows + tid;
+        staged_scale = 0.f;
+        if (c < n_slots) {
+          const int64_t pos = slot_pos(c);
+          if (pos < n_key) staged_scale = p.k_scale[phys_row(pos)];
+        }
+      }
 #pragma unroll
       for (int j = 0; j < kCodePerThread; ++j) {
         const int e = tid + j * kThreads, r = e / CU, u = e % CU;
@@ -342,6 +360,7 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
   };
   auto land_tile = [&](int buf) {
     if constexpr (E4M3) {
+      if (tid < kTileRows) sm.scale[buf][tid] = staged_scale;
 #pragma unroll
       for (int j = 0; j < kCodePerThread; ++j) {
         const int e = tid + j * kThreads, r = e / CU, u = e % CU;
@@ -373,7 +392,7 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
           uint32_t key = 0;
           if (pos >= lo && pos <= hi) {
             float s = half ? s_hi : s_lo;
-            if constexpr (E4M3) s *= p.k_scale[phys_row(pos)];
+            if constexpr (E4M3) s *= sm.scale[buf][16 * warp + (lane >> 2) + 8 * half];
             key = score_key(s);
           }
           sm.keys[c] = key;
