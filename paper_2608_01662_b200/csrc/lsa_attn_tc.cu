@@ -39,15 +39,17 @@ constexpr int kHalfKeys = 32;
 constexpr int kSoftmaxWarps = 4, kMmaWarps = 4, kLoadWarps = 4;
 constexpr int kThreadsAttnTc = 32 * (kSoftmaxWarps + kMmaWarps + kLoadWarps);
 constexpr uint32_t kTmemColsAttn = 512;
-constexpr uint32_t kColS = 256;              // two S buffers of 128 columns: two column sets of 64 partial sums
-constexpr uint32_t kSBuf = 128;
+constexpr int kKBufs = 3;                    // 64-key tile buffers in shared memory
+constexpr uint32_t kColQ = 256;              // Q[:, 0:512] as packed bf16: 128 columns, dims 0-255 | 256-511 by lane half
+constexpr uint32_t kColS = 384;              // two S / P buffers of 64 columns
+constexpr uint32_t kSBuf = 64;
 constexpr float kLog2eTc = 1.4426950408889634f;
 constexpr float kRescaleGap = 8.f;           // rescale O only when the row max grows by more than 2^8
 
 struct AttnTcSmem {
-  alignas(1024) uint8_t q[kAtoms][kAtomBytes];
-  alignas(1024) uint8_t k[2][kAtoms][kAtomBytes];   // [tile buffer][column block][64 rows x 128 B]
-  alignas(8) uint64_t q_full, k_full[2], k_empty[2], s_full[2], p_ready, pv_done[2];
+  alignas(1024) uint8_t q_rope[kAtomBytes];                 // Q[:, 512:576], 64 rows x 128 B
+  alignas(1024) uint8_t k[kKBufs][kAtoms][kAtomBytes];      // [tile buffer][column block][64 rows x 128 B]
+  alignas(8) uint64_t q_full, q_tmem, k_full[kKBufs], k_empty[kKBufs], s_full[2], p_ready[2], pv_done[2];
   uint32_t tmem_slot;
 };
 
@@ -89,13 +91,16 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
   // ---- set-up
   if (tid == 0) {
     tc::mbar_init(smem_u32(&sm.q_full), 32 * kLoadWarps);
-    for (int b = 0; b < 2; ++b) {
+    tc::mbar_init(smem_u32(&sm.q_tmem), kSoftmaxWarps);
+    for (int b = 0; b < kKBufs; ++b) {
       tc::mbar_init(smem_u32(&sm.k_full[b]), 32 * kLoadWarps);
       tc::mbar_init(smem_u32(&sm.k_empty[b]), kMmaWarps);
-      tc::mbar_init(smem_u32(&sm.s_full[b]), kMmaWarps);
     }
-    tc::mbar_init(smem_u32(&sm.p_ready), kSoftmaxWarps);
-    for (int b = 0; b < 2; ++b) tc::mbar_init(smem_u32(&sm.pv_done[b]), kMmaWarps);
+    for (int b = 0; b < 2; ++b) {
+      tc::mbar_init(smem_u32(&sm.s_full[b]), 2);
+      tc::mbar_init(smem_u32(&sm.pv_done[b]), kMmaWarps);
+      tc::mbar_init(smem_u32(&sm.p_ready[b]), kSoftmaxWarps);
+    }
     tc::fence_mbar_init();
   }
   if (warp == kSoftmaxWarps) {
@@ -111,11 +116,11 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     // ================= gather warps =================
     const int lt = tid - 32 * (kSoftmaxWarps + kMmaWarps);   // 0..127
     {
-      // Q: 64 rows of 1152 contiguous bytes
-      const uint8_t* qg = reinterpret_cast<const uint8_t*>(p.q) + static_cast<int64_t>(qi) * kH * kDQK * 2;
-      for (int e = lt; e < kH * 72; e += 32 * kLoadWarps) {
-        const int r = e / 72, c = e % 72;
-        cp_async16(smem_u32(sm.q[c >> 3]) + r * 128 + (((c & 7) ^ (r & 7)) << 4), qg + e * 16, 16);
+      // the rope part of Q (dims 512-575) stays in shared memory: 64 rows x 128 bytes
+      const uint8_t* qg = reinterpret_cast<const uint8_t*>(p.q) + static_cast<int64_t>(qi) * kH * kDQK * 2 + 512 * 2;
+      for (int e = lt; e < kH * 8; e += 32 * kLoadWarps) {
+        const int r = e >> 3, c = e & 7;
+        cp_async16(smem_u32(sm.q_rope) + r * 128 + ((c ^ (r & 7)) << 4), qg + r * kDQK * 2 + c * 16, 16);
       }
       cp_async_commit();
       cp_async_wait<0>();
@@ -133,9 +138,9 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     };
     int32_t my_row = my_key_row(0);
     for (int i = 0; i < n_tiles; ++i) {
-      const int b = i & 1;
+      const int b = i % kKBufs;
       const int32_t next_row = my_key_row(i + 1);   // fetched before the wait: off the critical path
-      if (!__all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.k_empty[b]), ((i >> 1) & 1) ^ 1, p.status))) break;
+      if (!__all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.k_empty[b]), ((i / kKBufs) & 1) ^ 1, p.status))) break;
 #pragma unroll 4
       for (int rr = 0; rr < kRowsPerWarp; ++rr) {
         const int32_t row = __shfl_sync(0xffffffffu, my_row, rr);
@@ -154,63 +159,62 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     }
   } else if (warp >= kSoftmaxWarps) {
     // ================= MMA issuers =================
-    const int x = warp - kSoftmaxWarps;   // 0..3: accumulation chain of this issuer
+    const int x = warp - kSoftmaxWarps;   // 0..3
     if (lane == 0 && n_tiles > 0) {
       constexpr uint32_t idesc_qk = tc::idesc_bf16(kH, kTileKeys, 0, 0);
       constexpr uint32_t idesc_pv = tc::idesc_bf16(kH, 128, 0, 1);   // B = V read MN-major
-      bool ok = tc::mbar_wait(smem_u32(&sm.q_full), 0, p.status);
+      bool ok = tc::mbar_wait(smem_u32(&sm.q_full), 0, p.status) && tc::mbar_wait(smem_u32(&sm.q_tmem), 0, p.status);
       // Descriptors are built once; inside the loops only the start-address word moves (one add per operand).
       constexpr uint32_t kBufBytes = kAtoms * kAtomBytes;
-      constexpr int kChain = kAtoms * 4 / kMmaWarps;   // 9 of the 36 K-steps of 16 dims per accumulation chain
-      const uint64_t dq0 = tc::smem_desc_sw128(smem_u32(sm.q), 16, 1024);
+      const uint64_t dqr = tc::smem_desc_sw128(smem_u32(sm.q_rope), 16, 1024);
       const uint64_t dk0 = tc::smem_desc_sw128(smem_u32(sm.k), 16, 1024);           // K-major view (Q K^T)
       const uint64_t dv0 = tc::desc_advance(tc::smem_desc_sw128(smem_u32(sm.k), kAtomBytes, 1024), 2 * x * kAtomBytes);  // MN-major view (P V)
       constexpr uint32_t kLane16 = 16u << 16;
-      // Q K^T: partial sum x goes to lane half x&1, column set x>>1 of the S buffer
-      const uint32_t s_dst = tmem_base + (x & 1) * kLane16 + kColS + (x >> 1) * kTileKeys;
-      // P V: value dims 128x .. 128x+127 = columns 128*(x&1) .. of the accumulator in lane half x>>1; P is read
-      // from the same lane half
+      // Q K^T (issuers 0 and 1): chain x = dims 256x .. 256x+255 with Q from tensor memory (lane half x), plus two of
+      // the four rope steps with Q from shared memory; its partial sum goes to lane half x of the S buffer
+      const uint32_t q_src = tmem_base + (x & 1) * kLane16 + kColQ;
+      const uint32_t s_dst = tmem_base + (x & 1) * kLane16 + kColS;
+      // P V (all four issuers): value dims 128x .. 128x+127 = columns 128*(x&1) .. of the accumulator in lane half
+      // x>>1; P is read from the same lane half
       const uint32_t o_dst = tmem_base + (x >> 1) * kLane16 + (x & 1) * 128;
       const uint32_t p_src = tmem_base + (x >> 1) * kLane16 + kColS;
-      auto issue_qk = [&](int i) {   // partial S_i over this issuer's K-steps
-        const int b = i & 1;
+      auto issue_qk = [&](int i) {
         tc::fence_after_sync();
-        const uint32_t d = s_dst + b * kSBuf;
-        const uint64_t dkb = tc::desc_advance(dk0, b * kBufBytes);
+        const uint32_t d = s_dst + (i & 1) * kSBuf;
+        const uint64_t dkb = tc::desc_advance(dk0, (i % kKBufs) * kBufBytes);
 #pragma unroll
-        for (int s = 0; s < kChain; ++s) {
-          const int ks = x * kChain + s;                    // K-step: column block ks/4, 32-byte slice ks%4
-          const uint32_t off = (ks >> 2) * kAtomBytes + (ks & 3) * 32;
-          tc::umma_ss(d, tc::desc_advance(dq0, off), tc::desc_advance(dkb, off), idesc_qk, s != 0);
-        }
-        tc::umma_commit(smem_u32(&sm.s_full[b]));
+        for (int s = 0; s < 16; ++s)   // dims 256x + 16s .. +15: column block 4x + s/4, 32-byte slice s%4
+          tc::umma_ts(d, q_src + 8 * s, tc::desc_advance(dkb, (4 * x + (s >> 2)) * kAtomBytes + (s & 3) * 32), idesc_qk, s != 0);
+#pragma unroll
+        for (int s = 0; s < 2; ++s)    // rope dims 512 + 32x + 16s .. +15
+          tc::umma_ss(d, tc::desc_advance(dqr, (2 * x + s) * 32), tc::desc_advance(dkb, 8 * kAtomBytes + (2 * x + s) * 32), idesc_qk, 1);
+        tc::umma_commit(smem_u32(&sm.s_full[i & 1]));
       };
       auto issue_pv = [&](int j) {   // O[:, 128x : 128x+128] += P_j V_j
-        const int b = j & 1;
         tc::fence_after_sync();
-        const uint64_t dvb = tc::desc_advance(dv0, b * kBufBytes);
+        const uint64_t dvb = tc::desc_advance(dv0, (j % kKBufs) * kBufBytes);
 #pragma unroll
         for (int kk = 0; kk < kTileKeys / 16; ++kk)   // keys 16*kk .. +15
-          tc::umma_ts(o_dst, p_src + b * kSBuf + kk * 8, tc::desc_advance(dvb, kk * 2048), idesc_pv, (j > 0) || (kk > 0));
-        tc::umma_commit(smem_u32(&sm.k_empty[b]));
-        tc::umma_commit(smem_u32(&sm.pv_done[b]));
+          tc::umma_ts(o_dst, p_src + (j & 1) * kSBuf + kk * 8, tc::desc_advance(dvb, kk * 2048), idesc_pv, (j > 0) || (kk > 0));
+        tc::umma_commit(smem_u32(&sm.k_empty[j % kKBufs]));
+        tc::umma_commit(smem_u32(&sm.pv_done[j & 1]));
       };
+      const bool does_qk = x < 2;
       // Two in-order queues, "next Q K^T" (at most one tile ahead of the softmax it feeds) and "next P V".
-      int qk_next = 0, pv_next = 0;
+      int qk_next = does_qk ? 0 : n_tiles, pv_next = 0;
       long long t_idle = clock64();
       uint32_t spins = 0;
       while (ok && pv_next < n_tiles) {
         bool did = false;
         if (qk_next < n_tiles && qk_next <= pv_next + 1) {
-          const int b = qk_next & 1;
-          // S buffer b also holds P of tile qk_next-2: it is free once that tile's P V has completed
-          if (tc::mbar_test(smem_u32(&sm.k_full[b]), (qk_next >> 1) & 1) &&
-              tc::mbar_test(smem_u32(&sm.pv_done[b]), ((qk_next >> 1) & 1) ^ 1)) {
+          // S buffer qk_next&1 also holds P of tile qk_next-2: it is free once that tile's P V has completed
+          if (tc::mbar_test(smem_u32(&sm.k_full[qk_next % kKBufs]), (qk_next / kKBufs) & 1) &&
+              tc::mbar_test(smem_u32(&sm.pv_done[qk_next & 1]), ((qk_next >> 1) & 1) ^ 1)) {
             issue_qk(qk_next++);
             did = true;
           }
         }
-        if (!did && pv_next < qk_next && tc::mbar_test(smem_u32(&sm.p_ready), pv_next & 1)) {
+        if (!did && (!does_qk || pv_next < qk_next) && tc::mbar_test(smem_u32(&sm.p_ready[pv_next & 1]), (pv_next >> 1) & 1)) {
           issue_pv(pv_next++);
           did = true;
         }
@@ -232,10 +236,30 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     const int quarter = warp;                 // TMEM lanes 32*warp .. +31
     const int r16 = lane & 15, hi = lane >> 4;
     const int row = 16 * quarter + r16;       // head; lanes l and l+16 share it: keys 0-31 / 32-63, O dims 0-255 / 256-511
+    const uint32_t lane_addr = static_cast<uint32_t>(32 * quarter) << 16;
+    {
+      // Q[row, 256*hi : 256*hi+256] -> 128 columns of this lane, in the order the tensor core reads an A operand
+      // (two consecutive dims per 32-bit column)
+      const uint4* qg = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(p.q) +
+                                                       ((static_cast<int64_t>(qi) * kH + row) * kDQK + 256 * hi) * 2);
+#pragma unroll 1
+      for (int part = 0; part < 2; ++part) {
+        uint32_t w[64];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const uint4 u = qg[part * 16 + j];
+          w[4 * j] = u.x; w[4 * j + 1] = u.y; w[4 * j + 2] = u.z; w[4 * j + 3] = u.w;
+        }
+        tc::tmem_st64(tmem_base + lane_addr + kColQ + part * 64, w);
+        tc::tmem_st_wait();
+      }
+      tc::fence_before_sync();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(smem_u32(&sm.q_tmem));
+    }
     const float zs = p.sm_scale * kLog2eTc;
     float m_used = -INFINITY, l_run = 0.f;    // m_used is kept identical in both lanes of a row; l_run is a partial sum
     bool ok = true;
-    const uint32_t lane_addr = static_cast<uint32_t>(32 * quarter) << 16;
     for (int i = 0; i < n_tiles && ok; ++i) {
       const int b = i & 1;
       ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.s_full[b]), (i >> 1) & 1, p.status));
@@ -244,18 +268,11 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       const uint32_t s_addr = tmem_base + lane_addr + kColS + b * kSBuf;
       uint32_t v[32];
       {
-        // This lane holds two chains' partial sums for all 64 keys (column sets 0 and 1); its partner lane (l ^ 16)
-        // the other two.  Lane l keeps keys 0-31, lane l+16 keys 32-63: add the own pair, send the half the
-        // partner finishes, add the one it sends.
+        // This lane holds one chain's partial sums for all 64 keys, its partner lane (l ^ 16) the other's.  Lane l
+        // keeps keys 0-31, lane l+16 keys 32-63: send the half the partner finishes, add the one it sends.
         uint32_t s64[64];
-        {
-          uint32_t t64[64];
-          tc::tmem_ld64(s_addr, s64);
-          tc::tmem_ld64(s_addr + kTileKeys, t64);
-          tc::tmem_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 64; ++j) s64[j] = __float_as_uint(__uint_as_float(s64[j]) + __uint_as_float(t64[j]));
-        }
+        tc::tmem_ld64(s_addr, s64);
+        tc::tmem_ld_wait();
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           const float give = __uint_as_float(hi ? s64[j] : s64[32 + j]);
@@ -325,7 +342,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
         tc::fence_before_sync();
       }
       __syncwarp();
-      if (lane == 0) tc::mbar_arrive(smem_u32(&sm.p_ready));
+      if (lane == 0) tc::mbar_arrive(smem_u32(&sm.p_ready[b]));
     }
     // ---- epilogue: O / l
     const float l_row = l_run + __shfl_xor_sync(0xffffffffu, l_run, 16);
