@@ -84,7 +84,7 @@ int check_params(const lsa_params* p, bool need_index, bool need_attn) {
 
 // Workspace map.  All offsets are multiples of 256 bytes.
 struct WsLayout {
-  size_t page_scores, rows, n_rows, part_out, part_lse, total;
+  size_t page_scores, rows, n_rows, part_out, part_lse, fine_keys, fine_pages, total;
   int ps_ld, rows_ld;
 };
 
@@ -103,6 +103,10 @@ WsLayout ws_layout(const lsa_params* p, int64_t n_query, int64_t n_key_max, int 
     off += align_up(static_cast<size_t>(batch) * kMaxSplit * p->n_heads * p->d_v * sizeof(float), 256);
     l.part_lse = off;
     off += align_up(static_cast<size_t>(batch) * kMaxSplit * p->n_heads * sizeof(float), 256);
+    l.fine_keys = off;
+    off += align_up(static_cast<size_t>(batch) * 4096 * sizeof(uint32_t), 256);
+    l.fine_pages = off;
+    off += align_up(static_cast<size_t>(batch) * 65 * sizeof(int32_t), 256);
   }
   const int P = p->page > 0 ? p->page : 64;
   l.ps_ld = static_cast<int>(align_up(static_cast<size_t>((n_key_max + P - 1) / P), 4));
@@ -159,6 +163,17 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
     a.sparse_idx = sparse_idx + q0 * p->k_sparse; a.n_sparse = n_sparse + q0;
     a.pages_out = pages_out ? pages_out + q0 * p->keep_pages : nullptr;
     a.status = status_word(c);
+    a.fine_parts = 1;
+    if (p->paged) {
+      // few queries and many SMs: several blocks score each query's candidates, a second kernel selects
+      int parts = 2 * c->sm_count / (batch > 0 ? batch : 1);   // two scoring blocks fit one SM
+      parts = parts > 4 ? 4 : parts;
+      if (parts > 1) {
+        a.fine_parts = parts;
+        a.fine_keys = reinterpret_cast<uint32_t*>(c->ws + l.fine_keys);
+        a.fine_pages = reinterpret_cast<int32_t*>(c->ws + l.fine_pages);
+      }
+    }
     cudaError_t e = cudaSuccess;
     if (p->hi_enable)
       e = timed(c, LSA_K_COARSE, [&] {

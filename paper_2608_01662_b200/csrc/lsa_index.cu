@@ -273,7 +273,10 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
   int32_t* out_idx = p.sparse_idx + static_cast<int64_t>(qi) * p.Ksp;
   int32_t* out_pages = p.pages_out ? p.pages_out + static_cast<int64_t>(qi) * p.M : nullptr;
   const int64_t lo = p.S, hi = t - p.W;
+  const int part = blockIdx.y, n_parts = gridDim.y;   // > 1: this block scores a share of the tiles only
   if (hi < lo) {
+    if (part != 0) return;
+    if (n_parts > 1) p.fine_pages[qi * (kMaxPages + 1) + kMaxPages] = 0;
     for (int i = tid; i < p.Ksp; i += kThreads) out_idx[i] = -1;
     if (out_pages) for (int i = tid; i < p.M; i += kThreads) out_pages[i] = -1;
     if (tid == 0) p.n_sparse[qi] = 0;
@@ -303,10 +306,18 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
   if (tid < HI / 4) cp_async16(smem_u32(&sm.w[tid * 4]), p.w + static_cast<int64_t>(qi) * HI + tid * 4, 16);
   cp_async_commit();
   __syncthreads();  // sm.pages visible
-  if (out_pages) for (int i = tid; i < p.M; i += kThreads) out_pages[i] = i < nP ? sm.pages[i] : -1;
+  if (out_pages && part == 0) for (int i = tid; i < p.M; i += kThreads) out_pages[i] = i < nP ? sm.pages[i] : -1;
+  if (n_parts > 1 && part == 0) {
+    int32_t* fp = p.fine_pages + qi * (kMaxPages + 1);
+    for (int i = tid; i < nP; i += kThreads) fp[i] = sm.pages[i];
+    if (tid == 0) fp[kMaxPages] = nP;
+  }
 
   const int n_slots = nP * p.P;
-  const int n_tiles = (n_slots + kTileRows - 1) / kTileRows;
+  const int n_tiles_all = (n_slots + kTileRows - 1) / kTileRows;
+  const int tiles_per = (n_tiles_all + n_parts - 1) / n_parts;
+  const int tile0 = part * tiles_per;
+  const int n_tiles = max(0, min(n_tiles_all, tile0 + tiles_per) - tile0);
   const int pshift = 31 - __clz(p.P);
   auto slot_pos = [&](int c) -> int64_t { return static_cast<int64_t>(sm.pages[c >> pshift]) * p.P + (c & (p.P - 1)); };
   auto phys_row = [&](int64_t pos) -> int64_t {
@@ -372,13 +383,13 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
     }
   };
 
-  issue_tile(0, 0);
-  for (int tile = 0; tile < n_tiles; ++tile) {
-    const int buf = tile & 1;
+  if (n_tiles > 0) issue_tile(tile0, 0);
+  for (int tile = tile0; tile < tile0 + n_tiles; ++tile) {
+    const int buf = (tile - tile0) & 1;
     land_tile(buf);
     cp_async_wait<0>();
     __syncthreads();  // tile `tile` (and, first time, q/w) in shared; buffer buf^1 free
-    if (tile + 1 < n_tiles) issue_tile(tile + 1, buf ^ 1);
+    if (tile + 1 < tile0 + n_tiles) issue_tile(tile + 1, buf ^ 1);
     uint32_t a[DI / 16][4];
     load_a_frags<DI>(a, smem_u32(sm.a[buf]));
     float s_lo, s_hi;
@@ -401,9 +412,37 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
     }
   }
   __syncthreads();
+  if (n_parts > 1) {
+    // hand this block's share of the candidate keys to the top-K kernel
+    uint32_t* fk = p.fine_keys + static_cast<int64_t>(qi) * kMaxSlots;
+    const int c0 = tile0 * kTileRows, c1 = min(n_slots, (tile0 + n_tiles) * kTileRows);
+    for (int c = c0 + tid; c < c1; c += kThreads) fk[c] = sm.keys[c];
+    return;
+  }
   const int n_sel = block_select_topk([&](int i) { return sm.keys[i]; },
                                       [&](int i) { return static_cast<int>(slot_pos(i)); }, n_slots, p.Ksp, out_idx,
                                       sm.sel);
+  if (tid == 0) p.n_sparse[qi] = n_sel;
+}
+
+// Second half of the split fine stage: top-K_sparse over the keys the scoring blocks left in global memory.
+__global__ void __launch_bounds__(kSelThreads) fine_topk_kernel(IndexArgs p) {
+  __shared__ uint32_t keys[kMaxSlots];
+  __shared__ int32_t pages[kMaxPages];
+  __shared__ SelectScratch sc;
+  const int qi = blockIdx.x, tid = threadIdx.x;
+  const int32_t* fp = p.fine_pages + qi * (kMaxPages + 1);
+  const int nP = fp[kMaxPages];
+  if (nP == 0) return;   // no candidates: the scoring kernel has written the empty result
+  const int n_slots = nP * p.P;
+  const uint32_t* fk = p.fine_keys + static_cast<int64_t>(qi) * kMaxSlots;
+  for (int i = tid; i < n_slots; i += kSelThreads) keys[i] = fk[i];
+  for (int i = tid; i < nP; i += kSelThreads) pages[i] = fp[i];
+  __syncthreads();
+  const int pshift = 31 - __clz(p.P);
+  const int n_sel = block_select_topk([&](int i) { return keys[i]; },
+                                      [&](int i) { return pages[i >> pshift] * p.P + (i & (p.P - 1)); }, n_slots, p.Ksp,
+                                      p.sparse_idx + static_cast<int64_t>(qi) * p.Ksp, sc);
   if (tid == 0) p.n_sparse[qi] = n_sel;
 }
 
@@ -535,7 +574,12 @@ static cudaError_t launch_fine_t(const IndexArgs& a, cudaStream_t st, int64_t* n
   const size_t smem = sizeof(FineSmem<HI, DI>);
   cudaError_t e = set_smem(fine_select_kernel<HI, DI, E4M3>, smem);
   if (e != cudaSuccess) return e;
-  fine_select_kernel<HI, DI, E4M3><<<a.n_query, kThreads, smem, st>>>(a);
+  const int parts = a.fine_parts > 1 ? a.fine_parts : 1;
+  fine_select_kernel<HI, DI, E4M3><<<dim3(a.n_query, parts), kThreads, smem, st>>>(a);
+  ++*n_launch;
+  e = cudaGetLastError();
+  if (e != cudaSuccess || parts == 1) return e;
+  fine_topk_kernel<<<a.n_query, kSelThreads, 0, st>>>(a);
   ++*n_launch;
   return cudaGetLastError();
 }

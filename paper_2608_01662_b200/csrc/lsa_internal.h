@@ -24,6 +24,10 @@ struct IndexArgs {
   int32_t* sparse_idx;    // [n_query, Ksp]
   int32_t* n_sparse;
   int32_t* pages_out;     // optional [n_query, M]
+  // split fine stage (few queries, many SMs): the scoring blocks leave their results here for the top-K kernel
+  int fine_parts;         // 1: fused kernel; >1: blocks per query in the scoring kernel
+  uint32_t* fine_keys;    // [n_query, 4096] order-preserving keys of the candidate slots (0 = not a candidate)
+  int32_t* fine_pages;    // [n_query, 65]: kept pages, then their count
   int* status;
 };
 
