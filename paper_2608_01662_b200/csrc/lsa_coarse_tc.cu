@@ -61,6 +61,7 @@ coarse_score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
   if (tc::status_raised(p.status)) return;   // an earlier block of this launch gave up on a wait
   const int64_t hi_max = t_max - p.W;
   const int spp = p.P / p.B;
+  const int spp_shift = 31 - __clz(spp);
   const int n_tiles = static_cast<int>(hi_max / (static_cast<int64_t>(kTileM) * p.B)) + 1;
   const int n_units = n_tiles * NG;
 
@@ -149,8 +150,7 @@ coarse_score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
       ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.acc_full[set]), (u >> 1) & 1, p.status));
       if (!ok) break;
       tc::fence_after_sync();
-      const int64_t sub = static_cast<int64_t>(k) * kTileM + row;
-      const int64_t page = sub / spp;
+      const int64_t page = (static_cast<int64_t>(k) * kTileM + row) >> spp_shift;   // spp is a power of two
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + set * 256 + half * 2 * kHI;
       const int ql0 = g * kGroupQ + half * 2;
       float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;

@@ -237,6 +237,90 @@ __global__ void __launch_bounds__(kThreads) coarse_score_kernel(IndexArgs p) {
   }
 }
 
+// Paged (decode) form of a1: one query per sequence, so a block keeps the query resident and streams several
+// mean-key tiles of that sequence through a double buffer (the mean cache is the large operand here: the stage
+// is an HBM read of the whole cache of means).
+constexpr int kCoarseTilesPerBlock = 8;
+
+template <int HI, int DI>
+struct CoarsePagedSmem {
+  alignas(128) uint8_t a[2][kTileRows * DI * 2];
+  alignas(128) uint8_t q[HI * DI * 2];
+  float w[HI];
+  float sub[kTileRows];
+};
+
+template <int HI, int DI>
+__global__ void __launch_bounds__(kThreads) coarse_score_paged_kernel(IndexArgs p) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  auto& sm = *reinterpret_cast<CoarsePagedSmem<HI, DI>*>(smem_raw);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int qi = blockIdx.y;
+  const int64_t n_key = p.ctx_len[qi];
+  const int64_t t = n_key - 1, hi = t - p.W;
+  const int spp = p.P / p.B, ppt = kTileRows / spp;
+  // the coarse stage runs only when more than M pages are eligible
+  if (hi < p.S || hi / p.P - p.S / p.P + 1 <= p.M) return;
+  const int64_t n_sub = (n_key + p.B - 1) / p.B;
+  const int tiles_needed = static_cast<int>(hi / p.P / ppt) + 1;   // tiles holding an eligible page
+  const int tile_begin = blockIdx.x * kCoarseTilesPerBlock;
+  const int tile_end = min(tiles_needed, tile_begin + kCoarseTilesPerBlock);
+  if (tile_begin >= tile_end) return;
+  const int32_t* pt = p.page_table + qi * p.pt_stride;
+  const uint8_t* km = reinterpret_cast<const uint8_t*>(p.kmean);
+  const int spp_shift = 31 - __clz(spp);   // spp is 8, 16 or 32
+  constexpr int U = DI / 8;
+  constexpr int kPer = kTileRows * U / kThreads;   // 16-byte chunks per thread and tile
+  auto issue_tile = [&](int tile, int buf) {
+    // page-table look-ups first, all in flight together; then the copies that depend on them
+    int64_t src_row[kPer];
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) {
+      const int r = (tid + j * kThreads) / U;
+      const int sub = tile * kTileRows + r;   // sub-block number (fits 32 bits: cache lengths do)
+      src_row[j] = sub < n_sub ? (static_cast<int64_t>(pt[sub >> spp_shift]) << spp_shift) + (sub & (spp - 1)) : -1;
+    }
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) {
+      const int e = tid + j * kThreads, r = e / U, u = e % U;
+      const bool ok = src_row[j] >= 0;
+      cp_async16(smem_u32(sm.a[buf]) + swz<DI * 2>(r, u), km + (ok ? src_row[j] : 0) * DI * 2 + u * 16, ok ? 16 : 0);
+    }
+    cp_async_commit();
+  };
+  load_q_async<HI, DI>(smem_u32(sm.q), reinterpret_cast<const __nv_bfloat16*>(p.q_idx) + static_cast<int64_t>(qi) * HI * DI);
+  if (tid < HI / 4) cp_async16(smem_u32(&sm.w[tid * 4]), p.w + static_cast<int64_t>(qi) * HI + tid * 4, 16);
+  issue_tile(tile_begin, 0);
+  for (int tile = tile_begin; tile < tile_end; ++tile) {
+    const int buf = (tile - tile_begin) & 1;
+    if (tile + 1 < tile_end) {
+      issue_tile(tile + 1, buf ^ 1);
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
+    }
+    __syncthreads();   // tile (and, first time, q / w) in shared
+    uint32_t a[DI / 16][4];
+    load_a_frags<DI>(a, smem_u32(sm.a[buf]));
+    float s_lo, s_hi;
+    score_16rows<HI, DI>(a, smem_u32(sm.q), sm.w, s_lo, s_hi);
+    if ((lane & 3) == 0) {
+      sm.sub[16 * warp + (lane >> 2)] = s_lo;
+      sm.sub[16 * warp + (lane >> 2) + 8] = s_hi;
+    }
+    __syncthreads();
+    if (tid < ppt) {
+      const int64_t page = static_cast<int64_t>(tile) * ppt + tid;
+      if (page * p.P <= hi) {
+        float s = 0.f;
+        for (int j = 0; j < spp; ++j) s += sm.sub[tid * spp + j];
+        p.page_scores[static_cast<int64_t>(qi) * p.ps_ld + page] = s;
+      }
+    }
+    __syncthreads();   // sub and buffer `buf` are reused two tiles on
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // a2-a4: per query: top-M pages, fine scores on their tokens, top-K_sparse.
 // ------------------------------------------------------------------------------------------------
@@ -488,13 +572,14 @@ __global__ void __launch_bounds__(128) convert_kernel(int S, int W, int Ksp, int
   const int n_sp = n_sparse[qi];
   const int n_tot = n_sink + n_sp + n_win;
   const int ld = S + Ksp + W;
+  const int kv_shift = paged ? 31 - __clz(kv_page) : 0;   // kv_page is a power of two
   int32_t* out = rows_out + static_cast<int64_t>(qi) * ld;
   auto row_of = [&](int i) -> int32_t {
     int64_t pos;
     if (i < n_sink) pos = i;
     else if (i < n_sink + n_sp) pos = sparse_idx[static_cast<int64_t>(qi) * Ksp + i - n_sink];
     else pos = win0 + (i - n_sink - n_sp);
-    return static_cast<int32_t>(paged ? static_cast<int64_t>(pt[pos / kv_page]) * kv_page + pos % kv_page : pos);
+    return static_cast<int32_t>(paged ? (static_cast<int64_t>(pt[pos >> kv_shift]) << kv_shift) + (pos & (kv_page - 1)) : pos);
   };
   int breaks = 0;
   for (int i = tid; i < ld; i += 128) {
@@ -555,8 +640,17 @@ static cudaError_t launch_coarse_t(const IndexArgs& a, int64_t n_key_max, cudaSt
   cudaError_t e = set_smem(coarse_score_kernel<HI, DI>, smem);
   if (e != cudaSuccess) return e;
   const int64_t n_sub = (n_key_max + a.B - 1) / a.B;
-  dim3 grid(static_cast<unsigned>((n_sub + kTileRows - 1) / kTileRows),
-            a.paged ? a.n_query : (a.n_query + kCoarseQG - 1) / kCoarseQG);
+  const unsigned n_tiles = static_cast<unsigned>((n_sub + kTileRows - 1) / kTileRows);
+  if (a.paged) {
+    const size_t psmem = sizeof(CoarsePagedSmem<HI, DI>);
+    e = set_smem(coarse_score_paged_kernel<HI, DI>, psmem);
+    if (e != cudaSuccess) return e;
+    dim3 pgrid((n_tiles + kCoarseTilesPerBlock - 1) / kCoarseTilesPerBlock, a.n_query);
+    coarse_score_paged_kernel<HI, DI><<<pgrid, kThreads, psmem, st>>>(a);
+    ++*n_launch;
+    return cudaGetLastError();
+  }
+  dim3 grid(n_tiles, (a.n_query + kCoarseQG - 1) / kCoarseQG);
   coarse_score_kernel<HI, DI><<<grid, kThreads, smem, st>>>(a);
   ++*n_launch;
   return cudaGetLastError();
