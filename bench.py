@@ -36,6 +36,7 @@ def parse_args():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-queries", type=int, default=24)
+    ap.add_argument("--no-decode", action="store_true", help="skip the cfg4 decode side measurement of the default run")
     ap.add_argument("--phase", default="group", choices=["group", "index"],
                     help="group: whole lsa_layer_group step; index: indexer only (no attention tensors are allocated; for profiling)")
     ap.add_argument("--attn-tc", type=int, default=-1, help="override LSA_TUNE_ATTN_TC (0 or 1)")
@@ -277,12 +278,12 @@ def main():
         dur_s = attn_ms / attn_n * 1e-3
         if decode:
             a = attn_bytes_per_launch(cfg, positions) / dur_s / 1e9
-            roofline = {"kernel": "sparse_attn_kernel", "bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"],
+            roofline = {"kernel": "sparse_attn_tc_kernel", "bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"],
                         "unit": "GB/s", "frac": a / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
                         "launch_ms": attn_ms / attn_n}
         else:
             a = attn_flops_per_launch(cfg, positions) / dur_s / 1e12
-            roofline = {"kernel": "sparse_attn_kernel", "bound": "tensor", "achieved": a,
+            roofline = {"kernel": "sparse_attn_tc_kernel" if cfg.H == 64 else "sparse_attn_kernel", "bound": "tensor", "achieved": a,
                         "peak": peaks["tensor_tflops"], "unit": "TFLOP/s", "frac": a / peaks["tensor_tflops"],
                         "traffic": None, "peak_source": peaks["source"], "launch_ms": attn_ms / attn_n}
     kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps}
@@ -302,6 +303,15 @@ def main():
                          f"{cfg.R} attention layers each, {secs:.1f} s"
                          + ("; value extrapolated to the batch of %d" % cfg.batch if decode else "")}
 
+    # ---- the metric's second half: decode us/step on cfg4, measured in the same run (single GPU, default workload)
+    decode_line = None
+    if not decode and world == 1 and args.config == "cfg3" and args.phase == "group" and not args.no_decode:
+        del wl
+        import gc
+        gc.collect()
+        torch.cuda.empty_cache()
+        decode_line = measure_decode(CONFIGS["cfg4"], dev, peaks)
+
     line = {
         "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": not decode,
@@ -312,12 +322,51 @@ def main():
                    "l2": "inputs larger than L2 (per-layer q and out are GBs); no flush" if not decode
                          else "KV pools are GBs per layer, far larger than L2; no flush"},
         "clocks": clocks.summary(), "gpu_launches": int(launches), "kernels": kernels,
-        "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
+        "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "decode": decode_line,
     }
     print(json.dumps(line))
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def measure_decode(cfg, dev, peaks, steps=50, warmup=10):
+    """cfg4: one lsa_layer_group call per step for the 64-sequence paged batch; returns the side-line dict."""
+    import numpy as np
+    import torch
+    from paper_2608_01662_b200.workload import make_workload
+    wl = make_workload(cfg, dev, with_lse=False)
+    wl.prepare()
+    for _ in range(warmup):
+        wl.step()
+    torch.cuda.synchronize()
+    assert wl.ctx.status() == 0
+    stream = torch.cuda.current_stream(dev)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0 = wl.ctx.launch_count()
+    ev0.record(stream)
+    for _ in range(steps):
+        wl.step()
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    us = ev0.elapsed_time(ev1) / steps * 1e3
+    launches = (wl.ctx.launch_count() - n0) // steps
+    wl.ctx.profile_enable(True)       # second pass: event pairs would perturb a step this short
+    for _ in range(steps):
+        wl.step()
+    prof = wl.ctx.profile_read()
+    wl.ctx.profile_enable(False)
+    positions = wl.ctx_len.cpu().numpy().astype(np.int64) - 1
+    attn_ms, attn_n = prof["sparse_attn"]
+    a = attn_bytes_per_launch(cfg, positions) / (attn_ms / attn_n * 1e-3) / 1e9
+    return {"metric": "LSA layer-group decode us/step", "value": us, "unit": "us/step", "higher_is_better": False,
+            "steps": steps, "gpu_launches_per_step": int(launches),
+            "config": {"workload": cfg.name, "batch": cfg.batch, "R": cfg.R, "ctx": [cfg.ctx_lo, cfg.ctx_hi],
+                       "l2": "KV pools are GBs per layer, far larger than L2; no flush"},
+            "kernels_us_per_step": {k: v[0] / steps * 1e3 for k, v in prof.items() if v[1] > 0},
+            "roofline": {"kernel": "sparse_attn_tc_kernel", "bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": a / peaks["hbm_gbs"], "traffic": None,
+                         "peak_source": peaks["source"], "launch_us": attn_ms / attn_n * 1e3}}
 
 
 def run_e2e(args, cfg, wl, dev):

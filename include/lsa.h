@@ -123,7 +123,7 @@ LSA_API int lsa_tune(lsa_ctx* ctx, int knob, int value);
  * launches go unrecorded).  lsa_profile_read waits for the stream and writes, per class, the summed
  * device time in ms and the number of recorded launches (host arrays of LSA_K_COUNT entries), then
  * starts over.  The first enable creates the events (host resources only). */
-enum { LSA_K_MEANS = 0, LSA_K_COARSE, LSA_K_FINE_SELECT, LSA_K_SELECT, LSA_K_CONVERT, LSA_K_ATTN, LSA_K_MERGE, LSA_K_COUNT };
+enum { LSA_K_MEANS = 0, LSA_K_COARSE, LSA_K_FINE_SELECT, LSA_K_SELECT, LSA_K_CONVERT, LSA_K_ATTN, LSA_K_MERGE, LSA_K_COUNT };   /* lsa_merge is timed as LSA_K_MERGE */
 LSA_API int lsa_profile_enable(lsa_ctx* ctx, int on);
 LSA_API int lsa_profile_read(lsa_ctx* ctx, double* total_ms, int64_t* launches);
 
@@ -231,6 +231,17 @@ LSA_API int lsa_sparse_attn(lsa_ctx* ctx, const lsa_params* p, const void* q, co
                     int64_t ld_k, int64_t ld_v, const int32_t* sparse_idx, const int32_t* n_sparse,
                     const int32_t* rows, const int32_t* n_rows, int64_t q_pos0, int64_t n_query,
                     int64_t n_key, const int32_t* ctx_len, int batch, void* out, float* lse);
+
+/* Merge attention results over disjoint key sets by their log-sum-exp (the rescaling merge of the two-branch
+ * operator, Sec. 4.1.1, and of the sharded-cache decode, App. B):
+ *     lse = log sum_i exp(lse_i),   out = sum_i exp(lse_i - lse) * out_i.
+ *   outs   HOST array of n_parts device pointers, each bf16 [n_query, H, d_v] (as written by lsa_sparse_attn)
+ *   lses   HOST array of n_parts device pointers, each fp32 [n_query, H]; -inf marks an empty part
+ *   out    bf16 [n_query, H, d_v]     lse  optional fp32 [n_query, H]
+ * 1 <= n_parts <= 8.  A part is produced by lsa_sparse_attn with the budget of the other parts set to zero
+ * (k_sparse = 0: sink + window only; k_sink = k_swa = 0: sparse only), or by a rank that holds a shard of the rows. */
+LSA_API int lsa_merge(lsa_ctx* ctx, const lsa_params* p, int n_parts, const void* const* outs,
+                      const float* const* lses, int64_t n_query, void* out, float* lse);
 
 /* ---- a7: one cross-layer group (Sec. 3.2) ---------------------------------------------------- */
 

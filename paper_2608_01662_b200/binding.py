@@ -59,6 +59,8 @@ EXPORTS = {
     "lsa_sparse_attn": (c_int, [c_void_p, POINTER(LsaParams), c_void_p, c_void_p, c_void_p, c_int64, c_int64,
                                 c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_int,
                                 c_void_p, c_void_p]),
+    "lsa_merge": (c_int, [c_void_p, POINTER(LsaParams), c_int, POINTER(c_void_p), POINTER(c_void_p), c_int64, c_void_p,
+                          c_void_p]),
     "lsa_layer_group": (c_int, [c_void_p, POINTER(LsaParams), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                 c_int64, c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int, POINTER(c_void_p),
                                 POINTER(c_void_p), POINTER(c_void_p), c_int64, c_int64, POINTER(c_void_p),
@@ -213,10 +215,16 @@ class Context:
                                     _p(runs_out)), "lsa_convert")
 
     def sparse_attn(self, q, k, v, sparse_idx, n_sparse, q_pos0, n_query, n_key, out, lse=None, rows=None,
-                    n_rows=None, ctx_len=None, batch=1):
-        self._chk(lib().lsa_sparse_attn(self.h, ctypes.byref(self.params), _p(q), _p(k), _p(v), k.stride(0),
+                    n_rows=None, ctx_len=None, batch=1, params=None):
+        prm = params if params is not None else self.params
+        self._chk(lib().lsa_sparse_attn(self.h, ctypes.byref(prm), _p(q), _p(k), _p(v), k.stride(0),
                                         v.stride(0), _p(sparse_idx), _p(n_sparse), _p(rows), _p(n_rows), q_pos0,
                                         n_query, n_key, _p(ctx_len), batch, _p(out), _p(lse)), "lsa_sparse_attn")
+
+    def merge(self, outs, lses, n_query, out, lse=None, params=None):
+        prm = params if params is not None else self.params
+        self._chk(lib().lsa_merge(self.h, ctypes.byref(prm), len(outs), _parr(outs), _parr(lses), n_query, _p(out),
+                                  _p(lse)), "lsa_merge")
 
     def layer_group(self, q_idx, w, k_idx, k_scale, kmean, q_pos0, n_query, n_key, q, k, v, out, lse, sparse_idx,
                     n_sparse, page_table=None, ctx_len=None):

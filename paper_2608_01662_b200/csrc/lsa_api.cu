@@ -437,6 +437,23 @@ int lsa_sparse_attn(lsa_ctx* c, const lsa_params* p, const void* q, const void* 
   return run_attn(c, p, q, k, v, ld_k, ld_v, sparse_idx, n_sparse, rows, n_rows, q_pos0, n_query, ctx_len, batch, out, lse);
 }
 
+int lsa_merge(lsa_ctx* c, const lsa_params* p, int n_parts, const void* const* outs, const float* const* lses,
+              int64_t n_query, void* out, float* lse) {
+  if (c == nullptr || p == nullptr || p->struct_size != sizeof(lsa_params)) return LSA_ERR_ARG;
+  if (n_parts < 1 || n_parts > 8 || outs == nullptr || lses == nullptr || out == nullptr || n_query < 0) return LSA_ERR_ARG;
+  if (p->n_heads <= 0 || p->d_v <= 0 || (p->d_v % 2)) return LSA_ERR_SHAPE;
+  lsa::MergeArgs a{};
+  a.n_parts = n_parts; a.H = p->n_heads; a.DV = p->d_v; a.n_query = static_cast<int>(n_query);
+  for (int i = 0; i < n_parts; ++i) {
+    if (outs[i] == nullptr || lses[i] == nullptr) return LSA_ERR_ARG;
+    a.outs[i] = outs[i];
+    a.lses[i] = lses[i];
+  }
+  a.out = out; a.lse = lse;
+  cudaError_t e = timed(c, LSA_K_MERGE, [&] { return lsa::launch_merge_parts(a, c->stream, &c->launches); });
+  return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
+}
+
 int lsa_layer_group(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w, const void* k_idx,
                     const float* k_scale, const void* kmean, int64_t q_pos0, int64_t n_query, int64_t n_key,
                     const int32_t* page_table, int64_t page_table_stride, const int32_t* ctx_len, int batch,

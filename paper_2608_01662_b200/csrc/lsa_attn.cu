@@ -305,6 +305,38 @@ __global__ void merge_splits_kernel(const float* __restrict__ part_out, const fl
   if (lse != nullptr && threadIdx.x == 0) lse[static_cast<int64_t>(qi) * H + h] = (m + log2f(den)) / kLog2e;
 }
 
+// lsa_merge: parts are finished results (bf16, natural-log lse) of attention over disjoint key sets.
+__global__ void merge_parts_kernel(MergeArgs a) {
+  const int qi = blockIdx.x, h = blockIdx.y;
+  const int64_t row = static_cast<int64_t>(qi) * a.H + h;
+  float wgt[8];
+  float m = -INFINITY;
+  for (int s = 0; s < a.n_parts; ++s) {
+    wgt[s] = a.lses[s][row];
+    m = fmaxf(m, wgt[s]);
+  }
+  float den = 0.f;
+  for (int s = 0; s < a.n_parts; ++s) {
+    wgt[s] = m > -INFINITY ? __expf(wgt[s] - m) : 0.f;
+    den += wgt[s];
+  }
+  const float inv = den > 0.f ? 1.f / den : 0.f;
+  for (int d = threadIdx.x * 2; d < a.DV; d += blockDim.x * 2) {
+    float2 acc = make_float2(0.f, 0.f);
+    for (int s = 0; s < a.n_parts; ++s) {
+      const float w = wgt[s] * inv;
+      if (w > 0.f) {
+        const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(
+            reinterpret_cast<const __nv_bfloat16*>(a.outs[s]) + row * a.DV + d));
+        acc.x += w * v.x;
+        acc.y += w * v.y;
+      }
+    }
+    *reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(a.out) + row * a.DV + d) = pack_bf16(acc.x, acc.y);
+  }
+  if (a.lse != nullptr && threadIdx.x == 0) a.lse[row] = den > 0.f ? m + logf(den) : -INFINITY;
+}
+
 template <int H, int DQK, int DV, bool SEP_V>
 cudaError_t launch_attn_t(const AttnArgs& a, cudaStream_t st, int64_t* n_launch) {
   const size_t smem = sizeof(AttnSmem<H, DQK, DV, SEP_V>);
@@ -321,6 +353,13 @@ cudaError_t launch_attn_t(const AttnArgs& a, cudaStream_t st, int64_t* n_launch)
 
 bool attn_shape_supported(int H, int DQK, int DV) {
   return (H == 16 && DQK == 128 && DV == 128) || (H == 64 && DQK == 576 && DV == 512);
+}
+
+cudaError_t launch_merge_parts(const MergeArgs& a, cudaStream_t st, int64_t* n_launch) {
+  if (a.n_query == 0) return cudaSuccess;
+  merge_parts_kernel<<<dim3(a.n_query, a.H), 128, 0, st>>>(a);
+  ++*n_launch;
+  return cudaGetLastError();
 }
 
 cudaError_t launch_merge(const AttnArgs& a, cudaStream_t st, int64_t* n_launch) {

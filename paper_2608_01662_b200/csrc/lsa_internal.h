@@ -77,6 +77,15 @@ bool attn_tc_supported(const AttnArgs& a);
 cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t st, int64_t* n_launch);
 cudaError_t launch_merge(const AttnArgs& a, cudaStream_t st, int64_t* n_launch);
 
+struct MergeArgs {
+  int n_parts, H, DV, n_query;
+  const void* outs[8];
+  const float* lses[8];
+  void* out;
+  float* lse;
+};
+cudaError_t launch_merge_parts(const MergeArgs& a, cudaStream_t st, int64_t* n_launch);
+
 bool index_shape_supported(int HI, int DI);
 bool attn_shape_supported(int H, int DQK, int DV);
 
