@@ -33,6 +33,7 @@ namespace {
 constexpr size_t kStatusBytes = 256;
 constexpr int kMaxSplit = 16;
 constexpr int kProfPairs = 4096;
+constexpr int64_t kFlatFusedMaxKeys = 4096;   // caches up to this length: the fused fine kernel scores every eligible page
 
 // Runs `launch` (a callable returning cudaError_t), bracketed by an event pair of class `cat` when
 // profiling is on and pairs are left.
@@ -84,7 +85,7 @@ int check_params(const lsa_params* p, bool need_index, bool need_attn) {
 
 // Workspace map.  All offsets are multiples of 256 bytes.
 struct WsLayout {
-  size_t page_scores, rows, n_rows, part_out, part_lse, fine_keys, fine_pages, total;
+  size_t page_scores, rows, n_rows, part_out, part_lse, fine_keys, fine_pages, wide_keys, total;
   int ps_ld, rows_ld;
 };
 
@@ -108,8 +109,15 @@ WsLayout ws_layout(const lsa_params* p, int64_t n_query, int64_t n_key_max, int 
     l.fine_pages = off;
     off += align_up(static_cast<size_t>(batch) * 65 * sizeof(int32_t), 256);
   }
+  const bool flat = !p->hi_enable && !p->paged && n_key_max > kFlatFusedMaxKeys;
+  if (flat && p->key_dtype == LSA_KEY_E4M3) {
+    // flat indexer on e4m3 keys: the codes widened to bf16 for the dense scoring
+    l.wide_keys = off;
+    off += align_up(static_cast<size_t>(n_key_max) * p->d_idx * 2, 256);
+  }
   const int P = p->page > 0 ? p->page : 64;
-  l.ps_ld = static_cast<int>(align_up(static_cast<size_t>((n_key_max + P - 1) / P), 4));
+  // hierarchical: one score per page; flat: one score per token
+  l.ps_ld = static_cast<int>(align_up(static_cast<size_t>(flat ? n_key_max : (n_key_max + P - 1) / P), 4));
   l.page_scores = off;
   off += align_up(static_cast<size_t>(nq) * l.ps_ld * sizeof(float), 256);
   l.total = off;
@@ -143,8 +151,8 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
   const int64_t nq = p->paged ? batch : n_query;
   if (nq == 0) return LSA_OK;
   const int64_t n_key_max = p->paged ? pt_stride * p->kv_page : n_key;
-  // without the coarse stage every eligible page is scored: the candidate buffer bounds the cache length
-  if (!p->hi_enable && n_key_max > 4096) return LSA_ERR_SHAPE;
+  const bool flat = !p->hi_enable && n_key_max > kFlatFusedMaxKeys;
+  if (flat && p->paged) return LSA_ERR_SHAPE;   // the flat indexer over long caches is built for contiguous caches only
   const int64_t chunk = (!p->paged && p->q_chunk > 0) ? p->q_chunk : nq;
   const WsLayout l = ws_layout(p, chunk < nq ? chunk : nq, n_key_max, batch);
   if (c->ws == nullptr || l.total > c->ws_bytes) return LSA_ERR_WORKSPACE;
@@ -175,6 +183,33 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
       }
     }
     cudaError_t e = cudaSuccess;
+    if (flat) {
+      // Eq. 7 without the hierarchy: dense causal token scores (the coarse kernel with one token per "page"), then
+      // the top-K_sparse of each row.  e4m3 keys are widened to bf16 once; their scale enters at the comparison.
+      const void* keys_bf16 = k_idx;
+      if (a.key_e4m3) {
+        void* wide = c->ws + l.wide_keys;
+        if (q0 == 0) e = timed(c, LSA_K_MEANS, [&] { return lsa::launch_widen_e4m3(k_idx, wide, n_key * p->d_idx, c->stream, &c->launches); });
+        keys_bf16 = wide;
+      }
+      lsa::IndexArgs d = a;
+      d.P = 1; d.B = 1; d.M = 0; d.kmean = keys_bf16; d.hi_enable = 1;
+      if (e == cudaSuccess)
+        e = timed(c, LSA_K_COARSE, [&] {
+          return lsa::coarse_tc_supported(d) ? lsa::launch_coarse_tc(d, c->tune[LSA_TUNE_COARSE_GROUPS], c->stream, &c->launches)
+                                             : lsa::launch_coarse(d, c->stream, &c->launches);
+        });
+      if (e == cudaSuccess)
+        e = timed(c, LSA_K_SELECT, [&] {
+          return lsa::launch_select(a.page_scores, a.ps_ld, nullptr, a.key_e4m3 ? k_scale : nullptr, a.q_pos0, a.n_query,
+                                    n_key, p->k_sparse, 1, p->k_sink, p->k_swa, a.sparse_idx, a.n_sparse, c->stream,
+                                    &c->launches);
+        });
+      if (e == cudaSuccess && a.pages_out != nullptr)
+        e = cudaMemsetAsync(a.pages_out, 0xff, static_cast<size_t>(a.n_query) * p->keep_pages * sizeof(int32_t), c->stream);
+      if (e != cudaSuccess) return cuda_fail(c, e);
+      continue;
+    }
     if (p->hi_enable)
       e = timed(c, LSA_K_COARSE, [&] {
         return lsa::coarse_tc_supported(a) ? lsa::launch_coarse_tc(a, c->tune[LSA_TUNE_COARSE_GROUPS], c->stream, &c->launches)
@@ -398,7 +433,7 @@ int lsa_select(lsa_ctx* c, const lsa_params* p, const float* scores, int64_t ld_
   if (k > 8192 || n_cand > 0x7fffffff) return LSA_ERR_SHAPE;
   if (n_query == 0 || k == 0) return LSA_OK;
   cudaError_t e = timed(c, LSA_K_SELECT, [&] {
-    return lsa::launch_select(scores, ld_scores, cand_pos, q_pos0, static_cast<int>(n_query), n_cand, k, apply_range,
+    return lsa::launch_select(scores, ld_scores, cand_pos, nullptr, q_pos0, static_cast<int>(n_query), n_cand, k, apply_range,
                               p->k_sink, p->k_swa, idx_out, n_out, c->stream, &c->launches);
   });
   return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);

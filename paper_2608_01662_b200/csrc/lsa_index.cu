@@ -534,7 +534,8 @@ __global__ void __launch_bounds__(kSelThreads) fine_topk_kernel(IndexArgs p) {
 // standalone selection on caller-given scores
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __restrict__ scores, int64_t ld,
-                                                            const int32_t* __restrict__ cand_pos, int64_t q_pos0,
+                                                            const int32_t* __restrict__ cand_pos,
+                                                            const float* __restrict__ pos_scale, int64_t q_pos0,
                                                             int64_t n_cand, int k, int apply_range, int S, int W,
                                                             int32_t* __restrict__ idx_out, int32_t* __restrict__ n_out) {
   __shared__ SelectScratch sc;
@@ -547,10 +548,24 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
     const int64_t s = id(i);
     if (s < 0) return 0u;
     if (apply_range && (s < lo || s > hi)) return 0u;
-    return score_key(row[i]);
+    // pos_scale: per-position factor of the score (the fp32 scale of an e4m3 key), applied before the comparison
+    return score_key(pos_scale ? row[i] * pos_scale[s] : row[i]);
   };
-  const int n = block_select_topk(key, id, static_cast<int>(n_cand), k, idx_out + static_cast<int64_t>(qi) * k, sc);
-  if (threadIdx.x == 0) n_out[qi] = n;
+  // columns that are positions: nothing beyond the range can take part, so it is not even scanned
+  int n = static_cast<int>(n_cand);
+  if (pos == nullptr && apply_range) n = static_cast<int>(max64(0, min64(n_cand, hi + 1)));
+  const int n_sel = block_select_topk(key, id, n, k, idx_out + static_cast<int64_t>(qi) * k, sc);
+  if (threadIdx.x == 0) n_out[qi] = n_sel;
+}
+
+// e4m3 codes -> the same values as bf16 (exact), for the dense scoring of the flat indexer
+__global__ void widen_e4m3_kernel(const uint4* __restrict__ codes, uint4* __restrict__ out, int64_t n_units) {
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= n_units) return;
+  uint4 lo16, hi16;
+  e4m3x16_to_bf16(codes[i], lo16, hi16);
+  out[2 * i] = lo16;
+  out[2 * i + 1] = hi16;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -685,11 +700,21 @@ cudaError_t launch_fine_select(const IndexArgs& a, cudaStream_t st, int64_t* n_l
   return a.key_e4m3 ? launch_fine_t<64, 128, true>(a, st, n_launch) : launch_fine_t<64, 128, false>(a, st, n_launch);
 }
 
-cudaError_t launch_select(const float* scores, int64_t ld, const int32_t* cand_pos, int64_t q_pos0, int n_query,
-                          int64_t n_cand, int k, int apply_range, int S, int W, int32_t* idx_out, int32_t* n_out,
-                          cudaStream_t st, int64_t* n_launch) {
+cudaError_t launch_widen_e4m3(const void* codes, void* out_bf16, int64_t n_elems, cudaStream_t st, int64_t* n_launch) {
+  const int64_t n_units = n_elems / 16;
+  if (n_units == 0) return cudaSuccess;
+  widen_e4m3_kernel<<<static_cast<unsigned>((n_units + 255) / 256), 256, 0, st>>>(
+      reinterpret_cast<const uint4*>(codes), reinterpret_cast<uint4*>(out_bf16), n_units);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_select(const float* scores, int64_t ld, const int32_t* cand_pos, const float* pos_scale,
+                          int64_t q_pos0, int n_query, int64_t n_cand, int k, int apply_range, int S, int W,
+                          int32_t* idx_out, int32_t* n_out, cudaStream_t st, int64_t* n_launch) {
   if (n_query == 0) return cudaSuccess;
-  select_kernel<<<n_query, kSelThreads, 0, st>>>(scores, ld, cand_pos, q_pos0, n_cand, k, apply_range, S, W, idx_out, n_out);
+  select_kernel<<<n_query, kSelThreads, 0, st>>>(scores, ld, cand_pos, pos_scale, q_pos0, n_cand, k, apply_range, S, W,
+                                                 idx_out, n_out);
   ++*n_launch;
   return cudaGetLastError();
 }

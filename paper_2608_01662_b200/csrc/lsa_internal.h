@@ -64,9 +64,10 @@ cudaError_t launch_coarse(const IndexArgs& a, cudaStream_t st, int64_t* n_launch
 bool coarse_tc_supported(const IndexArgs& a);
 cudaError_t launch_coarse_tc(const IndexArgs& a, int groups, cudaStream_t st, int64_t* n_launch);
 cudaError_t launch_fine_select(const IndexArgs& a, cudaStream_t st, int64_t* n_launch);
-cudaError_t launch_select(const float* scores, int64_t ld, const int32_t* cand_pos, int64_t q_pos0, int n_query,
-                          int64_t n_cand, int k, int apply_range, int S, int W, int32_t* idx_out, int32_t* n_out,
-                          cudaStream_t st, int64_t* n_launch);
+cudaError_t launch_select(const float* scores, int64_t ld, const int32_t* cand_pos, const float* pos_scale,
+                          int64_t q_pos0, int n_query, int64_t n_cand, int k, int apply_range, int S, int W,
+                          int32_t* idx_out, int32_t* n_out, cudaStream_t st, int64_t* n_launch);
+cudaError_t launch_widen_e4m3(const void* codes, void* out_bf16, int64_t n_elems, cudaStream_t st, int64_t* n_launch);
 cudaError_t launch_convert(int S, int W, int Ksp, int paged, int kv_page, const int32_t* sparse_idx,
                            const int32_t* n_sparse, int64_t q_pos0, int n_query, const int32_t* page_table,
                            int64_t pt_stride, const int32_t* ctx_len, int32_t* rows_out, int32_t* n_rows_out,

@@ -115,6 +115,30 @@ def test_small_mla_prefill(cuda_device, cfg):
     m.assert_ok(pu.TOL_FP8 if cfg.key_dtype == "e4m3" else pu.TOL_BF16)
 
 
+FLAT_BF16 = CONFIGS["cfg2"].replace(name="flat_bf16", L=5000, Ksp=512, W=256, R=1, seed=14, hi_enable=False)
+FLAT_FP8 = CONFIGS["cfg3"].replace(name="flat_fp8", L=6000, Ksp=512, W=384, R=1, seed=15, hi_enable=False)
+FLAT_SHORT = CONFIGS["cfg1"].replace(name="flat_short", hi_enable=False)          # cache <= 4096: fused kernel
+FLAT_CFG1 = CONFIGS["cfg1"].replace(name="flat_cfg1", L=4600, hi_enable=False)    # 8-head indexer, dense path
+
+
+@pytest.mark.parametrize("cfg", [FLAT_BF16, FLAT_FP8, FLAT_SHORT, FLAT_CFG1], ids=lambda c: c.name)
+def test_flat_indexer_without_the_hierarchy(cuda_device, cfg):
+    """hi_enable = 0: Eq. 7 over the whole scoring range (dense token scores + top-K for long caches)."""
+    wl = PrefillWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.step()
+    assert wl.ctx.status() == 0
+    m = pu.check_prefill(wl, pu.boundary_queries(cfg, 0, cfg.L, 60, seed=4))
+    print(cfg.name, m.summary())
+    m.assert_ok(pu.TOL_FP8 if cfg.key_dtype == "e4m3" else pu.TOL_BF16)
+    # flat and hierarchical agree wherever the hierarchy keeps every eligible page
+    hier = PrefillWorkload(cfg.replace(hi_enable=True), cuda_device)
+    hier.prepare()
+    hier.index()
+    t_all = (cfg.M + cfg.S // cfg.P) * cfg.P + cfg.W          # first query with more than M eligible pages
+    assert torch.equal(hier.sparse_idx[:t_all], wl.sparse_idx[:t_all])
+
+
 def test_prefill_query_window_with_offset_matches_whole_run(cuda_device):
     """Queries [q_pos0, q_pos0+n) scored alone (chunked prefill) give the rows of the full run."""
     cfg = SMALL_MLA.replace(R=1)
