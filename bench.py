@@ -40,6 +40,9 @@ def parse_args():
     ap.add_argument("--phase", default="group", choices=["group", "index"],
                     help="group: whole lsa_layer_group step; index: indexer only (no attention tensors are allocated; for profiling)")
     ap.add_argument("--attn-tc", type=int, default=-1, help="override LSA_TUNE_ATTN_TC (0 or 1)")
+    ap.add_argument("--seq-len", type=int, default=0, help="override the prefill length L of the config (profiling sweeps)")
+    ap.add_argument("--q-tail", type=int, default=0, help="score only the last N queries of the sequence")
+    ap.add_argument("--flat", action="store_true", help="hi_enable = 0: flat indexer (Eq. 7) instead of the hierarchy")
     ap.add_argument("--coarse-groups", type=int, default=0, help="override LSA_TUNE_COARSE_GROUPS (1 or 2)")
     return ap.parse_args()
 
@@ -210,6 +213,12 @@ def main():
     kw = {}
     if not decode and cfg.q_chunk and cfg.L > 262144:
         kw = dict(q_pos0=cfg.L - cfg.q_chunk, n_query=cfg.q_chunk)
+    if args.seq_len:
+        cfg = cfg.replace(L=args.seq_len)
+    if args.flat:
+        cfg = cfg.replace(hi_enable=False)
+    if args.q_tail:
+        kw = dict(q_pos0=cfg.L - args.q_tail, n_query=args.q_tail)
     if args.phase == "index":
         cfg = cfg.replace(R=0)
         args.no_e2e = True
@@ -305,7 +314,7 @@ def main():
 
     # ---- the metric's second half: decode us/step on cfg4, measured in the same run (single GPU, default workload)
     decode_line = None
-    if not decode and world == 1 and args.config == "cfg3" and args.phase == "group" and not args.no_decode:
+    if not decode and world == 1 and args.config == "cfg3" and args.phase == "group" and not args.no_decode and not (args.seq_len or args.q_tail or args.flat):
         del wl
         import gc
         gc.collect()
