@@ -124,6 +124,12 @@ def attn_bytes_per_launch(cfg, positions):
     return float(rows * cfg.d_qk * 2 + len(positions) * cfg.H * (cfg.d_qk + cfg.d_v) * 2)
 
 
+# DRAM traffic of one attention launch, from the ncu capture of the same kernel on cfg3 cut to 16384 queries
+# (profiles/sparse_attn_tc_cfg3_16k.md: dram__bytes_read.sum 1.346437 GB + dram__bytes_write.sum 1.041851 GB).
+# Traffic there is q + out (the KV latent stays in L2), so it scales with the number of queries of a launch.
+NCU_ATTN_DRAM_BYTES_PER_QUERY = (1.346437e9 + 1.041851e9) / 16384
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -294,7 +300,10 @@ def main():
             a = attn_flops_per_launch(cfg, positions) / dur_s / 1e12
             roofline = {"kernel": "sparse_attn_tc_kernel" if cfg.H == 64 else "sparse_attn_kernel", "bound": "tensor", "achieved": a,
                         "peak": peaks["tensor_tflops"], "unit": "TFLOP/s", "frac": a / peaks["tensor_tflops"],
-                        "traffic": None, "peak_source": peaks["source"], "launch_ms": attn_ms / attn_n}
+                        "traffic": NCU_ATTN_DRAM_BYTES_PER_QUERY * len(positions) if cfg.H == 64 else None,
+                        "traffic_source": "ncu capture at 16384 queries, scaled by queries per launch",
+                        "algorithmic_bytes": float(len(positions)) * cfg.H * (cfg.d_qk + cfg.d_v) * 2,
+                        "peak_source": peaks["source"], "launch_ms": attn_ms / attn_n}
     kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps}
                for k, v in prof.items() if v[1] > 0}
 
@@ -313,6 +322,7 @@ def main():
                          + ("; value extrapolated to the batch of %d" % cfg.batch if decode else "")}
 
     # ---- the metric's second half: decode us/step on cfg4, measured in the same run (single GPU, default workload)
+    queries_per_step = wl.units()
     decode_line = None
     if not decode and world == 1 and args.config == "cfg3" and args.phase == "group" and not args.no_decode and not (args.seq_len or args.q_tail or args.flat):
         del wl
@@ -327,7 +337,7 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "mode": cfg.mode, "L": cfg.L, "batch": cfg.batch, "R": cfg.R,
                    "indexer_keys": cfg.key_dtype, "P": cfg.P, "B": cfg.B, "M": cfg.M, "K_sparse": cfg.Ksp,
-                   "K_sink": cfg.S, "K_swa": cfg.W, "queries_per_step": wl.units(),
+                   "K_sink": cfg.S, "K_swa": cfg.W, "queries_per_step": queries_per_step,
                    "l2": "inputs larger than L2 (per-layer q and out are GBs); no flush" if not decode
                          else "KV pools are GBs per layer, far larger than L2; no flush"},
         "clocks": clocks.summary(), "gpu_launches": int(launches), "kernels": kernels,
