@@ -695,6 +695,13 @@ static cudaError_t launch_fine_t(const IndexArgs& a, cudaStream_t st, int64_t* n
 
 cudaError_t launch_fine_select(const IndexArgs& a, cudaStream_t st, int64_t* n_launch) {
   if (a.n_query == 0) return cudaSuccess;
+  if (fine_tc_supported(a)) {
+    cudaError_t e = launch_fine_select_tc(a, st, n_launch);
+    if (e != cudaSuccess || a.fine_parts <= 1) return e;
+    fine_topk_kernel<<<a.n_query, kSelThreads, 0, st>>>(a);
+    ++*n_launch;
+    return cudaGetLastError();
+  }
   if (a.HI == 8 && a.DI == 64)
     return a.key_e4m3 ? launch_fine_t<8, 64, true>(a, st, n_launch) : launch_fine_t<8, 64, false>(a, st, n_launch);
   return a.key_e4m3 ? launch_fine_t<64, 128, true>(a, st, n_launch) : launch_fine_t<64, 128, false>(a, st, n_launch);
