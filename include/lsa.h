@@ -157,7 +157,9 @@ LSA_API int lsa_block_means(lsa_ctx* ctx, const lsa_params* p, const void* k_idx
  *   sparse_idx  int32 [n_query, Ksp]  ascending positions (logical), padded with -1
  *   n_sparse    int32 [n_query]
  *   pages_out   optional int32 [n_query, M] kept pages ascending, -1 padded (NULL to skip)
- * Scratch: the page-score matrix fp32 [n_query, ceil(n_key_max/P)] in the workspace. */
+ * Scratch: the page-score matrix fp32 [n_query, ceil(n_key_max/P)] in the workspace; for e4m3 caches with the
+ * 64-head, 128-dim indexer also a bf16 copy of the codes [n_key_max, d_idx] (exact, unscaled), rewritten by every call,
+ * from which the fine stage fetches key tiles. */
 LSA_API int lsa_index(lsa_ctx* ctx, const lsa_params* p, const void* q_idx, const float* w, const void* k_idx,
               const float* k_scale, const void* kmean, int64_t q_pos0, int64_t n_query, int64_t n_key,
               const int32_t* page_table, int64_t page_table_stride, const int32_t* ctx_len, int batch,

@@ -110,8 +110,9 @@ WsLayout ws_layout(const lsa_params* p, int64_t n_query, int64_t n_key_max, int 
     off += align_up(static_cast<size_t>(batch) * 65 * sizeof(int32_t), 256);
   }
   const bool flat = !p->hi_enable && !p->paged && n_key_max > kFlatFusedMaxKeys;
-  if (flat && p->key_dtype == LSA_KEY_E4M3) {
-    // flat indexer on e4m3 keys: the codes widened to bf16 for the dense scoring
+  const bool tc_fine = !p->paged && p->n_heads_idx == 64 && p->d_idx == 128;
+  if ((flat || tc_fine) && p->key_dtype == LSA_KEY_E4M3) {
+    // e4m3 codes widened to bf16 once per call: dense scoring of the flat indexer, TMA source of the fine stage
     l.wide_keys = off;
     off += align_up(static_cast<size_t>(n_key_max) * p->d_idx * 2, 256);
   }
@@ -183,6 +184,13 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
       }
     }
     cudaError_t e = cudaSuccess;
+    if (!flat && a.key_e4m3 && l.wide_keys != 0) {
+      // the fine stage reads key tiles by TMA from a bf16 copy of the codes (exact; scales enter after the dot products)
+      void* wide = c->ws + l.wide_keys;
+      if (q0 == 0) e = timed(c, LSA_K_MEANS, [&] { return lsa::launch_widen_e4m3(k_idx, wide, n_key * p->d_idx, c->stream, &c->launches); });
+      if (e != cudaSuccess) return cuda_fail(c, e);
+      a.k_wide = wide;
+    }
     if (flat) {
       // Eq. 7 without the hierarchy: dense causal token scores (the coarse kernel with one token per "page"), then
       // the top-K_sparse of each row.  e4m3 keys are widened to bf16 once; their scale enters at the comparison.

@@ -208,12 +208,14 @@ coarse_score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_c
   if (warp == 1) tc::tmem_dealloc(tmem_base, kTmemCols);
 }
 
+}  // namespace
+
 // ---- host side: tensor maps -----------------------------------------------------------------------
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-EncodeTiledFn encode_tiled_fn() {
+static EncodeTiledFn encode_tiled_fn() {
   static EncodeTiledFn fn = [] {
     void* f = nullptr;
     cudaDriverEntryPointQueryResult q;
@@ -224,6 +226,8 @@ EncodeTiledFn encode_tiled_fn() {
   }();
   return fn;
 }
+
+bool tma_available() { return encode_tiled_fn() != nullptr; }
 
 // bf16 matrix [rows, 128] row-major, box = 64 columns x box_rows rows, 128-byte swizzle, zero fill outside.
 bool make_map_bf16_128(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows) {
@@ -237,6 +241,8 @@ bool make_map_bf16_128(CUtensorMap* map, const void* base, uint64_t rows, uint32
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+
+namespace {
 
 template <int NG>
 cudaError_t launch_tc(const IndexArgs& a, cudaStream_t st, int64_t* n_launch) {
@@ -260,7 +266,7 @@ cudaError_t launch_tc(const IndexArgs& a, cudaStream_t st, int64_t* n_launch) {
 
 bool coarse_tc_supported(const IndexArgs& a) {
   return a.HI == kHI && a.DI == kDI && !a.paged && (reinterpret_cast<uintptr_t>(a.q_idx) & 15u) == 0 &&
-         (reinterpret_cast<uintptr_t>(a.kmean) & 15u) == 0 && encode_tiled_fn() != nullptr;
+         (reinterpret_cast<uintptr_t>(a.kmean) & 15u) == 0 && tma_available();
 }
 
 cudaError_t launch_coarse_tc(const IndexArgs& a, int groups, cudaStream_t st, int64_t* n_launch) {

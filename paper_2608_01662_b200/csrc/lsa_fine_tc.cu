@@ -4,8 +4,10 @@
 // After the page top-M (Eq. 10), the kept pages are scored in tiles of 128 candidate keys: keys are the M = 128
 // rows of the MMA, the 64 heads its N, d_I = 128 its K (8 steps of M128 N64 K16 per tile):
 //
-//   warps 0-2   gather the tile's key rows; e4m3 codes are widened to bf16 in registers (exact) and stored in the
-//               128B-swizzled K-major layout tcgen05.mma reads; the per-token scales ride along
+//   warps 0-2   bring the tile's key rows into the 128B-swizzled K-major layout tcgen05.mma reads.  bf16 rows (bf16
+//               caches, or e4m3 caches the caller widened once per call: k_wide) come by TMA, four 64-row boxes per
+//               tile issued by one thread; without a widened copy the warps gather e4m3 codes and widen them in
+//               registers (exact), the per-token scales riding along
 //   warp 3      one thread issues the MMAs into one of two 64-column TMEM accumulators
 //   warps 4-7   epilogue: tcgen05.ld, sum_j w_j * relu(acc_j) in-thread (one thread = one key), times the key's
 //               scale, range check, order-preserving key into the candidate buffer
@@ -41,8 +43,10 @@ struct FineTcSmem {
   uint32_t tmem_slot;
 };
 
-template <bool E4M3>
-__global__ void __launch_bounds__(kFineThreads, 2) fine_select_tc_kernel(IndexArgs p) {
+// TMA: key tiles are bf16 rows fetched through `map`; otherwise e4m3 codes gathered and widened by warps 0-2.
+template <bool TMA>
+__global__ void __launch_bounds__(kFineThreads, 2) fine_select_tc_kernel(const __grid_constant__ CUtensorMap map, IndexArgs p) {
+  constexpr bool E4M3 = !TMA;   // the gather path exists for e4m3 codes only
   extern __shared__ uint8_t smem_raw[];
   FineTcSmem& sm = *reinterpret_cast<FineTcSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -93,7 +97,7 @@ __global__ void __launch_bounds__(kFineThreads, 2) fine_select_tc_kernel(IndexAr
   // ---- set-up of the tile pipeline
   if (tid == 0) {
     for (int b = 0; b < 2; ++b) {
-      tc::mbar_init(smem_u32(&sm.k_full[b]), kLoadThreads);
+      tc::mbar_init(smem_u32(&sm.k_full[b]), TMA ? 1 : kLoadThreads);
       tc::mbar_init(smem_u32(&sm.k_empty[b]), 1);
       tc::mbar_init(smem_u32(&sm.acc_full[b]), 1);
       tc::mbar_init(smem_u32(&sm.acc_empty[b]), 4);
@@ -137,7 +141,24 @@ __global__ void __launch_bounds__(kFineThreads, 2) fine_select_tc_kernel(IndexAr
     return p.paged ? static_cast<int64_t>(pt[pos >> pshift]) * p.P + (pos & (p.P - 1)) : pos;
   };
 
-  if (warp < 3) {
+  if (TMA && warp < 3) {
+    // ================= TMA producer =================
+    if (tid == 0) {
+      for (int i = 0; i < n_tiles; ++i) {
+        const int b = i & 1;
+        if (!tc::mbar_wait(smem_u32(&sm.k_empty[b]), ((i >> 1) & 1) ^ 1, p.status)) break;
+        tc::mbar_expect_tx(smem_u32(&sm.k_full[b]), 2 * kAtomA);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {   // 64 consecutive slots lie in one page; rows past the cache read as zero
+          const int c = (tile0 + i) * kTile + 64 * h;
+          const int row = c < n_slots ? static_cast<int>(slot_pos(c)) : static_cast<int>(n_key);
+#pragma unroll
+          for (int cb = 0; cb < 2; ++cb)
+            tc::tma_load_2d(smem_u32(sm.a[b][cb]) + h * 64 * 128, &map, cb * 64, row, smem_u32(&sm.k_full[b]));
+        }
+      }
+    }
+  } else if (warp < 3) {
     // ================= gather warps =================
     // Each thread owns whole key rows (rows tid and tid + 96 of the tile): all 16-byte loads of a row are in flight
     // together, then the row is widened and stored.  Rows of one page are consecutive in memory, so a warp's loads
@@ -206,13 +227,18 @@ __global__ void __launch_bounds__(kFineThreads, 2) fine_select_tc_kernel(IndexAr
     bool ok = true;
     for (int i = 0; i < n_tiles && ok; ++i) {
       const int b = i & 1;
+      const int c = (tile0 + i) * kTile + r;
+      const int64_t pos = c < n_slots ? slot_pos(c) : -1;
+      const bool cand = pos >= lo && pos <= hi;
+      float sc = 1.f;
+      if (TMA && p.key_e4m3 && cand) sc = p.k_scale[pos];   // in flight while the tile's MMAs run
       ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.acc_full[b]), (i >> 1) & 1, p.status));
       if (!ok) break;
       tc::fence_after_sync();
       uint32_t v[64];
       tc::tmem_ld64(tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + b * kHI, v);
       tc::tmem_ld_wait();
-      const float sc = E4M3 ? sm.scale[i & 3][r] : 1.f;   // read before the accumulator is handed back
+      if (!TMA) sc = sm.scale[i & 3][r];   // read before the accumulator is handed back
       tc::fence_before_sync();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(smem_u32(&sm.acc_empty[b]));
@@ -226,13 +252,7 @@ __global__ void __launch_bounds__(kFineThreads, 2) fine_select_tc_kernel(IndexAr
         a0 = fmaf(ww.z, fmaxf(__uint_as_float(v[4 * j + 2]), 0.f), a0);
         a1 = fmaf(ww.w, fmaxf(__uint_as_float(v[4 * j + 3]), 0.f), a1);
       }
-      const int c = (tile0 + i) * kTile + r;
-      if (c < n_slots) {
-        const int64_t pos = slot_pos(c);
-        uint32_t key = 0;
-        if (pos >= lo && pos <= hi) key = score_key((a0 + a1) * sc);
-        sm.keys[c] = key;
-      }
+      if (c < n_slots) sm.keys[c] = cand ? score_key((a0 + a1) * sc) : 0u;
     }
   }
   tc::fence_before_sync();
@@ -252,26 +272,39 @@ __global__ void __launch_bounds__(kFineThreads, 2) fine_select_tc_kernel(IndexAr
   if (tid == 0) p.n_sparse[qi] = n_sel;
 }
 
-template <bool E4M3>
-cudaError_t launch_t(const IndexArgs& a, cudaStream_t st, int64_t* n_launch) {
+template <bool TMA>
+cudaError_t launch_t(const IndexArgs& a, const CUtensorMap& map, cudaStream_t st, int64_t* n_launch) {
   const size_t smem = sizeof(FineTcSmem) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(fine_select_tc_kernel<E4M3>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  cudaError_t e = cudaFuncSetAttribute(fine_select_tc_kernel<TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
   const int parts = a.fine_parts > 1 ? a.fine_parts : 1;
-  fine_select_tc_kernel<E4M3><<<dim3(a.n_query, parts), kFineThreads, smem, st>>>(a);
+  fine_select_tc_kernel<TMA><<<dim3(a.n_query, parts), kFineThreads, smem, st>>>(map, a);
   ++*n_launch;
   return cudaGetLastError();
 }
 
+// bf16 key rows the TMA path can read: the cache itself, or the widened copy of an e4m3 cache
+const void* bf16_rows(const IndexArgs& a) { return a.key_e4m3 ? a.k_wide : a.k_idx; }
+
 }  // namespace
 
 // Contiguous caches only: a paged decode step has few tiles per block, where the pipeline set-up outweighs the gain.
-bool fine_tc_supported(const IndexArgs& a) { return a.HI == kHI && a.DI == kDI && !a.paged; }
+// bf16 caches need the 16-byte alignment of a TMA source.
+bool fine_tc_supported(const IndexArgs& a) {
+  if (a.HI != kHI || a.DI != kDI || a.paged) return false;
+  const void* rows = bf16_rows(a);
+  if (rows != nullptr) return (reinterpret_cast<uintptr_t>(rows) & 15u) == 0 && tma_available();
+  return a.key_e4m3 != 0;
+}
 
 // Scoring blocks only; with fine_parts > 1 the caller follows up with the top-K kernel of lsa_index.cu.
 cudaError_t launch_fine_select_tc(const IndexArgs& a, cudaStream_t st, int64_t* n_launch) {
   if (a.n_query == 0) return cudaSuccess;
-  return a.key_e4m3 ? launch_t<true>(a, st, n_launch) : launch_t<false>(a, st, n_launch);
+  CUtensorMap map{};
+  const void* rows = bf16_rows(a);
+  if (rows == nullptr) return launch_t<false>(a, map, st, n_launch);
+  if (!make_map_bf16_128(&map, rows, static_cast<uint64_t>(a.n_key), 64)) return cudaErrorInvalidValue;
+  return launch_t<true>(a, map, st, n_launch);
 }
 
 }  // namespace lsa

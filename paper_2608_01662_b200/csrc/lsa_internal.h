@@ -12,6 +12,7 @@ struct IndexArgs {
   const float* w;         // [n_query, HI]
   const void* k_idx;      // bf16 or e4m3 codes, rows of DI
   const float* k_scale;   // per token, e4m3 only
+  const void* k_wide;     // optional: the e4m3 codes widened to bf16 (unscaled), rows of DI, contiguous caches only
   const void* kmean;      // bf16 rows of DI
   int64_t q_pos0;
   int n_query;

@@ -211,4 +211,12 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 }
 
 }  // namespace tc
+
+// ---- host side (defined in lsa_coarse_tc.cu) -----------------------------------------------------------
+// True when the driver's tensor-map encoder could be looked up.
+bool tma_available();
+// Tensor map of a bf16 matrix [rows, 128] row-major: box = 64 columns x box_rows rows, 128-byte swizzle, zero fill
+// outside.  `base` must be 16-byte aligned.
+bool make_map_bf16_128(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows);
+
 }  // namespace lsa

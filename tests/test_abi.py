@@ -33,11 +33,11 @@ def test_host_only_entry_points():
         assert n % 256 == 0 and n > 0
     p = binding.make_params(CONFIGS["cfg3"])
     assert ctypes.sizeof(p) == p.struct_size == 76
-    # cfg3 page scores: 131072 queries x 1024 pages x 4 B
-    assert binding.workspace_bytes(p, 131072, 131072) == 131072 * 1024 * 4 + 256
+    # cfg3: page scores (131072 queries x 1024 pages x 4 B) + the e4m3 keys widened to bf16 (131072 x 128 x 2 B)
+    assert binding.workspace_bytes(p, 131072, 131072) == 131072 * 1024 * 4 + 131072 * 128 * 2 + 256
     # q_chunk bounds the scratch
     p5 = binding.make_params(CONFIGS["cfg5"])
-    assert binding.workspace_bytes(p5, 1 << 20, 1 << 20) == 16384 * 4096 * 4 + 256
+    assert binding.workspace_bytes(p5, 1 << 20, 1 << 20) == 16384 * 4096 * 4 + (1 << 20) * 128 * 2 + 256
     assert binding.host_stage_bytes(p, 4096) > 4096 * 64 * (576 + 512) * 2 * 4
 
 
