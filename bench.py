@@ -43,6 +43,7 @@ def parse_args():
     ap.add_argument("--seq-len", type=int, default=0, help="override the prefill length L of the config (profiling sweeps)")
     ap.add_argument("--q-tail", type=int, default=0, help="score only the last N queries of the sequence")
     ap.add_argument("--flat", action="store_true", help="hi_enable = 0: flat indexer (Eq. 7) instead of the hierarchy")
+    ap.add_argument("--attn-split", type=int, default=0, help="override LSA_TUNE_ATTN_SPLIT (decode row splits)")
     ap.add_argument("--coarse-groups", type=int, default=0, help="override LSA_TUNE_COARSE_GROUPS (1 or 2)")
     return ap.parse_args()
 
@@ -236,6 +237,8 @@ def main():
         wl.ctx.tune(0, args.coarse_groups)
     if args.attn_tc >= 0:
         wl.ctx.tune(1, args.attn_tc)
+    if args.attn_split:
+        wl.ctx.tune(2, args.attn_split)
     torch.cuda.synchronize()
 
     def barrier():

@@ -114,8 +114,10 @@ LSA_API int64_t lsa_launch_count(lsa_ctx* ctx);
 
 /* Launch-shape knobs; results never depend on them.
  *   LSA_TUNE_COARSE_GROUPS  4-query groups held per thread block of the coarse-score kernel (1 or 2; default 2)
- *   LSA_TUNE_ATTN_TC        1 (default): MLA-shape attention on tcgen05.mma; 0: the mma.sync kernel */
-enum { LSA_TUNE_COARSE_GROUPS = 0, LSA_TUNE_ATTN_TC, LSA_TUNE_COUNT };
+ *   LSA_TUNE_ATTN_TC        1 (default): MLA-shape attention on tcgen05.mma; 0: the mma.sync kernel
+ *   LSA_TUNE_ATTN_SPLIT     row splits per sequence in paged attention: 0 (default) = chosen by the wave cost model,
+ *                           1..16 = fixed */
+enum { LSA_TUNE_COARSE_GROUPS = 0, LSA_TUNE_ATTN_TC, LSA_TUNE_ATTN_SPLIT, LSA_TUNE_COUNT };
 LSA_API int lsa_tune(lsa_ctx* ctx, int knob, int value);
 
 /* Per-kernel timing.  While enabled, every kernel-launching call records a CUDA event pair on the

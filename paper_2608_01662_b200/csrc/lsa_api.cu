@@ -246,7 +246,7 @@ int run_attn(lsa_ctx* c, const lsa_params* p, const void* q, const void* k, cons
   if (p->paged) {
     const WsLayout l = ws_layout(p, nq, 0, batch);
     if (c->ws == nullptr || l.total > c->ws_bytes) return LSA_ERR_WORKSPACE;
-    a.n_split = pick_split(c->sm_count, batch, a.rows_ld);
+    a.n_split = c->tune[LSA_TUNE_ATTN_SPLIT] > 0 ? c->tune[LSA_TUNE_ATTN_SPLIT] : pick_split(c->sm_count, batch, a.rows_ld);
     a.part_out = reinterpret_cast<float*>(c->ws + l.part_out);
     a.part_lse = reinterpret_cast<float*>(c->ws + l.part_lse);
   }
@@ -355,6 +355,7 @@ const char* lsa_last_cuda_error(lsa_ctx* c) { return c ? c->cuda_msg : ""; }
 int lsa_tune(lsa_ctx* c, int knob, int value) {
   if (c == nullptr || knob < 0 || knob >= LSA_TUNE_COUNT) return LSA_ERR_ARG;
   if (knob == LSA_TUNE_COARSE_GROUPS && value != 1 && value != 2) return LSA_ERR_ARG;
+  if (knob == LSA_TUNE_ATTN_SPLIT && (value < 0 || value > kMaxSplit)) return LSA_ERR_ARG;
   c->tune[knob] = value;
   return LSA_OK;
 }

@@ -26,6 +26,35 @@
 #include "lsa_internal.h"
 #include "lsa_tc.cuh"
 
+#ifdef LSA_TIMELINE
+// Debug build only (-DLSA_TIMELINE): per-block SM-clock stamps at the phase boundaries of the attention kernel,
+// read back with lsa_debug_timeline.  0 entry, 1 set-up done, 2 Q ready, 3 first key tile landed, 4 first S ready,
+// 5 last P handed over, 6 last P V done, 7 exit.
+__device__ long long g_timeline[1024 * 8];
+__device__ long long g_wall[1024 * 2];   // globaltimer (ns) at entry and exit
+#define LSA_WALL(k)                                                                      \
+  do {                                                                                   \
+    const unsigned blk_ = blockIdx.x + gridDim.x * blockIdx.y;                           \
+    long long t_;                                                                        \
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                              \
+    if (blk_ < 1024) g_wall[blk_ * 2 + (k)] = t_;                                        \
+  } while (0)
+extern "C" __attribute__((visibility("default"))) int lsa_debug_wall(long long* host, int n_blocks) {
+  return cudaMemcpyFromSymbol(host, g_wall, sizeof(long long) * 2 * (n_blocks < 1024 ? n_blocks : 1024)) == cudaSuccess ? 0 : -1;
+}
+#define LSA_TL(k)                                                                        \
+  do {                                                                                   \
+    const unsigned blk_ = blockIdx.x + gridDim.x * blockIdx.y;                           \
+    if (blk_ < 1024) g_timeline[blk_ * 8 + (k)] = clock64();                             \
+  } while (0)
+extern "C" __attribute__((visibility("default"))) int lsa_debug_timeline(long long* host, int n_blocks) {
+  return cudaMemcpyFromSymbol(host, g_timeline, sizeof(long long) * 8 * (n_blocks < 1024 ? n_blocks : 1024)) == cudaSuccess ? 0 : -1;
+}
+#else
+#define LSA_TL(k)
+#define LSA_WALL(k)
+#endif
+
 namespace lsa {
 
 namespace {
@@ -90,6 +119,8 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
 
   // ---- set-up
   if (tid == 0) {
+    LSA_TL(0);
+    LSA_WALL(0);
     tc::mbar_init(smem_u32(&sm.q_full), 32 * kLoadWarps);
     tc::mbar_init(smem_u32(&sm.q_tmem), kSoftmaxWarps);
     for (int b = 0; b < kKBufs; ++b) {
@@ -111,21 +142,26 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
   __syncthreads();
   tc::fence_after_sync();
   const uint32_t tmem_base = sm.tmem_slot;
+  if (tid == 0) LSA_TL(1);
 
   if (warp >= kSoftmaxWarps + kMmaWarps) {
     // ================= gather warps =================
     const int lt = tid - 32 * (kSoftmaxWarps + kMmaWarps);   // 0..127
     {
-      // the rope part of Q (dims 512-575) stays in shared memory: 64 rows x 128 bytes
-      const uint8_t* qg = reinterpret_cast<const uint8_t*>(p.q) + static_cast<int64_t>(qi) * kH * kDQK * 2 + 512 * 2;
+      // Q of this query: the rope part (dims 512-575) stays in shared memory as an MMA operand; dims 0-511 are staged
+      // in the last key buffer (64 rows x 1024 B, 16-byte chunks swizzled by row) for the softmax warps, which move
+      // them to tensor memory.  The copies share the first cp.async group, handed over with the first key tile.
+      const uint8_t* qg = reinterpret_cast<const uint8_t*>(p.q) + static_cast<int64_t>(qi) * kH * kDQK * 2;
       for (int e = lt; e < kH * 8; e += 32 * kLoadWarps) {
         const int r = e >> 3, c = e & 7;
-        cp_async16(smem_u32(sm.q_rope) + r * 128 + ((c ^ (r & 7)) << 4), qg + r * kDQK * 2 + c * 16, 16);
+        cp_async16(smem_u32(sm.q_rope) + r * 128 + ((c ^ (r & 7)) << 4), qg + r * kDQK * 2 + 512 * 2 + c * 16, 16);
+      }
+      const uint32_t stage = smem_u32(sm.k[kKBufs - 1]);
+      for (int e = lt; e < kH * 64; e += 32 * kLoadWarps) {
+        const int r = e >> 6, c = e & 63;
+        cp_async16(stage + r * 1024 + ((c ^ (r & 7)) << 4), qg + r * kDQK * 2 + c * 16, 16);
       }
       cp_async_commit();
-      cp_async_wait<0>();
-      tc::fence_proxy_async();
-      tc::mbar_arrive(smem_u32(&sm.q_full));
     }
     // Every gather warp works on every tile: warp w copies rows 16w .. 16w+15, so a freed buffer is refilled by all
     // four warps at once.  Lanes 0-15 look up the cache row of their key once; the row number is then broadcast
@@ -137,10 +173,36 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       return (i < n_tiles && lane < kRowsPerWarp) ? row_of((tile_begin + i) * kTileKeys + kRowsPerWarp * lw + lane) : -1;
     };
     int32_t my_row = my_key_row(0);
+    // Copies of up to three tiles are in flight: a tile is handed to the MMA issuers (k_full) when its cp.async group
+    // has landed, which is looked at after the next tile's copies are issued, or at once when no buffer is free.
+    int first_pend = 0, n_pend = 0;   // tiles first_pend .. first_pend + n_pend - 1 are issued but not handed over
+    bool q_handed = false;
+    auto hand_over_q = [&]() {        // call after a wait that covers the first group
+      tc::fence_proxy_async();
+      tc::mbar_arrive(smem_u32(&sm.q_full));
+      q_handed = true;
+    };
+    auto hand_over_oldest = [&]() {
+      if (n_pend >= 3) cp_async_wait<2>();
+      else if (n_pend == 2) cp_async_wait<1>();
+      else cp_async_wait<0>();
+      if (!q_handed) hand_over_q();
+      tc::fence_proxy_async();
+      tc::mbar_arrive(smem_u32(&sm.k_full[first_pend % kKBufs]));
+      ++first_pend;
+      --n_pend;
+    };
     for (int i = 0; i < n_tiles; ++i) {
       const int b = i % kKBufs;
+      const uint32_t par = ((i / kKBufs) & 1) ^ 1;
       const int32_t next_row = my_key_row(i + 1);   // fetched before the wait: off the critical path
-      if (!__all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.k_empty[b]), ((i / kKBufs) & 1) ^ 1, p.status))) break;
+      if (i == kKBufs - 1) {
+        // first use of the buffer that staged Q: the softmax warps must have moved Q to tensor memory
+        while (n_pend > 0 && !__all_sync(0xffffffffu, tc::mbar_test(smem_u32(&sm.q_tmem), 0))) hand_over_oldest();
+        if (!__all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.q_tmem), 0, p.status))) break;
+      }
+      while (n_pend > 0 && !__all_sync(0xffffffffu, tc::mbar_test(smem_u32(&sm.k_empty[b]), par))) hand_over_oldest();
+      if (!__all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.k_empty[b]), par, p.status))) break;
 #pragma unroll 4
       for (int rr = 0; rr < kRowsPerWarp; ++rr) {
         const int32_t row = __shfl_sync(0xffffffffu, my_row, rr);
@@ -152,10 +214,14 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
           cp_async16(smem_u32(sm.k[b][c >> 3]) + r * 128 + (((c & 7) ^ (r & 7)) << 4), src + c * 16, nb);
       }
       cp_async_commit();
-      cp_async_wait<0>();
-      tc::fence_proxy_async();
-      tc::mbar_arrive(smem_u32(&sm.k_full[b]));
+      ++n_pend;
+      if (n_pend == kKBufs) hand_over_oldest();
       my_row = next_row;
+    }
+    while (n_pend > 0) hand_over_oldest();
+    if (!q_handed) {
+      cp_async_wait<0>();
+      hand_over_q();
     }
   } else if (warp >= kSoftmaxWarps) {
     // ================= MMA issuers =================
@@ -164,6 +230,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       constexpr uint32_t idesc_qk = tc::idesc_bf16(kH, kTileKeys, 0, 0);
       constexpr uint32_t idesc_pv = tc::idesc_bf16(kH, 128, 0, 1);   // B = V read MN-major
       bool ok = tc::mbar_wait(smem_u32(&sm.q_full), 0, p.status) && tc::mbar_wait(smem_u32(&sm.q_tmem), 0, p.status);
+      if (x == 0) LSA_TL(2);
       // Descriptors are built once; inside the loops only the start-address word moves (one add per operand).
       constexpr uint32_t kBufBytes = kAtoms * kAtomBytes;
       const uint64_t dqr = tc::smem_desc_sw128(smem_u32(sm.q_rope), 16, 1024);
@@ -210,6 +277,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
           // S buffer qk_next&1 also holds P of tile qk_next-2: it is free once that tile's P V has completed
           if (tc::mbar_test(smem_u32(&sm.k_full[qk_next % kKBufs]), (qk_next / kKBufs) & 1) &&
               tc::mbar_test(smem_u32(&sm.pv_done[qk_next & 1]), ((qk_next >> 1) & 1) ^ 1)) {
+            if (x == 0 && qk_next == 0) LSA_TL(3);
             issue_qk(qk_next++);
             did = true;
           }
@@ -237,17 +305,18 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     const int r16 = lane & 15, hi = lane >> 4;
     const int row = 16 * quarter + r16;       // head; lanes l and l+16 share it: keys 0-31 / 32-63, O dims 0-255 / 256-511
     const uint32_t lane_addr = static_cast<uint32_t>(32 * quarter) << 16;
+    bool ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.q_full), 0, p.status));
     {
-      // Q[row, 256*hi : 256*hi+256] -> 128 columns of this lane, in the order the tensor core reads an A operand
-      // (two consecutive dims per 32-bit column)
-      const uint4* qg = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(p.q) +
-                                                       ((static_cast<int64_t>(qi) * kH + row) * kDQK + 256 * hi) * 2);
+      // Q[row, 256*hi : 256*hi+256] from the staging buffer -> 128 columns of this lane, in the order the tensor core
+      // reads an A operand (two consecutive dims per 32-bit column)
+      const uint8_t* qs = sm.k[kKBufs - 1][0] + row * 1024;
 #pragma unroll 1
       for (int part = 0; part < 2; ++part) {
         uint32_t w[64];
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          const uint4 u = qg[part * 16 + j];
+          const int c = 32 * hi + 16 * part + j;
+          const uint4 u = *reinterpret_cast<const uint4*>(qs + ((c ^ (row & 7)) << 4));
           w[4 * j] = u.x; w[4 * j + 1] = u.y; w[4 * j + 2] = u.z; w[4 * j + 3] = u.w;
         }
         tc::tmem_st64(tmem_base + lane_addr + kColQ + part * 64, w);
@@ -259,11 +328,11 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     }
     const float zs = p.sm_scale * kLog2eTc;
     float m_used = -INFINITY, l_run = 0.f;    // m_used is kept identical in both lanes of a row; l_run is a partial sum
-    bool ok = true;
     for (int i = 0; i < n_tiles && ok; ++i) {
       const int b = i & 1;
       ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.s_full[b]), (i >> 1) & 1, p.status));
       if (!ok) break;
+      if (tid == 0 && i == 0) LSA_TL(4);
       tc::fence_after_sync();
       const uint32_t s_addr = tmem_base + lane_addr + kColS + b * kSBuf;
       uint32_t v[32];
@@ -344,18 +413,24 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(smem_u32(&sm.p_ready[b]));
     }
+    if (tid == 0) LSA_TL(5);
     // ---- epilogue: O / l
     const float l_row = l_run + __shfl_xor_sync(0xffffffffu, l_run, 16);
     const float m_row = m_used;
     bool have_o = ok && n_tiles > 0;
     if (have_o) have_o = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done[(n_tiles - 1) & 1]), ((n_tiles - 1) >> 1) & 1, p.status));
     tc::fence_after_sync();
+    if (tid == 0) LSA_TL(6);
     const float inv = (have_o && l_row > 0.f) ? 1.f / l_row : 0.f;
-    const int d0 = hi * 256;
-    __nv_bfloat16* out = nullptr;
-    float* pout = nullptr;
-    if (p.n_split == 1) out = reinterpret_cast<__nv_bfloat16*>(p.out) + (static_cast<int64_t>(qi) * kH + row) * kDV + d0;
-    else pout = p.part_out + ((static_cast<int64_t>(qi) * p.n_split + split) * kH + row) * kDV + d0;
+    // The block's output is one contiguous piece of memory (64 rows of 512 bf16, or of 512 fp32 for a split).  A
+    // thread owns half a row, so direct stores would scatter 16-byte pieces over 32 rows per instruction; instead
+    // each warp lays its 16 rows out in the (now idle) key buffers, with a 16-byte pad per row against bank
+    // conflicts, and copies them out with consecutive lanes on consecutive 16-byte chunks.
+    const bool to_part = p.n_split != 1;
+    const int row_bytes = to_part ? kDV * 4 : kDV * 2;
+    const int pitch = row_bytes + 16;
+    uint8_t* stage = &sm.k[0][0][0];
+    uint8_t* my_stage = stage + row * pitch + hi * (row_bytes / 2);
 #pragma unroll 1
     for (int c = 0; c < 256; c += 64) {
       uint32_t o[64];
@@ -366,7 +441,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
 #pragma unroll
         for (int j = 0; j < 64; ++j) o[j] = 0u;
       }
-      if (out != nullptr) {
+      if (!to_part) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           uint4 w4;
@@ -374,14 +449,28 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
           w4.y = pack_bf16(__uint_as_float(o[8 * j + 2]) * inv, __uint_as_float(o[8 * j + 3]) * inv);
           w4.z = pack_bf16(__uint_as_float(o[8 * j + 4]) * inv, __uint_as_float(o[8 * j + 5]) * inv);
           w4.w = pack_bf16(__uint_as_float(o[8 * j + 6]) * inv, __uint_as_float(o[8 * j + 7]) * inv);
-          *reinterpret_cast<uint4*>(out + c + 8 * j) = w4;
+          *reinterpret_cast<uint4*>(my_stage + (c + 8 * j) * 2) = w4;
         }
       } else {
 #pragma unroll
         for (int j = 0; j < 16; ++j)
-          *reinterpret_cast<float4*>(pout + c + 4 * j) =
+          *reinterpret_cast<float4*>(my_stage + (c + 4 * j) * 4) =
               make_float4(__uint_as_float(o[4 * j]) * inv, __uint_as_float(o[4 * j + 1]) * inv,
                           __uint_as_float(o[4 * j + 2]) * inv, __uint_as_float(o[4 * j + 3]) * inv);
+      }
+    }
+    __syncwarp();
+    {
+      uint8_t* dst = to_part ? reinterpret_cast<uint8_t*>(p.part_out + (static_cast<int64_t>(qi) * p.n_split + split) * kH * kDV)
+                             : reinterpret_cast<uint8_t*>(reinterpret_cast<__nv_bfloat16*>(p.out) + static_cast<int64_t>(qi) * kH * kDV);
+      const int chunks_per_row = row_bytes >> 4;                 // 64 or 128
+      const int cshift = to_part ? 7 : 6;
+      const int n_chunks = 16 * chunks_per_row;                  // this warp's 16 rows
+#pragma unroll 4
+      for (int e = lane; e < n_chunks; e += 32) {
+        const int r = 16 * quarter + (e >> cshift), cc = e & (chunks_per_row - 1);
+        *reinterpret_cast<uint4*>(dst + static_cast<int64_t>(r) * row_bytes + cc * 16) =
+            *reinterpret_cast<const uint4*>(stage + r * pitch + cc * 16);
       }
     }
     if (hi == 0) {
@@ -395,6 +484,10 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
   }
   tc::fence_before_sync();
   __syncthreads();
+  if (tid == 0) {
+    LSA_TL(7);
+    LSA_WALL(1);
+  }
   if (warp == kSoftmaxWarps) tc::tmem_dealloc(tmem_base, kTmemColsAttn);
 }
 
