@@ -129,12 +129,14 @@ int* status_word(lsa_ctx* c) { return c->ws ? reinterpret_cast<int*>(c->ws) : nu
 
 // Number of row splits per sequence in paged (decode) attention.  Blocks run one per SM in waves; a block costs its
 // share of the 64-key units plus a fixed part (Q load, tensor-memory set-up, fp32 partial output), taken as six
-// units' worth.  The split count with the smallest estimate wins; ties go to fewer splits (less merging).
-int pick_split(int sm_count, int batch, int max_rows) {
+// units' worth.  The split count with the smallest estimate wins; ties go to fewer splits (less merging).  The
+// tcgen05 kernel merges its splits inside a thread-block cluster and takes only the counts that allows.
+int pick_split(int sm_count, int batch, int max_rows, bool tc_kernel) {
   const int units = (max_rows + 63) / 64;
   int best = 1;
   long best_cost = -1;
   for (int s = 1; s <= kMaxSplit && s <= units; ++s) {
+    if (tc_kernel && !lsa::attn_tc_split_ok(s)) continue;
     const long waves = (static_cast<long>(batch) * s + sm_count - 1) / sm_count;
     const long cost = waves * ((units + s - 1) / s + 6);
     if (best_cost < 0 || cost < best_cost) {
@@ -243,19 +245,20 @@ int run_attn(lsa_ctx* c, const lsa_params* p, const void* q, const void* k, cons
   a.rows_ld = p->k_sink + p->k_sparse + p->k_swa;
   a.q_pos0 = q_pos0; a.n_query = static_cast<int>(nq); a.ctx_len = ctx_len; a.out = out; a.lse = lse;
   a.n_split = 1; a.status = status_word(c);
+  const bool use_tc = c->tune[LSA_TUNE_ATTN_TC] && lsa::attn_tc_supported(a);
   if (p->paged) {
     const WsLayout l = ws_layout(p, nq, 0, batch);
     if (c->ws == nullptr || l.total > c->ws_bytes) return LSA_ERR_WORKSPACE;
-    a.n_split = c->tune[LSA_TUNE_ATTN_SPLIT] > 0 ? c->tune[LSA_TUNE_ATTN_SPLIT] : pick_split(c->sm_count, batch, a.rows_ld);
+    a.n_split = c->tune[LSA_TUNE_ATTN_SPLIT] > 0 ? c->tune[LSA_TUNE_ATTN_SPLIT] : pick_split(c->sm_count, batch, a.rows_ld, use_tc);
+    if (use_tc && !lsa::attn_tc_split_ok(a.n_split)) return LSA_ERR_ARG;
     a.part_out = reinterpret_cast<float*>(c->ws + l.part_out);
     a.part_lse = reinterpret_cast<float*>(c->ws + l.part_lse);
   }
   if (a.H == 64 && !(v == k && ld_v == ld_k)) return LSA_ERR_SHAPE;
   cudaError_t e = timed(c, LSA_K_ATTN, [&] {
-    return (c->tune[LSA_TUNE_ATTN_TC] && lsa::attn_tc_supported(a)) ? lsa::launch_attn_tc(a, c->stream, &c->launches)
-                                                                  : lsa::launch_attn(a, c->stream, &c->launches);
+    return use_tc ? lsa::launch_attn_tc(a, c->stream, &c->launches) : lsa::launch_attn(a, c->stream, &c->launches);
   });
-  if (e == cudaSuccess && a.n_split > 1) e = timed(c, LSA_K_MERGE, [&] { return lsa::launch_merge(a, c->stream, &c->launches); });
+  if (e == cudaSuccess && a.n_split > 1 && !use_tc) e = timed(c, LSA_K_MERGE, [&] { return lsa::launch_merge(a, c->stream, &c->launches); });
   return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
 }
 

@@ -23,6 +23,9 @@
 //                     lane l finishes keys 0-31 and lane l+16 keys 32-63 of the tile.
 //   columns 384-447   P buffers 0 and 1 (32 columns = 64 bf16 each), one copy per lane half, because an MMA reads
 //                     its TMEM operand from the lanes its accumulator lives in
+#include <cstdio>
+#include <cstdlib>
+
 #include "lsa_internal.h"
 #include "lsa_tc.cuh"
 
@@ -30,7 +33,7 @@
 // Debug build only (-DLSA_TIMELINE): per-block SM-clock stamps at the phase boundaries of the attention kernel,
 // read back with lsa_debug_timeline.  0 entry, 1 set-up done, 2 Q ready, 3 first key tile landed, 4 first S ready,
 // 5 last P handed over, 6 last P V done, 7 exit.
-__device__ long long g_timeline[1024 * 8];
+__device__ long long g_timeline[1024 * 16];
 __device__ long long g_wall[1024 * 2];   // globaltimer (ns) at entry and exit
 #define LSA_WALL(k)                                                                      \
   do {                                                                                   \
@@ -45,10 +48,10 @@ extern "C" __attribute__((visibility("default"))) int lsa_debug_wall(long long* 
 #define LSA_TL(k)                                                                        \
   do {                                                                                   \
     const unsigned blk_ = blockIdx.x + gridDim.x * blockIdx.y;                           \
-    if (blk_ < 1024) g_timeline[blk_ * 8 + (k)] = clock64();                             \
+    if (blk_ < 1024) g_timeline[blk_ * 16 + (k)] = clock64();                             \
   } while (0)
 extern "C" __attribute__((visibility("default"))) int lsa_debug_timeline(long long* host, int n_blocks) {
-  return cudaMemcpyFromSymbol(host, g_timeline, sizeof(long long) * 8 * (n_blocks < 1024 ? n_blocks : 1024)) == cudaSuccess ? 0 : -1;
+  return cudaMemcpyFromSymbol(host, g_timeline, sizeof(long long) * 16 * (n_blocks < 1024 ? n_blocks : 1024)) == cudaSuccess ? 0 : -1;
 }
 #else
 #define LSA_TL(k)
@@ -73,6 +76,7 @@ constexpr uint32_t kColQ = 256;              // Q[:, 0:512] as packed bf16: 128 
 constexpr uint32_t kColS = 384;              // two S / P buffers of 64 columns
 constexpr uint32_t kSBuf = 64;
 constexpr float kLog2eTc = 1.4426950408889634f;
+constexpr int kMaxClusterSplit = 8;          // row splits of one sequence = blocks of one cluster (portable limit)
 constexpr float kRescaleGap = 8.f;           // rescale O only when the row max grows by more than 2^8
 
 struct AttnTcSmem {
@@ -80,42 +84,29 @@ struct AttnTcSmem {
   alignas(1024) uint8_t k[kKBufs][kAtoms][kAtomBytes];      // [tile buffer][column block][64 rows x 128 B]
   alignas(8) uint64_t q_full, q_tmem, k_full[kKBufs], k_empty[kKBufs], s_full[2], p_ready[2], pv_done[2];
   uint32_t tmem_slot;
+  float lse_own[kH];              // split launches: this block's log-sum-exp per head (log2 units)
 };
 
+// ---- thread-block cluster: barrier and loads from a peer block's shared memory
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// With n_split > 1 the kernel must be launched with clusters of (1, n_split, 1) blocks: the splits of one sequence
+// are co-scheduled and merge their partial results themselves (no second kernel).  Block s finishes heads
+// [s * 64 / n_split, (s + 1) * 64 / n_split): every block keeps its own share of the rows in shared memory and writes
+// the other rows (normalised, fp32) and all its log-sum-exps to the global scratch, where they stay in L2; after one
+// cluster barrier the owner of a row combines its own part with the others'.  (Distributed shared memory moved the
+// same rows at about a quarter of the L2 path's rate, so it carries nothing here.)
 __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnArgs p) {
   extern __shared__ uint8_t smem_raw[];
   AttnTcSmem& sm = *reinterpret_cast<AttnTcSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int qi = blockIdx.x, split = blockIdx.y;
 
-  // ---- this query's row list (same conventions as the mma.sync kernel)
-  const int64_t t = p.paged ? static_cast<int64_t>(p.ctx_len[qi]) - 1 : p.q_pos0 + qi;
-  int n_sink = 0, n_sp = 0, n_tot;
-  int64_t win0 = 0;
-  const int32_t* rows = nullptr;
-  if (p.rows != nullptr) {
-    rows = p.rows + static_cast<int64_t>(qi) * p.rows_ld;
-    n_tot = p.n_rows[qi];
-  } else {
-    n_sink = static_cast<int>(min64(p.S, t + 1));
-    win0 = max64(p.S, t - p.W + 1);
-    n_sp = p.n_sparse[qi];
-    n_tot = n_sink + n_sp + static_cast<int>(max64(0, t - win0 + 1));
-  }
-  const int32_t* sp = p.sparse_idx ? p.sparse_idx + static_cast<int64_t>(qi) * p.Ksp : nullptr;
-  auto row_of = [&](int i) -> int32_t {
-    if (i >= n_tot) return -1;
-    if (rows) return rows[i];
-    if (i < n_sink) return i;
-    if (i < n_sink + n_sp) return sp[i - n_sink];
-    return static_cast<int32_t>(win0 + (i - n_sink - n_sp));
-  };
-  const int tiles_all = (n_tot + kTileKeys - 1) / kTileKeys;
-  const int tiles_per = (tiles_all + p.n_split - 1) / p.n_split;
-  const int tile_begin = split * tiles_per;
-  const int n_tiles = max(0, min(tiles_all, tile_begin + tiles_per) - tile_begin);
-
-  if (tc::status_raised(p.status)) return;   // an earlier block of this launch gave up on a wait
+  const bool clustered = p.n_split > 1;
+  const bool dead = tc::status_raised(p.status);   // an earlier block of this launch (or an earlier launch) gave up on a wait
+  if (dead && !clustered) return;
 
   // ---- set-up
   if (tid == 0) {
@@ -143,6 +134,38 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
   tc::fence_after_sync();
   const uint32_t tmem_base = sm.tmem_slot;
   if (tid == 0) LSA_TL(1);
+  // Programmatic dependent launch: this block may have been placed while the previous kernel of the stream was still
+  // draining; what earlier kernels wrote is read only from here on.  The next kernel's blocks may be placed from now.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+  // ---- this query's row list (same conventions as the mma.sync kernel)
+  const int64_t t = p.paged ? static_cast<int64_t>(p.ctx_len[qi]) - 1 : p.q_pos0 + qi;
+  int n_sink = 0, n_sp = 0, n_tot;
+  int64_t win0 = 0;
+  const int32_t* rows = nullptr;
+  if (p.rows != nullptr) {
+    rows = p.rows + static_cast<int64_t>(qi) * p.rows_ld;
+    n_tot = p.n_rows[qi];
+  } else {
+    n_sink = static_cast<int>(min64(p.S, t + 1));
+    win0 = max64(p.S, t - p.W + 1);
+    n_sp = p.n_sparse[qi];
+    n_tot = n_sink + n_sp + static_cast<int>(max64(0, t - win0 + 1));
+  }
+  const int32_t* sp = p.sparse_idx ? p.sparse_idx + static_cast<int64_t>(qi) * p.Ksp : nullptr;
+  auto row_of = [&](int i) -> int32_t {
+    if (i >= n_tot) return -1;
+    if (rows) return rows[i];
+    if (i < n_sink) return i;
+    if (i < n_sink + n_sp) return sp[i - n_sink];
+    return static_cast<int32_t>(win0 + (i - n_sink - n_sp));
+  };
+  const int tiles_all = (n_tot + kTileKeys - 1) / kTileKeys;
+  const int tiles_per = (tiles_all + p.n_split - 1) / p.n_split;
+  const int tile_begin = split * tiles_per;
+  int n_tiles = max(0, min(tiles_all, tile_begin + tiles_per) - tile_begin);
+  if (dead) n_tiles = 0;   // the peers of this cluster still expect this block at the cluster barrier
 
   if (warp >= kSoftmaxWarps + kMmaWarps) {
     // ================= gather warps =================
@@ -196,6 +219,9 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       const int b = i % kKBufs;
       const uint32_t par = ((i / kKBufs) & 1) ^ 1;
       const int32_t next_row = my_key_row(i + 1);   // fetched before the wait: off the critical path
+      // Q and the first tile go out alone: requested together with the next tiles they would share the memory pipe
+      // with them and the first Q K^T would start two tiles' worth of traffic later
+      if (i == 1) while (n_pend > 0) hand_over_oldest();
       if (i == kKBufs - 1) {
         // first use of the buffer that staged Q: the softmax warps must have moved Q to tensor memory
         while (n_pend > 0 && !__all_sync(0xffffffffu, tc::mbar_test(smem_u32(&sm.q_tmem), 0))) hand_over_oldest();
@@ -422,26 +448,25 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     tc::fence_after_sync();
     if (tid == 0) LSA_TL(6);
     const float inv = (have_o && l_row > 0.f) ? 1.f / l_row : 0.f;
-    // The block's output is one contiguous piece of memory (64 rows of 512 bf16, or of 512 fp32 for a split).  A
-    // thread owns half a row, so direct stores would scatter 16-byte pieces over 32 rows per instruction; instead
-    // each warp lays its 16 rows out in the (now idle) key buffers, with a 16-byte pad per row against bank
-    // conflicts, and copies them out with consecutive lanes on consecutive 16-byte chunks.
-    const bool to_part = p.n_split != 1;
-    const int row_bytes = to_part ? kDV * 4 : kDV * 2;
-    const int pitch = row_bytes + 16;
+    const float lse2 = (have_o && l_row > 0.f) ? m_row + log2f(l_row) : -INFINITY;   // log2 domain
     uint8_t* stage = &sm.k[0][0][0];
-    uint8_t* my_stage = stage + row * pitch + hi * (row_bytes / 2);
+    if (!clustered) {
+      // The block's output is one contiguous piece of memory (64 rows of 512 bf16).  A thread owns half a row, so
+      // direct stores would scatter 16-byte pieces over 32 rows per instruction; instead each warp lays its 16 rows
+      // out in the (now idle) key buffers, with a 16-byte pad per row against bank conflicts, and copies them out
+      // with consecutive lanes on consecutive 16-byte chunks.
+      constexpr int kRowBytes = kDV * 2, kPitch = kRowBytes + 16;
+      uint8_t* my_stage = stage + row * kPitch + hi * (kRowBytes / 2);
 #pragma unroll 1
-    for (int c = 0; c < 256; c += 64) {
-      uint32_t o[64];
-      if (have_o) {
-        tc::tmem_ld64(tmem_base + lane_addr + c, o);
-        tc::tmem_ld_wait();
-      } else {
+      for (int c = 0; c < 256; c += 64) {
+        uint32_t o[64];
+        if (have_o) {
+          tc::tmem_ld64(tmem_base + lane_addr + c, o);
+          tc::tmem_ld_wait();
+        } else {
 #pragma unroll
-        for (int j = 0; j < 64; ++j) o[j] = 0u;
-      }
-      if (!to_part) {
+          for (int j = 0; j < 64; ++j) o[j] = 0u;
+        }
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           uint4 w4;
@@ -451,47 +476,158 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
           w4.w = pack_bf16(__uint_as_float(o[8 * j + 6]) * inv, __uint_as_float(o[8 * j + 7]) * inv);
           *reinterpret_cast<uint4*>(my_stage + (c + 8 * j) * 2) = w4;
         }
-      } else {
+      }
+      __syncwarp();
+      uint8_t* dst = reinterpret_cast<uint8_t*>(reinterpret_cast<__nv_bfloat16*>(p.out) + static_cast<int64_t>(qi) * kH * kDV);
+      constexpr int kChunksPerRow = kRowBytes / 16;
+#pragma unroll 4
+      for (int e = lane; e < 16 * kChunksPerRow; e += 32) {   // this warp's 16 rows
+        const int r = 16 * quarter + e / kChunksPerRow, cc = e % kChunksPerRow;
+        *reinterpret_cast<uint4*>(dst + static_cast<int64_t>(r) * kRowBytes + cc * 16) =
+            *reinterpret_cast<const uint4*>(stage + r * kPitch + cc * 16);
+      }
+      if (hi == 0 && p.lse != nullptr) p.lse[static_cast<int64_t>(qi) * kH + row] = lse2 / kLog2eTc;
+    } else {
+      // partial result of a split: normalised fp32 rows in the key buffers (padded against bank conflicts)
+      constexpr int kPitchPart = kDV * 4 + 16;
+      uint8_t* my_stage = stage + row * kPitchPart + hi * (kDV * 2);
+#pragma unroll 1
+      for (int c = 0; c < 256; c += 64) {
+        uint32_t o[64];
+        if (have_o) {
+          tc::tmem_ld64(tmem_base + lane_addr + c, o);
+          tc::tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 64; ++j) o[j] = 0u;
+        }
 #pragma unroll
         for (int j = 0; j < 16; ++j)
           *reinterpret_cast<float4*>(my_stage + (c + 4 * j) * 4) =
               make_float4(__uint_as_float(o[4 * j]) * inv, __uint_as_float(o[4 * j + 1]) * inv,
                           __uint_as_float(o[4 * j + 2]) * inv, __uint_as_float(o[4 * j + 3]) * inv);
       }
-    }
-    __syncwarp();
-    {
-      uint8_t* dst = to_part ? reinterpret_cast<uint8_t*>(p.part_out + (static_cast<int64_t>(qi) * p.n_split + split) * kH * kDV)
-                             : reinterpret_cast<uint8_t*>(reinterpret_cast<__nv_bfloat16*>(p.out) + static_cast<int64_t>(qi) * kH * kDV);
-      const int chunks_per_row = row_bytes >> 4;                 // 64 or 128
-      const int cshift = to_part ? 7 : 6;
-      const int n_chunks = 16 * chunks_per_row;                  // this warp's 16 rows
-#pragma unroll 4
-      for (int e = lane; e < n_chunks; e += 32) {
-        const int r = 16 * quarter + (e >> cshift), cc = e & (chunks_per_row - 1);
-        *reinterpret_cast<uint4*>(dst + static_cast<int64_t>(r) * row_bytes + cc * 16) =
-            *reinterpret_cast<const uint4*>(stage + r * pitch + cc * 16);
-      }
-    }
-    if (hi == 0) {
-      const float lse2 = (have_o && l_row > 0.f) ? m_row + log2f(l_row) : -INFINITY;   // log2 domain
-      if (p.n_split == 1) {
-        if (p.lse != nullptr) p.lse[static_cast<int64_t>(qi) * kH + row] = lse2 / kLog2eTc;
-      } else {
+      if (hi == 0) {
+        sm.lse_own[row] = lse2;
         p.part_lse[(static_cast<int64_t>(qi) * p.n_split + split) * kH + row] = lse2;
       }
     }
   }
+  if (tid == 0) LSA_TL(8);
   tc::fence_before_sync();
   __syncthreads();
+  if (tid == 0) LSA_TL(9);
+  if (warp == kSoftmaxWarps) tc::tmem_dealloc(tmem_base, kTmemColsAttn);
+  if (clustered) {
+    // ---- merge of the splits (Sec. 4.1.1: online-softmax rescaling) for this block's heads: weights
+    // 2^(lse_j - max) / sum, O = sum_j w_j O_j, bf16 to global.
+    const int n = p.n_split;
+    const int rows_per = kH / n;
+    const int row0 = split * rows_per;
+    constexpr int kPitchPart = kDV * 4 + 16;
+    constexpr int kRowChunks = kDV / 4;   // 16-byte chunks of an fp32 row
+    const uint8_t* stage = &sm.k[0][0][0];
+    // rows owned by the other blocks -> global scratch, consecutive threads on consecutive chunks
+    float* mine = p.part_out + (static_cast<int64_t>(qi) * n + split) * kH * kDV;
+    for (int e = tid; e < (kH - rows_per) * kRowChunks; e += kThreadsAttnTc) {
+      const int fr = e / kRowChunks, cc = e % kRowChunks;
+      const int r = fr < row0 ? fr : fr + rows_per;
+      *reinterpret_cast<float4*>(mine + r * kDV + cc * 4) = *reinterpret_cast<const float4*>(stage + r * kPitchPart + cc * 16);
+    }
+    __threadfence();
+    if (tid == 0) LSA_TL(10);
+    cluster_sync_all();   // every block of the cluster has written its rows
+    if (tid == 0) LSA_TL(11);
+    // Warp w finishes rows w, w + 12, ... of this block's share (at most three).  Lane 8k + j first fetches the
+    // log-sum-exp of split j for the warp's k-th row, so that all of them are in flight together.
+    constexpr int kWarps = kThreadsAttnTc / 32;
+    const int k_of = lane >> 3, j_of = lane & 7;
+    const int rl_mine = warp + kWarps * k_of;
+    float my_l = -INFINITY;
+    if (k_of < 3 && rl_mine < rows_per && j_of < n)
+      my_l = j_of == split ? sm.lse_own[row0 + rl_mine]
+                           : __ldcg(p.part_lse + (static_cast<int64_t>(qi) * n + j_of) * kH + row0 + rl_mine);
+    float m = my_l;
+#pragma unroll
+    for (int d = 1; d < 8; d <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+    float wgt = m > -INFINITY ? exp2f(my_l - m) : 0.f;
+    float den = wgt;
+#pragma unroll
+    for (int d = 1; d < 8; d <<= 1) den += __shfl_xor_sync(0xffffffffu, den, d);
+    wgt = den > 0.f ? wgt / den : 0.f;
+    if (p.lse != nullptr && j_of == 0 && k_of < 3 && rl_mine < rows_per)
+      p.lse[static_cast<int64_t>(qi) * kH + row0 + rl_mine] = den > 0.f ? (m + log2f(den)) / kLog2eTc : -INFINITY;
+    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + (static_cast<int64_t>(qi) * kH + row0) * kDV;
+    for (int k = 0; k < 3; ++k) {
+      const int rl = warp + kWarps * k;   // warp-uniform
+      if (rl >= rows_per) break;
+      float4 acc[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int j = 0; j < n; ++j) {
+        const float w = __shfl_sync(0xffffffffu, wgt, 8 * k + j);
+        float4 v[4];
+        if (j == split) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const float4*>(stage + (row0 + rl) * kPitchPart + (lane + 32 * u) * 16);
+        } else {
+          const float4* src = reinterpret_cast<const float4*>(p.part_out + ((static_cast<int64_t>(qi) * n + j) * kH + row0 + rl) * kDV);
+#pragma unroll
+          for (int u = 0; u < 4; ++u) v[u] = __ldcg(src + lane + 32 * u);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          acc[u].x += w * v[u].x; acc[u].y += w * v[u].y; acc[u].z += w * v[u].z; acc[u].w += w * v[u].w;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        uint2 o;
+        o.x = pack_bf16(acc[u].x, acc[u].y);
+        o.y = pack_bf16(acc[u].z, acc[u].w);
+        *reinterpret_cast<uint2*>(out + static_cast<int64_t>(rl) * kDV + (lane + 32 * u) * 4) = o;
+      }
+    }
+    if (tid == 0) LSA_TL(12);
+  }
   if (tid == 0) {
     LSA_TL(7);
     LSA_WALL(1);
   }
-  if (warp == kSoftmaxWarps) tc::tmem_dealloc(tmem_base, kTmemColsAttn);
 }
 
 }  // namespace
+
+// Largest cluster of full-SM blocks of this kernel the device can place (queried once per process).
+static_assert(sizeof(AttnTcSmem) + 1024 <= 227 * 1024, "shared memory of the attention kernel exceeds one SM");
+
+static int max_cluster_blocks() {
+  static const int n = [] {
+    const size_t smem = sizeof(AttnTcSmem) + 1024;
+    if (cudaFuncSetAttribute(sparse_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) return 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(1, kMaxClusterSplit);
+    cfg.blockDim = dim3(kThreadsAttnTc);
+    cfg.dynamicSmemBytes = smem;
+    int size = 0;
+    const cudaError_t eq = cudaOccupancyMaxPotentialClusterSize(&size, sparse_attn_tc_kernel, &cfg);
+    if (eq != cudaSuccess) {
+      if (getenv("LSA_DEBUG")) fprintf(stderr, "[lsa] cluster size query failed: %s\n", cudaGetErrorString(eq));
+      (void)cudaGetLastError();
+      return 1;
+    }
+    if (getenv("LSA_DEBUG")) fprintf(stderr, "[lsa] attention kernel: max cluster size %d\n", size);
+    return size < 1 ? 1 : size;
+  }();
+  return n;
+}
+
+// Row splits the tcgen05 kernel can merge inside a cluster: a power of two that divides the 64 heads, at most 8 blocks
+// and at most what the device can co-schedule.
+bool attn_tc_split_ok(int n_split) {
+  if (n_split == 1) return true;
+  return (n_split == 2 || n_split == 4 || n_split == 8) && n_split <= max_cluster_blocks();
+}
 
 bool attn_tc_supported(const AttnArgs& a) {
   return a.H == kH && a.DQK == kDQK && a.DV == kDV && a.v == a.k && a.ld_v == a.ld_k;
@@ -502,7 +638,30 @@ cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t st, int64_t* n_launch
   const size_t smem = sizeof(AttnTcSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(sparse_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
-  sparse_attn_tc_kernel<<<dim3(a.n_query, a.n_split), kThreadsAttnTc, smem, st>>>(a);
+  if (a.n_split <= 1) {
+    sparse_attn_tc_kernel<<<dim3(a.n_query, 1), kThreadsAttnTc, smem, st>>>(a);
+  } else {
+    if (!attn_tc_split_ok(a.n_split)) return cudaErrorInvalidValue;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(a.n_query, a.n_split);
+    cfg.blockDim = dim3(kThreadsAttnTc);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2]{};
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = static_cast<unsigned>(a.n_split);
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see griddepcontrol.wait in the kernel
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    e = cudaLaunchKernelEx(&cfg, sparse_attn_tc_kernel, a);
+    if (e != cudaSuccess) {
+      if (getenv("LSA_DEBUG")) fprintf(stderr, "[lsa] cluster launch (%d x %d blocks) failed: %s\n", a.n_query, a.n_split, cudaGetErrorString(e));
+      return e;
+    }
+  }
   ++*n_launch;
   return cudaGetLastError();
 }

@@ -79,6 +79,8 @@ cudaError_t launch_convert(int S, int W, int Ksp, int paged, int kv_page, const 
 cudaError_t launch_attn(const AttnArgs& a, cudaStream_t st, int64_t* n_launch);
 // tcgen05 version of the attention kernel (MLA latent shape only)
 bool attn_tc_supported(const AttnArgs& a);
+// row splits that kernel merges itself (clusters of n_split blocks); other counts need launch_merge
+bool attn_tc_split_ok(int n_split);
 cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t st, int64_t* n_launch);
 cudaError_t launch_merge(const AttnArgs& a, cudaStream_t st, int64_t* n_launch);
 

@@ -178,6 +178,32 @@ def test_small_paged_decode(cuda_device):
     m.assert_ok(pu.TOL_FP8)
 
 
+@pytest.mark.parametrize("n_split", [1, 2, 4, 8])
+def test_paged_decode_row_splits(cuda_device, n_split):
+    """Each row-split count of the decode attention (blocks of one thread-block cluster merging their parts by
+    log-sum-exp) matches the oracle; the split is a launch shape, not part of the result's definition."""
+    cfg = SMALL_DEC
+    wl = DecodeWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.ctx.tune(2, n_split)          # LSA_TUNE_ATTN_SPLIT
+    wl.step()
+    assert wl.ctx.status() == 0
+    m = pu.check_decode(wl, range(cfg.batch))
+    print(cfg.name, n_split, m.summary())
+    m.assert_ok(pu.TOL_FP8)
+
+
+def test_decode_split_count_is_checked(cuda_device):
+    cfg = SMALL_DEC
+    if cfg.H != 64:
+        pytest.skip("cluster splits belong to the 64-head kernel")
+    wl = DecodeWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.ctx.tune(2, 3)                # three blocks do not divide the 64 heads evenly
+    with pytest.raises(binding.LsaError):
+        wl.step()
+
+
 def test_convert_lists_physical_rows(cuda_device):
     cfg = SMALL_DEC
     wl = DecodeWorkload(cfg, cuda_device)
