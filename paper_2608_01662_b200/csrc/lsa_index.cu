@@ -238,20 +238,22 @@ __global__ void __launch_bounds__(kThreads) coarse_score_kernel(IndexArgs p) {
 }
 
 // Paged (decode) form of a1: one query per sequence, so a block keeps the query resident and streams several
-// mean-key tiles of that sequence through a double buffer (the mean cache is the large operand here: the stage
-// is an HBM read of the whole cache of means).
+// mean-key tiles of that sequence through a three-deep ring (the mean cache is the large operand here: the stage
+// is an HBM read of the whole cache of means, and a tile costs a page-table look-up plus an HBM round trip, so two
+// blocks per SM with two tiles each in flight are what keeps the memory pipe full).
 constexpr int kCoarseTilesPerBlock = 8;
+constexpr int kCoarseStages = 3;
 
 template <int HI, int DI>
 struct CoarsePagedSmem {
-  alignas(128) uint8_t a[2][kTileRows * DI * 2];
+  alignas(128) uint8_t a[kCoarseStages][kTileRows * DI * 2];
   alignas(128) uint8_t q[HI * DI * 2];
   float w[HI];
   float sub[kTileRows];
 };
 
 template <int HI, int DI>
-__global__ void __launch_bounds__(kThreads) coarse_score_paged_kernel(IndexArgs p) {
+__global__ void __launch_bounds__(kThreads, 2) coarse_score_paged_kernel(IndexArgs p) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   auto& sm = *reinterpret_cast<CoarsePagedSmem<HI, DI>*>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -290,15 +292,17 @@ __global__ void __launch_bounds__(kThreads) coarse_score_paged_kernel(IndexArgs 
   };
   load_q_async<HI, DI>(smem_u32(sm.q), reinterpret_cast<const __nv_bfloat16*>(p.q_idx) + static_cast<int64_t>(qi) * HI * DI);
   if (tid < HI / 4) cp_async16(smem_u32(&sm.w[tid * 4]), p.w + static_cast<int64_t>(qi) * HI + tid * 4, 16);
-  issue_tile(tile_begin, 0);
+  // one cp.async group per tile, also when there is no tile left (an empty group), so the wait depth is constant
+  for (int j = 0; j < kCoarseStages - 1; ++j) {
+    if (tile_begin + j < tile_end) issue_tile(tile_begin + j, j);
+    else cp_async_commit();
+  }
   for (int tile = tile_begin; tile < tile_end; ++tile) {
-    const int buf = (tile - tile_begin) & 1;
-    if (tile + 1 < tile_end) {
-      issue_tile(tile + 1, buf ^ 1);
-      cp_async_wait<1>();
-    } else {
-      cp_async_wait<0>();
-    }
+    const int buf = (tile - tile_begin) % kCoarseStages;
+    // the buffer refilled here was read two iterations ago; the barrier that ended that iteration covers it
+    if (tile + kCoarseStages - 1 < tile_end) issue_tile(tile + kCoarseStages - 1, (buf + kCoarseStages - 1) % kCoarseStages);
+    else cp_async_commit();
+    cp_async_wait<kCoarseStages - 1>();
     __syncthreads();   // tile (and, first time, q / w) in shared
     uint32_t a[DI / 16][4];
     load_a_frags<DI>(a, smem_u32(sm.a[buf]));
@@ -571,7 +575,9 @@ __global__ void widen_e4m3_kernel(const uint4* __restrict__ codes, uint4* __rest
 // ------------------------------------------------------------------------------------------------
 // a5: index set -> cache rows  [sink run | sparse ascending | window run]
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128) convert_kernel(int S, int W, int Ksp, int paged, int kv_page,
+constexpr int kConvertThreads = 1024;   // every row of a query has its own thread or nearly: the look-ups are two dependent loads
+
+__global__ void __launch_bounds__(kConvertThreads) convert_kernel(int S, int W, int Ksp, int paged, int kv_page,
                                                      const int32_t* __restrict__ sparse_idx,
                                                      const int32_t* __restrict__ n_sparse, int64_t q_pos0,
                                                      const int32_t* __restrict__ page_table, int64_t pt_stride,
@@ -597,26 +603,29 @@ __global__ void __launch_bounds__(128) convert_kernel(int S, int W, int Ksp, int
     return static_cast<int32_t>(paged ? (static_cast<int64_t>(pt[pos >> kv_shift]) << kv_shift) + (pos & (kv_page - 1)) : pos);
   };
   int breaks = 0;
-  for (int i = tid; i < ld; i += 128) {
+#pragma unroll 4
+  for (int i = tid; i < ld; i += kConvertThreads) {
     int32_t r = -1;
     if (i < n_tot) {
       r = row_of(i);
-      if (i == 0 || row_of(i - 1) + 1 != r) ++breaks;
+      if (runs_out != nullptr && (i == 0 || row_of(i - 1) + 1 != r)) ++breaks;
     }
     out[i] = r;
   }
   if (tid == 0) n_rows_out[qi] = n_tot;
   if (runs_out != nullptr) {
-    __shared__ int sh[4];
+    __shared__ int sh[kConvertThreads / 32];
     breaks = __reduce_add_sync(0xffffffffu, breaks);
     if ((tid & 31) == 0) sh[tid >> 5] = breaks;
     __syncthreads();
     if (tid == 0) {
+      int total = 0;
+      for (int i = 0; i < kConvertThreads / 32; ++i) total += sh[i];
       int32_t* ro = runs_out + static_cast<int64_t>(qi) * 4;
       ro[0] = n_sink;
       ro[1] = n_sp;
       ro[2] = n_win;
-      ro[3] = sh[0] + sh[1] + sh[2] + sh[3];
+      ro[3] = total;
     }
   }
 }
@@ -674,6 +683,7 @@ static cudaError_t launch_coarse_t(const IndexArgs& a, int64_t n_key_max, cudaSt
 cudaError_t launch_coarse(const IndexArgs& a, cudaStream_t st, int64_t* n_launch) {
   // key tiles that any query can need: up to the largest cached length
   const int64_t n_key_max = a.paged ? a.pt_stride * a.P : a.n_key;
+  if (coarse_paged_tc_supported(a)) return launch_coarse_paged_tc(a, st, n_launch);
   if (a.HI == 8 && a.DI == 64) return launch_coarse_t<8, 64>(a, n_key_max, st, n_launch);
   return launch_coarse_t<64, 128>(a, n_key_max, st, n_launch);
 }
@@ -731,7 +741,7 @@ cudaError_t launch_convert(int S, int W, int Ksp, int paged, int kv_page, const 
                            int64_t pt_stride, const int32_t* ctx_len, int32_t* rows_out, int32_t* n_rows_out,
                            int32_t* runs_out, cudaStream_t st, int64_t* n_launch) {
   if (n_query == 0) return cudaSuccess;
-  convert_kernel<<<n_query, 128, 0, st>>>(S, W, Ksp, paged, kv_page, sparse_idx, n_sparse, q_pos0, page_table,
+  convert_kernel<<<n_query, kConvertThreads, 0, st>>>(S, W, Ksp, paged, kv_page, sparse_idx, n_sparse, q_pos0, page_table,
                                           pt_stride, ctx_len, rows_out, n_rows_out, runs_out);
   ++*n_launch;
   return cudaGetLastError();

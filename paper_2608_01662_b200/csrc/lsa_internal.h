@@ -64,6 +64,9 @@ cudaError_t launch_coarse(const IndexArgs& a, cudaStream_t st, int64_t* n_launch
 // tcgen05 version of the coarse stage (contiguous caches, H_I = 64, d_I = 128); groups = 4-query groups per block
 bool coarse_tc_supported(const IndexArgs& a);
 cudaError_t launch_coarse_tc(const IndexArgs& a, int groups, cudaStream_t st, int64_t* n_launch);
+// tcgen05 version of the coarse stage for paged caches (H_I = 64, d_I = 128); used by launch_coarse
+bool coarse_paged_tc_supported(const IndexArgs& a);
+cudaError_t launch_coarse_paged_tc(const IndexArgs& a, cudaStream_t st, int64_t* n_launch);
 cudaError_t launch_fine_select(const IndexArgs& a, cudaStream_t st, int64_t* n_launch);
 // tcgen05 version of the fine stage's scoring blocks (H_I = 64, d_I = 128); used by launch_fine_select
 bool fine_tc_supported(const IndexArgs& a);
