@@ -99,6 +99,27 @@ def block_means(k_hat, B, round_bf16=True):
     return bf16_round(km) if round_bf16 else km
 
 
+def block_minmax(k_hat, B, round_bf16=True):
+    """Per-dimension extrema of the keys of each sub-block (pooling variant of Sec. 5 "Pooling method", Eq. 13):
+    k_max[n, d] = max_{s in sub-block n} k[s, d],  k_min[n, d] = min likewise.
+
+    A trailing partial sub-block takes the extrema of the tokens present.  Returns (k_max, k_min), each
+    [ceil(n_key/B), d]; the cache stores bf16 (an extremum is one of the key values, rounded once).
+    """
+    k_hat = np.asarray(k_hat, dtype=np.float64)
+    n_key, d = k_hat.shape
+    n_sub = -(-n_key // B)
+    kmax = np.zeros((n_sub, d), dtype=np.float64)
+    kmin = np.zeros((n_sub, d), dtype=np.float64)
+    for n in range(n_sub):
+        blk = k_hat[n * B:min((n + 1) * B, n_key)]
+        kmax[n] = blk.max(axis=0)
+        kmin[n] = blk.min(axis=0)
+    if round_bf16:
+        return bf16_round(kmax), bf16_round(kmin)
+    return kmax, kmin
+
+
 # ----------------------------------------------------------------------------
 # scores
 # ----------------------------------------------------------------------------
@@ -129,6 +150,32 @@ def page_scores(q_I, w, km, P, B, pages):
         blk = km[p * spp:min((p + 1) * spp, km.shape[0])]
         # sum over sub-blocks of the per-sub-block Eq.-1-style score
         out[i] = indexer_scores(q_I, w, blk).sum()
+    return out
+
+
+def page_scores_minmax(q_I, w, kmax, kmin, P, B, pages):
+    """Eq. 13 in place of the mean-pooled dot product of Eq. 9: for sub-block n and head j
+
+        s~[n, j] = sum_d max(q_I[j, d] * k_max[n, d], q_I[j, d] * k_min[n, d]),
+
+    an upper bound of every token score q_I[j] . k[s] inside the sub-block, and
+    I_page[p] = sum_j w[j] * sum_{n in page p} ReLU(s~[n, j]).  (The paper's inner sum runs to "N"; it is the
+    sum over the sub-blocks of the page, as in Eq. 9.)  Returns one score per entry of `pages`.
+    """
+    q_I = np.asarray(q_I, dtype=np.float64)
+    w = np.asarray(w, dtype=np.float64)
+    kmax = np.asarray(kmax, dtype=np.float64)
+    kmin = np.asarray(kmin, dtype=np.float64)
+    spp = P // B
+    out = np.zeros(len(pages), dtype=np.float64)
+    for i, p in enumerate(pages):
+        lo, hi = p * spp, min((p + 1) * spp, kmax.shape[0])
+        total = 0.0
+        for n in range(lo, hi):
+            # [H_I, d]: the larger of the two products, dimension by dimension
+            s_tilde = np.maximum(q_I * kmax[n][None, :], q_I * kmin[n][None, :]).sum(axis=1)
+            total += float((w * np.maximum(s_tilde, 0.0)).sum())
+        out[i] = total
     return out
 
 
@@ -169,7 +216,7 @@ def eligible_pages(t, S, W, P):
     return np.arange(lo // P, hi // P + 1, dtype=np.int64)
 
 
-def select_sparse(t, q_I, w, k_hat, km, *, P, B, M, Ksp, S, W, hi_enable=True):
+def select_sparse(t, q_I, w, k_hat, km, *, P, B, M, Ksp, S, W, hi_enable=True, minmax=None):
     """S_sparse of query t (absolute position) and the recalled pages.
 
     Stage 1 (Eq. 9-10): if more than M pages are eligible, keep the M with the
@@ -178,7 +225,8 @@ def select_sparse(t, q_I, w, k_hat, km, *, P, B, M, Ksp, S, W, hi_enable=True):
     when at most M pages are eligible, every eligible page is kept, which is
     the flat selection of Eq. 7.
 
-    k_hat [n_key, d_I] real key values, km [ceil(n_key/B), d_I] mean cache.
+    k_hat [n_key, d_I] real key values, km [ceil(n_key/B), d_I] mean cache.  minmax = (k_max, k_min) switches
+    stage 1 to the MinMax pooling of Eq. 13 (km is then unused).
     Returns (sparse positions ascending, kept pages ascending).
     """
     lo, hi = candidate_range(t, S, W)
@@ -186,7 +234,10 @@ def select_sparse(t, q_I, w, k_hat, km, *, P, B, M, Ksp, S, W, hi_enable=True):
     if E.size == 0:
         return np.zeros(0, dtype=np.int64), E
     if hi_enable and E.size > M:
-        pages = top_k(page_scores(q_I, w, km, P, B, E), E, M)
+        if minmax is not None:
+            pages = top_k(page_scores_minmax(q_I, w, minmax[0], minmax[1], P, B, E), E, M)
+        else:
+            pages = top_k(page_scores(q_I, w, km, P, B, E), E, M)
     else:
         pages = E
     cand = np.concatenate([np.arange(max(lo, p * P), min(hi, p * P + P - 1) + 1, dtype=np.int64)

@@ -25,13 +25,23 @@ class HostCaches:
         else:
             self.k_hat = k_idx.astype(np.float64)
         self.km = orc.block_means(self.k_hat, B)
+        self.B = B
+        self._minmax = None
         self.k = [logical(k).astype(np.float64) for k in k_layers]
         self.v = [logical(v).astype(np.float64) for v in v_layers]
 
 
-def select_query(t, q_I, w, caches: HostCaches, *, P, B, M, Ksp, S, W, hi_enable=True):
+    def minmax(self):
+        """(k_max, k_min) caches of Eq. 13, built on first use."""
+        if self._minmax is None:
+            self._minmax = orc.block_minmax(self.k_hat, self.B)
+        return self._minmax
+
+
+def select_query(t, q_I, w, caches: HostCaches, *, P, B, M, Ksp, S, W, hi_enable=True, pooling="mean"):
     return orc.select_sparse(t, np.asarray(q_I, dtype=np.float64), np.asarray(w, dtype=np.float64), caches.k_hat,
-                             caches.km, P=P, B=B, M=M, Ksp=Ksp, S=S, W=W, hi_enable=hi_enable)
+                             caches.km, P=P, B=B, M=M, Ksp=Ksp, S=S, W=W, hi_enable=hi_enable,
+                             minmax=caches.minmax() if pooling == "minmax" else None)
 
 
 def attend_query(t, q_layers, caches: HostCaches, sparse, *, S, W, sm_scale, d_v):

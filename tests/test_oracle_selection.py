@@ -226,3 +226,92 @@ def test_select_fp32_matches_sorted_reference_on_float32_compare():
     pos[::11] = -1
     got = orc.select_fp32(sc, pos, 0, 20, apply_range=False)
     assert list(got) == _sorted_topk([(float(s), int(p)) for s, p in zip(sc, pos) if p >= 0], 20)
+
+
+# ---------------------------------------------------------------- MinMax pooling (Eq. 13)
+def _eq13_loops(q, w, keys_of_page, B):
+    """Eq. 13 page score with scalar loops over sub-blocks, heads and dimensions, extrema found token by token."""
+    tot = 0.0
+    n_tok = len(keys_of_page)
+    for n0 in range(0, n_tok, B):
+        blk = keys_of_page[n0:n0 + B]
+        for j in range(q.shape[0]):
+            s_tilde = 0.0
+            for c in range(q.shape[1]):
+                hi_c = max(float(k_s[c]) for k_s in blk)
+                lo_c = min(float(k_s[c]) for k_s in blk)
+                s_tilde += max(q[j, c] * hi_c, q[j, c] * lo_c)
+            tot += w[j] * max(s_tilde, 0.0)
+    return tot
+
+
+def test_minmax_page_scores_equal_scalar_loops():
+    rng = np.random.default_rng(31)
+    P, B, H, d = 16, 4, 3, 8
+    q, w, k = _rand_problem(rng, 70, H, d)             # 70 keys: the last page is partial, so is its last sub-block
+    kmax, kmin = orc.block_minmax(k, B, round_bf16=False)
+    pages = np.arange(-(-70 // P))
+    got = orc.page_scores_minmax(q[5], w[5], kmax, kmin, P, B, pages)
+    for p in pages:
+        want = _eq13_loops(q[5], w[5], k[p * P:min((p + 1) * P, 70)], B)
+        assert got[p] == pytest.approx(want, rel=1e-12, abs=1e-12)
+
+
+def test_minmax_upper_bounds_every_token_score_and_B1_is_the_token_score():
+    """s~ of Eq. 13 bounds q.k for every token of the sub-block from above (the reason the paper gives for it), so
+    with non-negative head weights a page's MinMax score is at least the largest token score in it; with B = 1 the
+    extrema are the key itself and MinMax, mean pooling and Eq. 1 coincide."""
+    rng = np.random.default_rng(32)
+    P, B, H, d = 8, 4, 2, 6
+    q, w, k = _rand_problem(rng, 64, H, d)
+    w = np.abs(w)
+    kmax, kmin = orc.block_minmax(k, B, round_bf16=False)
+    for n in range(kmax.shape[0]):
+        s_tilde = np.maximum(q[9] * kmax[n], q[9] * kmin[n]).sum(axis=1)          # [H]
+        for s in range(n * B, n * B + B):
+            assert (s_tilde >= q[9] @ k[s] - 1e-12).all()
+    pages = np.arange(64 // P)
+    page_mm = orc.page_scores_minmax(q[9], w[9], kmax, kmin, P, B, pages)
+    tok = orc.indexer_scores(q[9], w[9], k)
+    for p in pages:
+        assert page_mm[p] >= tok[p * P:(p + 1) * P].max() - 1e-12
+    # B = 1
+    k1max, k1min = orc.block_minmax(k, 1, round_bf16=False)
+    assert np.array_equal(k1max, k) and np.array_equal(k1min, k)
+    mm1 = orc.page_scores_minmax(q[9], w[9], k1max, k1min, P, 1, pages)
+    mean1 = orc.page_scores(q[9], w[9], orc.block_means(k, 1, round_bf16=False), P, 1, pages)
+    np.testing.assert_allclose(mm1, mean1, rtol=1e-12)
+    np.testing.assert_allclose(mm1, tok.reshape(-1, P).sum(axis=1), rtol=1e-12)
+
+
+def test_minmax_is_a_dot_product_of_split_queries():
+    """max(q*a, q*b) with a >= b is q*a for q >= 0 and q*b for q < 0, so Eq. 13 is [q+ | q-] . [k_max | k_min]:
+    the identity the GPU path computes with."""
+    rng = np.random.default_rng(33)
+    q, w, k = _rand_problem(rng, 32, 4, 8)
+    kmax, kmin = orc.block_minmax(k, 8, round_bf16=False)
+    qp, qm = np.maximum(q[3], 0.0), np.minimum(q[3], 0.0)
+    for n in range(kmax.shape[0]):
+        direct = np.maximum(q[3] * kmax[n], q[3] * kmin[n]).sum(axis=1)
+        np.testing.assert_allclose(qp @ kmax[n] + qm @ kmin[n], direct, rtol=1e-12, atol=1e-15)
+
+
+def test_minmax_selection_keeps_the_needle_page():
+    """A page holding one key strongly aligned with the query is recalled by MinMax stage 1 even when the other keys
+    of its sub-block are anti-aligned (a case where the mean cancels): the upper-bound property at work."""
+    rng = np.random.default_rng(34)
+    L, P, B, H, d = 512, 16, 8, 2, 16
+    q, w, k = _rand_problem(rng, L, H, d)
+    w = np.abs(w)
+    t = L - 1
+    needle = 100
+    k[needle] = 6.0 * q[t, 0] / np.linalg.norm(q[t, 0])
+    for s in range(96, 104):                     # the needle's sub-block: the others pull the mean the other way
+        if s != needle:
+            k[s] = -k[needle] / 7.0
+    kw = dict(P=P, B=B, M=4, Ksp=32, S=2, W=8)
+    mm = orc.block_minmax(k, B)
+    sparse_mm, pages_mm = orc.select_sparse(t, q[t], w[t], k, None, minmax=mm, **kw)
+    assert needle // P in pages_mm and needle in sparse_mm
+    sparse_mean, pages_mean = orc.select_sparse(t, q[t], w[t], k, orc.block_means(k, B), **kw)
+    assert needle // P not in pages_mean
