@@ -88,7 +88,11 @@ typedef struct {
                            1: caches are pools [n_phys_pages*kv_page, d] read through page_table and there is
                               one query per sequence at position ctx_len[b]-1 (decode) */
   int32_t kv_page;      /* tokens per physical cache page (paged mode) */
+  int32_t pooling;      /* coarse-stage pooling of a sub-block: LSA_POOL_MEAN (Eq. 9, the paper's choice) or
+                           LSA_POOL_MINMAX (Eq. 13, the variant of its pooling ablation; contiguous caches only) */
 } lsa_params;
+
+enum { LSA_POOL_MEAN = 0, LSA_POOL_MINMAX = 1 };
 
 /* ---- context ------------------------------------------------------------------------------ */
 
@@ -140,7 +144,10 @@ LSA_API int lsa_profile_read(lsa_ctx* ctx, double* total_ms, int64_t* launches);
  * [n_phys_pages*kv_page/B, d_I]: sub-block j of physical page g is row g*(kv_page/B)+j.  The means of
  * sequence b's first ctx_len[b] tokens are written (a trailing partial sub-block averages the tokens
  * present); n_key is ignored; page_table int32 [batch, page_table_stride].
- * Prefill: page_table = ctx_len = NULL, batch = 1. */
+ * Prefill: page_table = ctx_len = NULL, batch = 1.
+ * With pooling = LSA_POOL_MINMAX (Sec. 5, "Pooling method") the cache holds the per-dimension extrema instead:
+ *   kmean    bf16 [ceil(n_key/B), 2*d_I]: row n = [max over the sub-block's tokens | min over them], each value
+ *            the dequantised key value rounded to bf16; paged mode returns LSA_ERR_SHAPE. */
 LSA_API int lsa_block_means(lsa_ctx* ctx, const lsa_params* p, const void* k_idx, const float* k_scale,
                     int64_t n_key, const int32_t* page_table, int64_t page_table_stride,
                     const int32_t* ctx_len, int batch, void* kmean);
@@ -150,7 +157,9 @@ LSA_API int lsa_block_means(lsa_ctx* ctx, const lsa_params* p, const void* k_idx
 /* For each query: eligible pages E = pages meeting C(t); if hi_enable and |E| > M keep the M pages
  * with the largest Eq.-9 score, else all of E; score the tokens of the kept pages inside C(t) with
  * Eq. 1 (fp32 accumulation of bf16 products; e4m3 keys are widened exactly and the per-token scale is
- * applied to the dot product); keep the Ksp largest.
+ * applied to the dot product); keep the Ksp largest.  With pooling = LSA_POOL_MINMAX the page score uses
+ * s~ = sum_d max(q_d k_max_d, q_d k_min_d) (Eq. 13) in place of the mean-key dot product, computed as
+ * [max(q,0) | min(q,0)] . [k_max | k_min]; `kmean` is then the extrema cache of lsa_block_means.
  *   q_idx       bf16 [n_query, H_I, d_I]       w  fp32 [n_query, H_I]
  *   k_idx/k_scale/kmean  as in lsa_block_means
  *   prefill (paged=0): query row i sits at position q_pos0+i; n_key tokens are cached (>= q_pos0+n_query);

@@ -18,6 +18,7 @@ _LIB = None
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblsa.so")
 
 LSA_KEY_BF16, LSA_KEY_E4M3 = 0, 1
+LSA_POOL_MEAN, LSA_POOL_MINMAX = 0, 1
 KERNEL_CLASSES = ("block_means", "coarse_score", "fine_select", "select", "convert", "sparse_attn", "merge_splits")
 
 
@@ -32,7 +33,7 @@ class LsaParams(ctypes.Structure):
                 ("page", c_int32), ("sub_block", c_int32), ("keep_pages", c_int32), ("k_sparse", c_int32),
                 ("k_sink", c_int32), ("k_swa", c_int32), ("n_heads", c_int32), ("d_qk", c_int32), ("d_v", c_int32),
                 ("sm_scale", c_float), ("n_layers", c_int32), ("q_chunk", c_int32), ("hi_enable", c_int32),
-                ("paged", c_int32), ("kv_page", c_int32)]
+                ("paged", c_int32), ("kv_page", c_int32), ("pooling", c_int32)]
 
 
 EXPORTS = {
@@ -90,7 +91,8 @@ def lib() -> ctypes.CDLL:
 def make_params(cfg: LsaConfig) -> LsaParams:
     return LsaParams(ctypes.sizeof(LsaParams), cfg.H_I, cfg.d_I, LSA_KEY_E4M3 if cfg.key_dtype == "e4m3" else LSA_KEY_BF16,
                      cfg.P, cfg.B, cfg.M, cfg.Ksp, cfg.S, cfg.W, cfg.H, cfg.d_qk, cfg.d_v, cfg.sm_scale, cfg.R,
-                     cfg.q_chunk, 1 if cfg.hi_enable else 0, 1 if cfg.mode == "decode" else 0, cfg.kv_page)
+                     cfg.q_chunk, 1 if cfg.hi_enable else 0, 1 if cfg.mode == "decode" else 0, cfg.kv_page,
+                     LSA_POOL_MINMAX if cfg.pooling == "minmax" else LSA_POOL_MEAN)
 
 
 def _p(t):

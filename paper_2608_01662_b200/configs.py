@@ -39,6 +39,7 @@ class LsaConfig:
     boost_prob: float = 0.0   # share of tokens whose indexer key is scaled by boost_gain
     boost_gain: float = 1.0
     hi_enable: bool = True
+    pooling: str = "mean"   # coarse-stage pooling: "mean" (Eq. 9) or "minmax" (Eq. 13)
 
     def replace(self, **kw) -> "LsaConfig":
         return dataclasses.replace(self, **kw)

@@ -74,6 +74,8 @@ int check_params(const lsa_params* p, bool need_index, bool need_attn) {
     if (static_cast<int64_t>(p->keep_pages) * p->page > 4096) return LSA_ERR_SHAPE;
     if (p->k_sparse > 4096 || p->k_sparse % 4 != 0) return LSA_ERR_SHAPE;
     if (p->paged && p->kv_page != p->page) return LSA_ERR_SHAPE;
+    if (p->pooling != LSA_POOL_MEAN && p->pooling != LSA_POOL_MINMAX) return LSA_ERR_ARG;
+    if (p->pooling == LSA_POOL_MINMAX && p->paged) return LSA_ERR_SHAPE;   // the variant is built for contiguous caches
   }
   if (need_attn) {
     if (!lsa::attn_shape_supported(p->n_heads, p->d_qk, p->d_v)) return LSA_ERR_SHAPE;
@@ -220,7 +222,9 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
       if (e != cudaSuccess) return cuda_fail(c, e);
       continue;
     }
-    if (p->hi_enable)
+    if (p->hi_enable && p->pooling == LSA_POOL_MINMAX)
+      e = timed(c, LSA_K_COARSE, [&] { return lsa::launch_coarse_minmax(a, c->stream, &c->launches); });
+    else if (p->hi_enable)
       e = timed(c, LSA_K_COARSE, [&] {
         return lsa::coarse_tc_supported(a) ? lsa::launch_coarse_tc(a, c->tune[LSA_TUNE_COARSE_GROUPS], c->stream, &c->launches)
                                            : lsa::launch_coarse(a, c->stream, &c->launches);
@@ -407,6 +411,13 @@ int lsa_block_means(lsa_ctx* c, const lsa_params* p, const void* k_idx, const fl
   if (p->key_dtype == LSA_KEY_E4M3 && k_scale == nullptr) return LSA_ERR_ARG;
   if (p->paged && (page_table == nullptr || ctx_len == nullptr || batch <= 0 || page_table_stride <= 0)) return LSA_ERR_ARG;
   if (!aligned16(k_idx) || !aligned16(kmean)) return LSA_ERR_SHAPE;
+  if (p->pooling == LSA_POOL_MINMAX) {
+    const cudaError_t em = timed(c, LSA_K_MEANS, [&] {
+      return lsa::launch_block_minmax(p->d_idx, p->key_dtype == LSA_KEY_E4M3, p->sub_block, k_idx, k_scale, n_key, kmean,
+                                      c->stream, &c->launches);
+    });
+    return em == cudaSuccess ? LSA_OK : cuda_fail(c, em);
+  }
   cudaError_t e = timed(c, LSA_K_MEANS, [&] {
     return lsa::launch_block_means(p->d_idx, p->key_dtype == LSA_KEY_E4M3, p->sub_block, p->kv_page, k_idx, k_scale,
                                    n_key, p->paged ? page_table : nullptr, page_table_stride, ctx_len, batch, kmean,

@@ -630,6 +630,169 @@ __global__ void __launch_bounds__(kConvertThreads) convert_kernel(int S, int W, 
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// MinMax pooling (Eq. 13), contiguous caches: the coarse stage with per-dimension extrema of a sub-block in
+// place of its mean.  max(q*a, q*b) with a >= b is q*a for q >= 0 and q*b for q < 0, so
+// s~ = [max(q,0) | min(q,0)] . [k_max | k_min]: the Eq. 9 kernel's tile with rows of 2*d_I dims.
+// ------------------------------------------------------------------------------------------------
+template <bool E4M3>
+__global__ void block_minmax_kernel(const uint8_t* __restrict__ k_idx, const float* __restrict__ k_scale,
+                                    int64_t n_key, int DI, int B, __nv_bfloat16* __restrict__ kminmax) {
+  const int U = DI / 8;  // 8 dims per thread
+  const int64_t gid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int64_t sub = gid / U;
+  const int u = static_cast<int>(gid % U);
+  if (sub * B >= n_key) return;
+  const int64_t row0 = sub * B;
+  const int cnt = static_cast<int>(min64(B, n_key - row0));
+  float hi[8], lo[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    hi[j] = -INFINITY;
+    lo[j] = INFINITY;
+  }
+  for (int r = 0; r < cnt; ++r) {
+    const int64_t row = row0 + r;
+    float v[8];
+    if (E4M3) {
+      const uint2 c = *reinterpret_cast<const uint2*>(k_idx + row * DI + u * 8);
+      const float sc = k_scale[row];
+      const uint32_t w[2] = {c.x, c.y};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        __half2_raw h = __nv_cvt_fp8x2_to_halfraw2(
+            static_cast<__nv_fp8x2_storage_t>((w[j >> 1] >> ((j & 1) * 16)) & 0xffff), __NV_E4M3);
+        const float2 f = __half22float2(*reinterpret_cast<__half2*>(&h));
+        v[2 * j] = f.x * sc;
+        v[2 * j + 1] = f.y * sc;
+      }
+    } else {
+      const uint4 c = *reinterpret_cast<const uint4*>(k_idx + (row * DI + u * 8) * 2);
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&c);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 f = __bfloat1622float2(h[j]);
+        v[2 * j] = f.x;
+        v[2 * j + 1] = f.y;
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      hi[j] = fmaxf(hi[j], v[j]);
+      lo[j] = fminf(lo[j], v[j]);
+    }
+  }
+  uint4 oh, ol;
+  oh.x = pack_bf16(hi[0], hi[1]); oh.y = pack_bf16(hi[2], hi[3]); oh.z = pack_bf16(hi[4], hi[5]); oh.w = pack_bf16(hi[6], hi[7]);
+  ol.x = pack_bf16(lo[0], lo[1]); ol.y = pack_bf16(lo[2], lo[3]); ol.z = pack_bf16(lo[4], lo[5]); ol.w = pack_bf16(lo[6], lo[7]);
+  __nv_bfloat16* out = kminmax + sub * 2 * DI;
+  *reinterpret_cast<uint4*>(out + u * 8) = oh;          // [k_max | k_min]
+  *reinterpret_cast<uint4*>(out + DI + u * 8) = ol;
+}
+
+template <int HI, int DI>
+struct CoarseMinMaxSmem {
+  alignas(128) uint8_t a[kTileRows * DI * 4];     // 128 sub-blocks x [k_max | k_min]
+  alignas(128) uint8_t q[2][HI * DI * 4];         // [q+ | q-] per head, two queries in flight
+  float w[2][HI];
+  float sub[kTileRows];
+};
+
+// One block = one tile of 128 sub-blocks x a group of queries (as coarse_score_kernel); a query's heads are split
+// into positive and negative parts on their way into shared memory.
+template <int HI, int DI>
+__global__ void __launch_bounds__(kThreads) coarse_minmax_kernel(IndexArgs p) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  auto& sm = *reinterpret_cast<CoarseMinMaxSmem<HI, DI>*>(smem_raw);
+  constexpr int D2 = 2 * DI;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int spp = p.P / p.B;
+  const int ppt = kTileRows / spp;
+  const int64_t sub0 = static_cast<int64_t>(blockIdx.x) * kTileRows;
+  const int64_t page0 = sub0 / spp;
+  const int q_begin = blockIdx.y * kCoarseQG;
+  const int q_end = min(p.n_query, q_begin + kCoarseQG);
+  const int64_t n_key = p.n_key;
+  // a query needs this tile iff the tile's first page is eligible and the coarse stage runs at all for it
+  const int64_t t_need = max(page0 * p.P + p.W, (static_cast<int64_t>(p.M) + p.S / p.P) * p.P + p.W);
+  if (p.q_pos0 + q_end - 1 < t_need) return;
+  int q_first = q_begin;
+  if (t_need - p.q_pos0 > q_begin) q_first = static_cast<int>(t_need - p.q_pos0);
+
+  const int64_t n_sub = (n_key + p.B - 1) / p.B;
+  {
+    constexpr int U = D2 / 8;
+    const uint8_t* km = reinterpret_cast<const uint8_t*>(p.kmean);
+    for (int e = tid; e < kTileRows * U; e += kThreads) {
+      const int r = e / U, u = e % U;
+      const int64_t sub = sub0 + r;
+      cp_async16(smem_u32(sm.a) + swz<D2 * 2>(r, u), km + (sub < n_sub ? sub : 0) * D2 * 2 + u * 16, sub < n_sub ? 16 : 0);
+    }
+    cp_async_commit();
+  }
+  constexpr int UQ = DI / 8;                       // 16-byte units of one head's query row
+  constexpr int kPerThread = (HI * UQ + kThreads - 1) / kThreads;
+  const uint8_t* qg = reinterpret_cast<const uint8_t*>(p.q_idx);
+  auto load_q = [&](int qi, uint4 (&v)[kPerThread]) {
+#pragma unroll
+    for (int j = 0; j < kPerThread; ++j) {
+      const int e = tid + j * kThreads;
+      v[j] = e < HI * UQ ? *reinterpret_cast<const uint4*>(qg + (static_cast<int64_t>(qi) * HI * UQ + e) * 16) : make_uint4(0, 0, 0, 0);
+    }
+  };
+  auto store_q = [&](int qi, int buf, const uint4 (&v)[kPerThread]) {
+    const __nv_bfloat162 zero = __floats2bfloat162_rn(0.f, 0.f);
+#pragma unroll
+    for (int j = 0; j < kPerThread; ++j) {
+      const int e = tid + j * kThreads;
+      if (e >= HI * UQ) continue;
+      const int h = e / UQ, u = e % UQ;
+      uint4 pos, neg;
+      const __nv_bfloat162* x = reinterpret_cast<const __nv_bfloat162*>(&v[j]);
+      __nv_bfloat162* xp = reinterpret_cast<__nv_bfloat162*>(&pos);
+      __nv_bfloat162* xn = reinterpret_cast<__nv_bfloat162*>(&neg);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        xp[i] = __hmax2(x[i], zero);
+        xn[i] = __hmin2(x[i], zero);
+      }
+      *reinterpret_cast<uint4*>(sm.q[buf] + swz<D2 * 2>(h, u)) = pos;
+      *reinterpret_cast<uint4*>(sm.q[buf] + swz<D2 * 2>(h, UQ + u)) = neg;
+    }
+    if (tid < HI) sm.w[buf][tid] = p.w[static_cast<int64_t>(qi) * HI + tid];
+  };
+  uint4 qv[kPerThread];
+  load_q(q_first, qv);
+  store_q(q_first, 0, qv);
+  cp_async_wait<0>();
+  __syncthreads();
+  uint32_t a[D2 / 16][4];
+  load_a_frags<D2>(a, smem_u32(sm.a));
+
+  for (int qi = q_first; qi < q_end; ++qi) {
+    const int buf = (qi - q_first) & 1;
+    if (qi + 1 < q_end) load_q(qi + 1, qv);       // in flight during the scoring
+    float s_lo, s_hi;
+    score_16rows<HI, D2>(a, smem_u32(sm.q[buf]), sm.w[buf], s_lo, s_hi);
+    if ((lane & 3) == 0) {
+      sm.sub[16 * warp + (lane >> 2)] = s_lo;
+      sm.sub[16 * warp + (lane >> 2) + 8] = s_hi;
+    }
+    if (qi + 1 < q_end) store_q(qi + 1, buf ^ 1, qv);   // the other buffer: last read one iteration ago, before a barrier
+    __syncthreads();
+    if (tid < ppt) {
+      const int64_t page = page0 + tid;
+      const int64_t hi = p.q_pos0 + qi - p.W;
+      if (page * p.P <= hi) {
+        float s = 0.f;
+        for (int j = 0; j < spp; ++j) s += sm.sub[tid * spp + j];
+        p.page_scores[static_cast<int64_t>(qi) * p.ps_ld + page] = s;
+      }
+    }
+    __syncthreads();
+  }
+}
+
 template <class K>
 cudaError_t set_smem(K kernel, size_t bytes) {
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
@@ -686,6 +849,41 @@ cudaError_t launch_coarse(const IndexArgs& a, cudaStream_t st, int64_t* n_launch
   if (coarse_paged_tc_supported(a)) return launch_coarse_paged_tc(a, st, n_launch);
   if (a.HI == 8 && a.DI == 64) return launch_coarse_t<8, 64>(a, n_key_max, st, n_launch);
   return launch_coarse_t<64, 128>(a, n_key_max, st, n_launch);
+}
+
+cudaError_t launch_block_minmax(int DI, int key_e4m3, int B, const void* k_idx, const float* k_scale, int64_t n_key,
+                                void* kminmax, cudaStream_t st, int64_t* n_launch) {
+  const int U = DI / 8;
+  const int64_t n_sub = (n_key + B - 1) / B;
+  if (n_sub == 0) return cudaSuccess;
+  const int threads = 256;
+  const unsigned blocks = static_cast<unsigned>((n_sub * U + threads - 1) / threads);
+  auto* kp = reinterpret_cast<const uint8_t*>(k_idx);
+  auto* out = reinterpret_cast<__nv_bfloat16*>(kminmax);
+  if (key_e4m3) block_minmax_kernel<true><<<blocks, threads, 0, st>>>(kp, k_scale, n_key, DI, B, out);
+  else block_minmax_kernel<false><<<blocks, threads, 0, st>>>(kp, k_scale, n_key, DI, B, out);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+template <int HI, int DI>
+static cudaError_t launch_coarse_minmax_t(const IndexArgs& a, cudaStream_t st, int64_t* n_launch) {
+  const size_t smem = sizeof(CoarseMinMaxSmem<HI, DI>);
+  cudaError_t e = set_smem(coarse_minmax_kernel<HI, DI>, smem);
+  if (e != cudaSuccess) return e;
+  const int64_t n_sub = (a.n_key + a.B - 1) / a.B;
+  dim3 grid(static_cast<unsigned>((n_sub + kTileRows - 1) / kTileRows), (a.n_query + kCoarseQG - 1) / kCoarseQG);
+  coarse_minmax_kernel<HI, DI><<<grid, kThreads, smem, st>>>(a);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+// a.kmean is the extrema cache [ceil(n_key/B), 2*DI]; contiguous caches only
+cudaError_t launch_coarse_minmax(const IndexArgs& a, cudaStream_t st, int64_t* n_launch) {
+  if (a.n_query == 0) return cudaSuccess;
+  if (a.paged) return cudaErrorInvalidValue;
+  if (a.HI == 8 && a.DI == 64) return launch_coarse_minmax_t<8, 64>(a, st, n_launch);
+  return launch_coarse_minmax_t<64, 128>(a, st, n_launch);
 }
 
 template <int HI, int DI, bool E4M3>

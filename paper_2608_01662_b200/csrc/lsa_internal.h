@@ -61,6 +61,10 @@ cudaError_t launch_block_means(int DI, int key_e4m3, int B, int kv_page, const v
                                int64_t n_key, const int32_t* page_table, int64_t pt_stride,
                                const int32_t* ctx_len, int batch, void* kmean, cudaStream_t st, int64_t* n_launch);
 cudaError_t launch_coarse(const IndexArgs& a, cudaStream_t st, int64_t* n_launch);
+// MinMax pooling (Eq. 13), contiguous caches: extrema cache [ceil(n_key/B), 2*DI] = [k_max | k_min], and the coarse stage on it
+cudaError_t launch_block_minmax(int DI, int key_e4m3, int B, const void* k_idx, const float* k_scale, int64_t n_key,
+                                void* kminmax, cudaStream_t st, int64_t* n_launch);
+cudaError_t launch_coarse_minmax(const IndexArgs& a, cudaStream_t st, int64_t* n_launch);
 // tcgen05 version of the coarse stage (contiguous caches, H_I = 64, d_I = 128); groups = 4-query groups per block
 bool coarse_tc_supported(const IndexArgs& a);
 cudaError_t launch_coarse_tc(const IndexArgs& a, int groups, cudaStream_t st, int64_t* n_launch);

@@ -41,6 +41,7 @@ extern "C" int lsa_index_static(int device, void* cuda_stream, const lsa_params*
   if (p == nullptr || p->struct_size != sizeof(lsa_params)) return LSA_ERR_ARG;
   if (device < 0 || device >= kMaxDevices) return LSA_ERR_ARG;
   if (p->paged) return LSA_ERR_ARG;  // contiguous caches only
+  if (p->pooling != LSA_POOL_MEAN) return LSA_ERR_SHAPE;  // mean pooling only
   if (p->key_dtype != LSA_KEY_BF16 && p->key_dtype != LSA_KEY_E4M3) return LSA_ERR_ARG;
   if (p->k_sink < 0 || p->k_swa < 0 || p->k_sparse < 0 || p->keep_pages <= 0 || p->sub_block <= 0) return LSA_ERR_ARG;
   if (!lsa::index_shape_supported(p->n_heads_idx, p->d_idx)) return LSA_ERR_SHAPE;

@@ -34,7 +34,8 @@ class PrefillWorkload:
             self.out.append(torch.empty((self.n_query, cfg.H, cfg.d_v), dtype=torch.bfloat16, device=dev))
             self.lse.append(torch.empty((self.n_query, cfg.H), dtype=torch.float32, device=dev) if with_lse else None)
         n_sub = (self.n_key + cfg.B - 1) // cfg.B
-        self.kmean = torch.empty((n_sub, cfg.d_I), dtype=torch.bfloat16, device=dev)
+        # mean keys, or [k_max | k_min] rows for the MinMax pooling variant
+        self.kmean = torch.empty((n_sub, cfg.d_I * (2 if cfg.pooling == "minmax" else 1)), dtype=torch.bfloat16, device=dev)
         self.sparse_idx = torch.empty((self.n_query, cfg.Ksp), dtype=torch.int32, device=dev)
         self.n_sparse = torch.empty((self.n_query,), dtype=torch.int32, device=dev)
         self.ctx = binding.Context(self.params, self.n_query, self.n_key, 1, device=dev) if make_ctx else None

@@ -90,7 +90,8 @@ def check_prefill(wl, queries, check_attention=True, pages=None) -> Metrics:
         n_sp = int(wl.n_sparse[i])
         gpu_sparse = to_np(wl.sparse_idx[i])
         check_invariants(cfg, t, gpu_sparse, n_sp)
-        ref_sparse, ref_pages = ref.select_query(t, to_np(wl.q_idx[i]), to_np(wl.w[i]), caches, hi_enable=cfg.hi_enable, **kw)
+        ref_sparse, ref_pages = ref.select_query(t, to_np(wl.q_idx[i]), to_np(wl.w[i]), caches, hi_enable=cfg.hi_enable,
+                                                 pooling=cfg.pooling, **kw)
         assert n_sp == len(ref_sparse), (t, n_sp, len(ref_sparse))
         gp = None
         if pages is not None:

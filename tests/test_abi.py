@@ -32,7 +32,7 @@ def test_host_only_entry_points():
         n = binding.workspace_bytes(p, cfg.L or cfg.batch, cfg.L or cfg.ctx_hi, cfg.batch)
         assert n % 256 == 0 and n > 0
     p = binding.make_params(CONFIGS["cfg3"])
-    assert ctypes.sizeof(p) == p.struct_size == 76
+    assert ctypes.sizeof(p) == p.struct_size == 80
     # cfg3: page scores (131072 queries x 1024 pages x 4 B) + the e4m3 keys widened to bf16 (131072 x 128 x 2 B)
     assert binding.workspace_bytes(p, 131072, 131072) == 131072 * 1024 * 4 + 131072 * 128 * 2 + 256
     # q_chunk bounds the scratch

@@ -229,6 +229,39 @@ def test_convert_lists_physical_rows(cuda_device):
         assert r[3] <= n_sp + cfg.W // cfg.kv_page + 3
 
 
+# ---------------------------------------------------------------- MinMax pooling (Eq. 13)
+@pytest.mark.parametrize("base", ["fp8", "bf16"])
+def test_minmax_cache_and_selection(cuda_device, base):
+    """The extrema cache equals the oracle's (an extremum is a key value: one rounding), and the two-stage selection
+    with Eq. 13 page scores picks the oracle's pages and tokens."""
+    if base == "fp8":
+        cfg = SMALL_FP8.replace(name="mm_fp8", pooling="minmax", R=1)
+    else:
+        cfg = CONFIGS["cfg1"].replace(name="mm_bf16", pooling="minmax", L=1500, seed=41)
+    wl = PrefillWorkload(cfg, cuda_device)
+    wl.prepare()
+    k_hat = (orc.dequant_keys(pu.to_np(wl.keys["k"]), pu.to_np(wl.keys["scale"])) if "scale" in wl.keys
+             else pu.to_np(wl.keys["k"]).astype(np.float64))
+    kmax, kmin = orc.block_minmax(k_hat, cfg.B)
+    got = pu.to_np(wl.kmean).astype(np.float64)
+    want = np.concatenate([kmax, kmin], axis=1)
+    # e4m3: the kernel rounds code x scale to fp32 before bf16, the oracle rounds the exact product once
+    diff = np.abs(got - want)
+    assert (diff <= np.abs(want) * 2.0 ** -7).all() and (diff > 0).mean() < 2e-3
+    pages = torch.full((wl.n_query, cfg.M), -7, dtype=torch.int32, device=cuda_device)
+    wl.index(pages)
+    assert wl.ctx.status() == 0
+    m = pu.check_prefill(wl, pu.boundary_queries(cfg, 0, cfg.L, 60, seed=5), check_attention=False, pages=pages)
+    print(cfg.name, m.summary())
+    assert m.summary()["mean_overlap"] >= pu.MIN_OVERLAP
+
+
+def test_minmax_rejects_paged_caches(cuda_device):
+    p = binding.make_params(SMALL_DEC.replace(pooling="minmax"))
+    with pytest.raises(binding.LsaError):
+        binding.workspace_bytes(p, 8, 4096, 8)
+
+
 # ---------------------------------------------------------------- edge cases and errors
 def test_short_sequences_and_empty_calls(cuda_device):
     cfg = CONFIGS["cfg1"].replace(L=100, name="short")            # L < S + W: every query sees [0, t]
