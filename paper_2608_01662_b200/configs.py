@@ -38,6 +38,8 @@ class LsaConfig:
     kv_page: int = 0     # decode: tokens per physical cache page
     boost_prob: float = 0.0   # share of tokens whose indexer key is scaled by boost_gain
     boost_gain: float = 1.0
+    segment_corr: float = 0.0  # share of an indexer key's variance that is common to its run of segment_len tokens
+    segment_len: int = 64
     hi_enable: bool = True
     pooling: str = "mean"   # coarse-stage pooling: "mean" (Eq. 9) or "minmax" (Eq. 13)
 

@@ -8,7 +8,11 @@ own seed, so that any row range of a huge tensor can be regenerated alone.
 
 Laws: indexer q_I, k_I ~ N(0, 1/d_I); head weights w ~ N(0, 1/H_I); attention
 q, k, v (or the MLA latent) ~ N(0, 1).  With boost_prob > 0 a Bernoulli share of
-tokens has its indexer key multiplied by boost_gain before it is stored.
+tokens has its indexer key multiplied by boost_gain before it is stored.  With
+segment_corr = rho > 0 the indexer keys of each run of segment_len consecutive
+tokens share a direction: k_s = sqrt(rho) c_seg + sqrt(1 - rho) e_s with c, e
+of the same law (text whose neighbouring tokens attend alike, the structure a
+page-level score can see); the marginal law of a key is unchanged.
 """
 from __future__ import annotations
 
@@ -20,7 +24,7 @@ from .configs import LsaConfig
 
 GEN_ROWS = 16384
 
-T_QI, T_KI, T_W, T_BOOST, T_Q, T_KV, T_V, T_CTX, T_PERM = 0, 1, 2, 3, 10, 20, 40, 30, 31
+T_QI, T_KI, T_W, T_BOOST, T_SEG, T_Q, T_KV, T_V, T_CTX, T_PERM = 0, 1, 2, 3, 4, 10, 20, 40, 30, 31
 
 E4M3_MAX = 448.0
 
@@ -70,6 +74,11 @@ def indexer_keys(cfg: LsaConfig, n_rows: int, device):
     for r0 in range(0, n_rows, GEN_ROWS):
         n = min(GEN_ROWS, n_rows - r0)
         k = _rows(cfg, T_KI, r0, n, (cfg.d_I,), 1.0 / math.sqrt(cfg.d_I), device)
+        if cfg.segment_corr > 0:
+            seg0, seg1 = r0 // cfg.segment_len, (r0 + n - 1) // cfg.segment_len
+            c = _rows(cfg, T_SEG, seg0, seg1 - seg0 + 1, (cfg.d_I,), 1.0 / math.sqrt(cfg.d_I), device)
+            seg_of = torch.arange(r0, r0 + n, device=device) // cfg.segment_len - seg0
+            k = math.sqrt(cfg.segment_corr) * c[seg_of] + math.sqrt(1.0 - cfg.segment_corr) * k
         if cfg.boost_prob > 0:
             u = _rows(cfg, T_BOOST, r0, n, (), 1.0, device, uniform=True)
             k = torch.where((u < cfg.boost_prob)[:, None], k * cfg.boost_gain, k)
