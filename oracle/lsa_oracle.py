@@ -55,6 +55,51 @@ def e4m3_decode(codes):
     return sign * val
 
 
+def e4m3_encode(x):
+    """Real value -> OCP FP8 E4M3 code, round to nearest (ties to the even mantissa), saturating at +-448.
+
+    Written as a search over the 127 non-negative finite code values, so that it shares nothing with e4m3_decode's
+    closed form except the table that function produces; NaN is not expected.
+    """
+    x = np.asarray(x, dtype=np.float64)
+    mags = e4m3_decode(np.arange(0, 127, dtype=np.uint8))          # codes 0x00..0x7e, ascending values 0..448
+    a = np.minimum(np.abs(x), 448.0)
+    hi = np.searchsorted(mags, a, side="left").clip(0, 126)        # first code value >= a
+    lo = np.maximum(hi - 1, 0)
+    d_hi, d_lo = mags[hi] - a, a - mags[lo]
+    pick_lo = (d_lo < d_hi) | ((d_lo == d_hi) & (lo % 2 == 0))     # tie: the code with the even mantissa bit
+    code = np.where(pick_lo, lo, hi).astype(np.uint8)
+    return np.where(np.signbit(x), code | 0x80, code).astype(np.uint8)
+
+
+def quantize_token(k_row):
+    """One indexer key (any real dtype) -> (e4m3 codes uint8 [d], fp32 scale): scale = amax / 448 (1 for a zero row),
+    code = RNE(k / scale).  The scale and the quotient are fp32 values, as on the device: a quantised code is an
+    integer decision and both sides take it in the same precision."""
+    k = np.asarray(k_row, dtype=np.float32)
+    amax = np.float32(np.abs(k).max()) if k.size else np.float32(0)
+    scale = np.float32(amax / np.float32(448.0)) if amax > 0 else np.float32(1.0)
+    return e4m3_encode((k / scale).astype(np.float32)), scale
+
+
+def append_token(k_codes, k_scale, km, n_key, k_new, B):
+    """Cache maintenance of one decode step for one sequence (Sec. 3.3: the mean keys are maintained with the cache):
+    the new token's indexer key is quantised and stored at position n_key, and the mean of the sub-block that holds
+    it is recomputed over the tokens now present.  Arrays are logical (unpaged) and large enough; returns n_key + 1.
+    With k_scale None the cache holds real (bf16) keys and k_new is stored as is."""
+    if k_scale is not None:
+        codes, scale = quantize_token(k_new)
+        k_codes[n_key] = codes
+        k_scale[n_key] = scale
+    else:
+        k_codes[n_key] = k_new
+    n = n_key // B
+    lo, hi = n * B, n_key + 1
+    blk = dequant_keys(k_codes[lo:hi], k_scale[lo:hi]) if k_scale is not None else np.asarray(k_codes[lo:hi], np.float64)
+    km[n] = bf16_round(blk.sum(axis=0) / (hi - lo))
+    return n_key + 1
+
+
 def dequant_keys(k_codes, k_scale):
     """Stored fp8 indexer keys -> real keys: decode(code) * per-token scale."""
     return e4m3_decode(k_codes) * np.asarray(k_scale, dtype=np.float64)[:, None]

@@ -97,3 +97,69 @@ def test_generators_are_deterministic_and_chunk_consistent():
     used = table[table >= 0]
     assert used.numel() == n_pg and torch.equal(torch.sort(used).values, torch.arange(n_pg, dtype=torch.int32))
     assert ((ctx >= 100) & (ctx <= 300)).all()
+
+
+# ---------------------------------------------------------------- e4m3 encoding and the append-token maintenance
+def test_e4m3_encode_round_trips_every_code_and_matches_a_library_cast():
+    import torch
+    codes = np.arange(256, dtype=np.uint8)
+    finite = codes[(codes & 0x7f) != 0x7f]
+    vals = orc.e4m3_decode(finite)
+    back = orc.e4m3_encode(vals)
+    keep = finite != 0x80                                   # -0 encodes as 0x80 as well: compare values there
+    assert np.array_equal(back[keep], finite[keep]) and orc.e4m3_decode(back[~keep])[0] == 0.0
+    # an independent implementation of the same rounding: torch's float8_e4m3fn cast (saturation applied by hand)
+    rng = np.random.default_rng(5)
+    x = np.concatenate([rng.standard_normal(20000) * 100.0, rng.standard_normal(20000) * 0.01,
+                        np.array([0.0, 448.0, 460.0, -1000.0, 2.0 ** -9, 2.0 ** -10, 1.5 * 2.0 ** -9, 17.0, 19.0, 0.0625 * 1.0625])])
+    x32 = x.astype(np.float32)
+    want = torch.from_numpy(x32).clamp(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    got = orc.e4m3_encode(x32)
+    same_value = orc.e4m3_decode(got) == orc.e4m3_decode(want)      # +0 / -0 may differ in sign bit only
+    assert same_value.all()
+    # ties go to the even mantissa: 17 lies between 16 (m=0) and 18 (m=1); 19 between 18 (m=1) and 20 (m=2)
+    assert orc.e4m3_decode(orc.e4m3_encode(np.array([17.0, 19.0]))).tolist() == [16.0, 20.0]
+
+
+def test_quantize_token_scale_and_error_bound():
+    rng = np.random.default_rng(6)
+    k = (rng.standard_normal(128) * 0.3).astype(np.float32)
+    codes, scale = orc.quantize_token(k)
+    assert scale == np.float32(np.abs(k).max() / np.float32(448.0))
+    err = np.abs(orc.e4m3_decode(codes) * float(scale) - k)
+    # relative step of e4m3 is 2^-3 for normal values: half a step, plus the subnormal floor 2^-10 * scale
+    assert (err <= np.maximum(np.abs(k) * 2.0 ** -4, 2.0 ** -10 * float(scale)) * 1.0001).all()
+    assert np.abs(orc.e4m3_decode(codes)).max() == 448.0
+    z, s1 = orc.quantize_token(np.zeros(16, np.float32))
+    assert s1 == 1.0 and (z == 0).all()
+
+
+def test_append_token_equals_rebuilding_the_caches():
+    """Appending tokens one at a time leaves the caches exactly as quantising all keys and calling block_means on
+    the whole sequence would (the scale is per token, a mean is a function of its sub-block alone)."""
+    rng = np.random.default_rng(7)
+    d, B, n0, n_add = 16, 8, 21, 30
+    keys = (rng.standard_normal((n0 + n_add, d)) * 0.2).astype(np.float32)
+    codes = np.zeros((n0 + n_add, d), np.uint8)
+    scales = np.ones(n0 + n_add, np.float32)
+    for i in range(n0):
+        codes[i], scales[i] = orc.quantize_token(keys[i])
+    km = np.zeros((-(-(n0 + n_add) // B), d))
+    km[:-(-n0 // B)] = orc.block_means(orc.dequant_keys(codes[:n0], scales[:n0]), B)
+    n = n0
+    for i in range(n_add):
+        n = orc.append_token(codes, scales, km, n, keys[n], B)
+        want = orc.block_means(orc.dequant_keys(codes[:n], scales[:n]), B)
+        assert np.array_equal(km[:want.shape[0]], want)
+    full_codes = np.stack([orc.quantize_token(k)[0] for k in keys])
+    assert n == n0 + n_add and np.array_equal(codes, full_codes)
+    # bf16 cache form
+    kb = orc.bf16_round(keys.astype(np.float64))
+    cache = np.zeros_like(kb)
+    cache[:n0] = kb[:n0]
+    km2 = np.zeros_like(km)
+    km2[:-(-n0 // B)] = orc.block_means(kb[:n0], B)
+    n = n0
+    for i in range(n_add):
+        n = orc.append_token(cache, None, km2, n, kb[n], B)
+    assert np.array_equal(km2, orc.block_means(kb, B))
