@@ -130,6 +130,7 @@ LSA_API int lsa_tune(lsa_ctx* ctx, int knob, int value);
  * launches go unrecorded).  lsa_profile_read waits for the stream and writes, per class, the summed
  * device time in ms and the number of recorded launches (host arrays of LSA_K_COUNT entries), then
  * starts over.  The first enable creates the events (host resources only). */
+/* lsa_append is timed as LSA_K_MEANS */
 enum { LSA_K_MEANS = 0, LSA_K_COARSE, LSA_K_FINE_SELECT, LSA_K_SELECT, LSA_K_CONVERT, LSA_K_ATTN, LSA_K_MERGE, LSA_K_COUNT };   /* lsa_merge is timed as LSA_K_MERGE */
 LSA_API int lsa_profile_enable(lsa_ctx* ctx, int on);
 LSA_API int lsa_profile_read(lsa_ctx* ctx, double* total_ms, int64_t* launches);
@@ -151,6 +152,25 @@ LSA_API int lsa_profile_read(lsa_ctx* ctx, double* total_ms, int64_t* launches);
 LSA_API int lsa_block_means(lsa_ctx* ctx, const lsa_params* p, const void* k_idx, const float* k_scale,
                     int64_t n_key, const int32_t* page_table, int64_t page_table_stride,
                     const int32_t* ctx_len, int batch, void* kmean);
+
+/* Cache maintenance of one decode step (paged mode only; Sec. 3.3 keeps the mean keys with the cache, Sec. 4.1
+ * lists their upkeep among the costs of decoding): for every sequence b the new token's indexer key is stored at
+ * position ctx_len[b] and the mean of the sub-block holding that position is recomputed over the tokens now present
+ * (the same arithmetic as lsa_block_means, so an appended cache equals a rebuilt one bit for bit).
+ *   k_new    bf16 [batch, d_I]: the new indexer keys.  For e4m3 caches each is quantised here: scale = amax / 448
+ *            (1 for a zero row), code = round-to-nearest-even of k / scale in fp32, saturating.
+ *   k_idx / k_scale / kmean   the pools of lsa_block_means, written in place
+ *   ctx_len  int32 [batch]: lengths BEFORE the append; the physical page of position ctx_len[b] must already be in
+ *            page_table (pages are handed out by the caller)
+ *   ctx_len_out  optional int32 [batch] = ctx_len + 1 (may be ctx_len itself)
+ *   kv_new / kv_pool  optional HOST arrays of n_kv device pointers: row b of kv_new[i] ([batch, kv_row_bytes] bytes)
+ *            is copied to the row of pool i that holds position ctx_len[b] (the attention caches of the group's
+ *            layers); kv_row_bytes is a multiple of 16, n_kv <= 8; n_kv = 0 skips this.
+ * One launch.  pooling = LSA_POOL_MINMAX returns LSA_ERR_SHAPE. */
+LSA_API int lsa_append(lsa_ctx* ctx, const lsa_params* p, const void* k_new, void* k_idx, float* k_scale, void* kmean,
+                       const int32_t* page_table, int64_t page_table_stride, const int32_t* ctx_len, int batch,
+                       int32_t* ctx_len_out, int n_kv, const void* const* kv_new, void* const* kv_pool,
+                       int64_t kv_row_bytes);
 
 /* ---- a1-a4: the indexer (Eq. 9-12 with the scoring range of Eq. 7) -------------------------- */
 

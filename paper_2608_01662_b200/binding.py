@@ -60,6 +60,8 @@ EXPORTS = {
     "lsa_sparse_attn": (c_int, [c_void_p, POINTER(LsaParams), c_void_p, c_void_p, c_void_p, c_int64, c_int64,
                                 c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_int,
                                 c_void_p, c_void_p]),
+    "lsa_append": (c_int, [c_void_p, POINTER(LsaParams), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64,
+                           c_void_p, c_int, c_void_p, c_int, POINTER(c_void_p), POINTER(c_void_p), c_int64]),
     "lsa_merge": (c_int, [c_void_p, POINTER(LsaParams), c_int, POINTER(c_void_p), POINTER(c_void_p), c_int64, c_void_p,
                           c_void_p]),
     "lsa_layer_group": (c_int, [c_void_p, POINTER(LsaParams), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -222,6 +224,14 @@ class Context:
         self._chk(lib().lsa_sparse_attn(self.h, ctypes.byref(prm), _p(q), _p(k), _p(v), k.stride(0),
                                         v.stride(0), _p(sparse_idx), _p(n_sparse), _p(rows), _p(n_rows), q_pos0,
                                         n_query, n_key, _p(ctx_len), batch, _p(out), _p(lse)), "lsa_sparse_attn")
+
+    def append(self, k_new, k_idx, k_scale, kmean, page_table, ctx_len, ctx_len_out=None, kv_new=(), kv_pool=()):
+        batch = page_table.shape[0]
+        row_bytes = kv_pool[0].stride(0) * kv_pool[0].element_size() if len(kv_pool) else 0
+        self._chk(lib().lsa_append(self.h, ctypes.byref(self.params), _p(k_new), _p(k_idx), _p(k_scale), _p(kmean),
+                                   _p(page_table), page_table.shape[1], _p(ctx_len), batch, _p(ctx_len_out),
+                                   len(kv_pool), _parr(list(kv_new)) if len(kv_pool) else None,
+                                   _parr(list(kv_pool)) if len(kv_pool) else None, row_bytes), "lsa_append")
 
     def merge(self, outs, lses, n_query, out, lse=None, params=None):
         prm = params if params is not None else self.params

@@ -36,6 +36,7 @@ class LsaConfig:
     ctx_lo: int = 0      # decode: context length ~ U{ctx_lo..ctx_hi}
     ctx_hi: int = 0
     kv_page: int = 0     # decode: tokens per physical cache page
+    ctx_grow: int = 0    # decode: tokens each sequence can still append (pages mapped ahead)
     boost_prob: float = 0.0   # share of tokens whose indexer key is scaled by boost_gain
     boost_gain: float = 1.0
     segment_corr: float = 0.0  # share of an indexer key's variance that is common to its run of segment_len tokens

@@ -426,6 +426,34 @@ int lsa_block_means(lsa_ctx* c, const lsa_params* p, const void* k_idx, const fl
   return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
 }
 
+int lsa_append(lsa_ctx* c, const lsa_params* p, const void* k_new, void* k_idx, float* k_scale, void* kmean,
+               const int32_t* page_table, int64_t page_table_stride, const int32_t* ctx_len, int batch,
+               int32_t* ctx_len_out, int n_kv, const void* const* kv_new, void* const* kv_pool, int64_t kv_row_bytes) {
+  if (c == nullptr) return LSA_ERR_ARG;
+  int r = check_params(p, true, false);
+  if (r != LSA_OK) return r;
+  if (!p->paged || p->pooling != LSA_POOL_MEAN) return LSA_ERR_SHAPE;
+  if (k_new == nullptr || k_idx == nullptr || kmean == nullptr || page_table == nullptr || ctx_len == nullptr) return LSA_ERR_ARG;
+  if (batch < 0 || page_table_stride <= 0) return LSA_ERR_ARG;
+  if (p->key_dtype == LSA_KEY_E4M3 && k_scale == nullptr) return LSA_ERR_ARG;
+  if (n_kv < 0 || n_kv > 8) return LSA_ERR_ARG;
+  if (n_kv > 0 && (kv_new == nullptr || kv_pool == nullptr || kv_row_bytes <= 0 || kv_row_bytes % 16 != 0)) return LSA_ERR_ARG;
+  if (!aligned16(k_idx) || !aligned16(kmean) || !aligned16(k_new)) return LSA_ERR_SHAPE;
+  lsa::AppendArgs a{};
+  a.DI = p->d_idx; a.key_e4m3 = p->key_dtype == LSA_KEY_E4M3; a.B = p->sub_block; a.kv_page = p->kv_page;
+  a.batch = batch; a.n_kv = n_kv;
+  a.k_new = k_new; a.k_idx = k_idx; a.k_scale = k_scale; a.kmean = kmean;
+  a.page_table = page_table; a.pt_stride = page_table_stride; a.ctx_len = ctx_len; a.ctx_len_out = ctx_len_out;
+  for (int i = 0; i < n_kv; ++i) {
+    if (kv_new[i] == nullptr || kv_pool[i] == nullptr || !aligned16(kv_new[i]) || !aligned16(kv_pool[i])) return LSA_ERR_ARG;
+    a.kv_new[i] = kv_new[i];
+    a.kv_pool[i] = kv_pool[i];
+  }
+  a.kv_row_bytes = kv_row_bytes;
+  cudaError_t e = timed(c, LSA_K_MEANS, [&] { return lsa::launch_append(a, c->stream, &c->launches); });
+  return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
+}
+
 int lsa_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w, const void* k_idx,
               const float* k_scale, const void* kmean, int64_t q_pos0, int64_t n_query, int64_t n_key,
               const int32_t* page_table, int64_t page_table_stride, const int32_t* ctx_len, int batch,

@@ -793,6 +793,96 @@ __global__ void __launch_bounds__(kThreads) coarse_minmax_kernel(IndexArgs p) {
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Decode-step cache maintenance: store the new token's indexer key (quantised for e4m3 caches), recompute the
+// mean of its sub-block, copy the new rows of the attention caches.  One block per sequence, one thread per
+// 8 key dims for the mean (same accumulation order and arithmetic as block_means_kernel).
+// ------------------------------------------------------------------------------------------------
+constexpr int kAppendThreads = 128;
+
+__global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a) {
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const int DI = a.DI, U = DI / 8;
+  const int64_t pos = a.ctx_len[b];
+  const int64_t phys = a.page_table[b * a.pt_stride + pos / a.kv_page];
+  const int64_t row = phys * a.kv_page + pos % a.kv_page;
+  const __nv_bfloat16* kn = reinterpret_cast<const __nv_bfloat16*>(a.k_new) + static_cast<int64_t>(b) * DI;
+  __shared__ float red[kAppendThreads / 32];
+  __shared__ float s_scale;
+  if (a.key_e4m3) {
+    // per-token scale: amax / 448, then one code per dim
+    float amax = 0.f;
+    for (int d = tid; d < DI; d += kAppendThreads) amax = fmaxf(amax, fabsf(__bfloat162float(kn[d])));
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((tid & 31) == 0) red[tid >> 5] = amax;
+    __syncthreads();
+    if (tid == 0) {
+      float m = 0.f;
+      for (int i = 0; i < kAppendThreads / 32; ++i) m = fmaxf(m, red[i]);
+      const float sc = m > 0.f ? __fdiv_rn(m, 448.0f) : 1.0f;
+      s_scale = sc;
+      a.k_scale[row] = sc;
+    }
+    __syncthreads();
+    const float sc = s_scale;
+    uint8_t* dst = reinterpret_cast<uint8_t*>(a.k_idx) + row * DI;
+    for (int d = tid; d < DI; d += kAppendThreads)
+      dst[d] = static_cast<uint8_t>(__nv_cvt_float_to_fp8(__fdiv_rn(__bfloat162float(kn[d]), sc), __NV_SATFINITE, __NV_E4M3));
+  } else {
+    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.k_idx) + row * DI;
+    for (int d = tid; d < DI; d += kAppendThreads) dst[d] = kn[d];
+  }
+  // attention caches of the group's layers
+  for (int i = 0; i < a.n_kv; ++i) {
+    const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(a.kv_new[i]) + b * a.kv_row_bytes);
+    uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(a.kv_pool[i]) + row * a.kv_row_bytes);
+    for (int c = tid; c < a.kv_row_bytes / 16; c += kAppendThreads) dst[c] = src[c];
+  }
+  if (tid == 0 && a.ctx_len_out != nullptr) a.ctx_len_out[b] = static_cast<int32_t>(pos + 1);
+  __syncthreads();   // the new key is in the pool (this block wrote it): the mean reads it back like any other row
+  if (tid < U) {
+    const int u = tid;
+    const int64_t in_page = pos % a.kv_page;
+    const int64_t pos0 = pos - pos % a.B;                  // first token of the sub-block (B divides kv_page)
+    const int64_t row0 = row - (pos - pos0);
+    const int cnt = static_cast<int>(pos - pos0 + 1);
+    const int64_t out_row = phys * (a.kv_page / a.B) + in_page / a.B;
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int r = 0; r < cnt; ++r) {
+      const int64_t rr = row0 + r;
+      if (a.key_e4m3) {
+        const uint2 c = *reinterpret_cast<const uint2*>(reinterpret_cast<const uint8_t*>(a.k_idx) + rr * DI + u * 8);
+        const float sc = a.k_scale[rr];
+        const uint32_t w[2] = {c.x, c.y};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          __half2_raw h = __nv_cvt_fp8x2_to_halfraw2(
+              static_cast<__nv_fp8x2_storage_t>((w[j >> 1] >> ((j & 1) * 16)) & 0xffff), __NV_E4M3);
+          const float2 f = __half22float2(*reinterpret_cast<__half2*>(&h));
+          acc[2 * j] += f.x * sc;
+          acc[2 * j + 1] += f.y * sc;
+        }
+      } else {
+        const uint4 c = *reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(a.k_idx) + (rr * DI + u * 8) * 2);
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&c);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float2 f = __bfloat1622float2(h[j]);
+          acc[2 * j] += f.x;
+          acc[2 * j + 1] += f.y;
+        }
+      }
+    }
+    const float inv = static_cast<float>(cnt);
+    uint4 o;
+    o.x = pack_bf16(acc[0] / inv, acc[1] / inv);
+    o.y = pack_bf16(acc[2] / inv, acc[3] / inv);
+    o.z = pack_bf16(acc[4] / inv, acc[5] / inv);
+    o.w = pack_bf16(acc[6] / inv, acc[7] / inv);
+    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(a.kmean) + out_row * DI + u * 8) = o;
+  }
+}
+
 template <class K>
 cudaError_t set_smem(K kernel, size_t bytes) {
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
@@ -849,6 +939,13 @@ cudaError_t launch_coarse(const IndexArgs& a, cudaStream_t st, int64_t* n_launch
   if (coarse_paged_tc_supported(a)) return launch_coarse_paged_tc(a, st, n_launch);
   if (a.HI == 8 && a.DI == 64) return launch_coarse_t<8, 64>(a, n_key_max, st, n_launch);
   return launch_coarse_t<64, 128>(a, n_key_max, st, n_launch);
+}
+
+cudaError_t launch_append(const AppendArgs& a, cudaStream_t st, int64_t* n_launch) {
+  if (a.batch == 0) return cudaSuccess;
+  append_kernel<<<a.batch, kAppendThreads, 0, st>>>(a);
+  ++*n_launch;
+  return cudaGetLastError();
 }
 
 cudaError_t launch_block_minmax(int DI, int key_e4m3, int B, const void* k_idx, const float* k_scale, int64_t n_key,

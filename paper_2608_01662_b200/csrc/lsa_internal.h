@@ -60,6 +60,21 @@ struct AttnArgs {
 cudaError_t launch_block_means(int DI, int key_e4m3, int B, int kv_page, const void* k_idx, const float* k_scale,
                                int64_t n_key, const int32_t* page_table, int64_t pt_stride,
                                const int32_t* ctx_len, int batch, void* kmean, cudaStream_t st, int64_t* n_launch);
+struct AppendArgs {
+  int DI, key_e4m3, B, kv_page, batch, n_kv;
+  const void* k_new;        // bf16 [batch, DI]
+  void* k_idx;
+  float* k_scale;
+  void* kmean;
+  const int32_t* page_table;
+  int64_t pt_stride;
+  const int32_t* ctx_len;
+  int32_t* ctx_len_out;
+  const void* kv_new[8];
+  void* kv_pool[8];
+  int64_t kv_row_bytes;
+};
+cudaError_t launch_append(const AppendArgs& a, cudaStream_t st, int64_t* n_launch);
 cudaError_t launch_coarse(const IndexArgs& a, cudaStream_t st, int64_t* n_launch);
 // MinMax pooling (Eq. 13), contiguous caches: extrema cache [ceil(n_key/B), 2*DI] = [k_max | k_min], and the coarse stage on it
 cudaError_t launch_block_minmax(int DI, int key_e4m3, int B, const void* k_idx, const float* k_scale, int64_t n_key,

@@ -115,12 +115,12 @@ def decode_layout(cfg: LsaConfig, device):
     """(ctx_len int32 [batch], page_table int32 [batch, max_pages], n_phys_pages).
 
     Context lengths are uniform integers in [ctx_lo, ctx_hi]; the physical pages
-    are a random permutation dealt to the sequences in order; unused table
-    entries are -1.
+    are a random permutation dealt to the sequences in order (enough of them
+    for cfg.ctx_grow more tokens per sequence); unused table entries are -1.
     """
     g = _generator(cfg, T_CTX, 0, "cpu")
     ctx = torch.randint(cfg.ctx_lo, cfg.ctx_hi + 1, (cfg.batch,), generator=g, dtype=torch.int64)
-    n_pages = (ctx + cfg.kv_page - 1) // cfg.kv_page
+    n_pages = (ctx + cfg.ctx_grow + cfg.kv_page - 1) // cfg.kv_page   # room for ctx_grow appended tokens
     n_pg = int(n_pages.sum())
     perm = torch.randperm(n_pg, generator=_generator(cfg, T_PERM, 0, "cpu"))
     table = torch.full((cfg.batch, int(n_pages.max())), -1, dtype=torch.int32)

@@ -229,6 +229,76 @@ def test_convert_lists_physical_rows(cuda_device):
         assert r[3] <= n_sp + cfg.W // cfg.kv_page + 3
 
 
+# ---------------------------------------------------------------- decode-step cache maintenance
+def test_append_tokens_then_decode(cuda_device):
+    """37 decode steps of cache maintenance (crossing sub-block and page boundaries): the stored codes and scales are
+    the oracle's, the means equal both the oracle's and a rebuild by lsa_block_means, the attention rows land where
+    the page table says, and a decode step on the grown caches matches the oracle."""
+    n_add = 37
+    cfg = SMALL_DEC.replace(name="dec_append", ctx_grow=n_add + 3, R=2, seed=17)
+    wl = DecodeWorkload(cfg, cuda_device)
+    wl.prepare()
+    ctx0 = pu.to_np(wl.ctx_len).astype(np.int64)
+    table = pu.to_np(wl.page_table)
+    # oracle-side logical caches of every sequence, with room to grow
+    host = []
+    k_pool0, s_pool0 = pu.to_np(wl.keys["k"]), pu.to_np(wl.keys["scale"])
+    for b in range(cfg.batch):
+        n0 = int(ctx0[b])
+        rows = orc.paged_rows(np.arange(n0), table[b], cfg.kv_page)
+        codes = np.zeros((n0 + n_add, cfg.d_I), np.uint8)
+        scales = np.ones(n0 + n_add, np.float32)
+        codes[:n0], scales[:n0] = k_pool0[rows], s_pool0[rows]
+        km = np.zeros((-(-(n0 + n_add) // cfg.B), cfg.d_I))
+        km[:-(-n0 // cfg.B)] = orc.block_means(orc.dequant_keys(codes[:n0], scales[:n0]), cfg.B)
+        host.append([codes, scales, km, n0])
+    g = torch.Generator(device=cuda_device)
+    g.manual_seed(1234)
+    kv_rows = {}
+    for step in range(n_add):
+        k_new = (torch.randn((cfg.batch, cfg.d_I), generator=g, device=cuda_device) / math.sqrt(cfg.d_I)).to(torch.bfloat16)
+        if step == 5:
+            k_new[1] = 0                                   # a zero key: scale 1, codes 0
+        kv_new = [torch.randn((cfg.batch, cfg.d_qk), generator=g, device=cuda_device).to(torch.bfloat16) for _ in range(cfg.R)]
+        wl.ctx.append(k_new, wl.keys["k"], wl.keys["scale"], wl.kmean, wl.page_table, wl.ctx_len, wl.ctx_len, kv_new, wl.k)
+        kn = pu.to_np(k_new)
+        for b in range(cfg.batch):
+            h = host[b]
+            kv_rows[(b, h[3])] = [pu.to_np(x[b]) for x in kv_new]
+            h[3] = orc.append_token(h[0], h[1], h[2], h[3], kn[b], cfg.B)
+    assert wl.ctx.status() == 0
+    assert np.array_equal(pu.to_np(wl.ctx_len), ctx0 + n_add)
+    k_pool, s_pool, km_pool = pu.to_np(wl.keys["k"]), pu.to_np(wl.keys["scale"]), pu.to_np(wl.kmean).astype(np.float64)
+    # a rebuild of the mean cache from the grown pools
+    km2 = torch.zeros_like(wl.kmean)
+    wl.ctx.block_means(wl.keys["k"], wl.keys.get("scale"), 0, km2, wl.page_table, wl.ctx_len)
+    km2 = pu.to_np(km2).astype(np.float64)
+    spp_kv = cfg.kv_page // cfg.B
+    n_diff = n_tot = 0
+    for b in range(cfg.batch):
+        codes, scales, km, n = host[b]
+        rows = orc.paged_rows(np.arange(n), table[b], cfg.kv_page)
+        assert np.array_equal(k_pool[rows], codes[:n]) and np.array_equal(s_pool[rows], scales[:n])
+        subs = np.arange(-(-n // cfg.B))
+        mrows = table[b][subs * cfg.B // cfg.kv_page].astype(np.int64) * spp_kv + (subs * cfg.B % cfg.kv_page) // cfg.B
+        assert np.array_equal(km_pool[mrows], km2[mrows])                    # appended == rebuilt, bit for bit
+        d = np.abs(km_pool[mrows] - km[:len(subs)])
+        # fp32 against fp64 accumulation: at most one bf16 ulp of the mean, or the fp32 error of the sum when it cancels
+        assert (d <= np.abs(km[:len(subs)]) * 2.0 ** -7 + 1e-6).all()
+        n_diff += int((d > 0).sum())
+        n_tot += d.size
+        for pos in range(int(ctx0[b]), n):
+            r = int(orc.paged_rows(np.array([pos]), table[b], cfg.kv_page)[0])
+            for layer in range(cfg.R):
+                assert np.array_equal(pu.to_np(wl.k[layer][r]), kv_rows[(b, pos)][layer])
+    assert n_diff < 0.005 * n_tot
+    wl.step()
+    assert wl.ctx.status() == 0
+    m = pu.check_decode(wl, range(cfg.batch))
+    print(cfg.name, m.summary())
+    m.assert_ok(pu.TOL_FP8)
+
+
 # ---------------------------------------------------------------- MinMax pooling (Eq. 13)
 @pytest.mark.parametrize("base", ["fp8", "bf16"])
 def test_minmax_cache_and_selection(cuda_device, base):
