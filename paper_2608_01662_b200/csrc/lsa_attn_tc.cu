@@ -253,7 +253,11 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     // ================= MMA issuers =================
     const int x = warp - kSoftmaxWarps;   // 0..3
     if (lane == 0 && n_tiles > 0) {
+#ifdef LSA_DBG_QKN
+      constexpr uint32_t idesc_qk = tc::idesc_bf16(kH, LSA_DBG_QKN, 0, 0);   // timing experiment only: wrong results
+#else
       constexpr uint32_t idesc_qk = tc::idesc_bf16(kH, kTileKeys, 0, 0);
+#endif
       constexpr uint32_t idesc_pv = tc::idesc_bf16(kH, 128, 0, 1);   // B = V read MN-major
       bool ok = tc::mbar_wait(smem_u32(&sm.q_full), 0, p.status) && tc::mbar_wait(smem_u32(&sm.q_tmem), 0, p.status);
       if (x == 0) LSA_TL(2);
@@ -281,6 +285,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
 #pragma unroll
         for (int s = 0; s < 2; ++s)    // rope dims 512 + 32x + 16s .. +15
           tc::umma_ss(d, tc::desc_advance(dqr, (2 * x + s) * 32), tc::desc_advance(dkb, 8 * kAtomBytes + (2 * x + s) * 32), idesc_qk, 1);
+        if (x == 0 && i == 22) LSA_TL(9);
         tc::umma_commit(smem_u32(&sm.s_full[i & 1]));
       };
       auto issue_pv = [&](int j) {   // O[:, 128x : 128x+128] += P_j V_j
@@ -304,6 +309,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
           if (tc::mbar_test(smem_u32(&sm.k_full[qk_next % kKBufs]), (qk_next / kKBufs) & 1) &&
               tc::mbar_test(smem_u32(&sm.pv_done[qk_next & 1]), ((qk_next >> 1) & 1) ^ 1)) {
             if (x == 0 && qk_next == 0) LSA_TL(3);
+            if (x == 0 && qk_next == 22) LSA_TL(15);
             issue_qk(qk_next++);
             did = true;
           }
@@ -359,6 +365,8 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.s_full[b]), (i >> 1) & 1, p.status));
       if (!ok) break;
       if (tid == 0 && i == 0) LSA_TL(4);
+      if (tid == 0 && i == 20) LSA_TL(10);
+      if (tid == 0 && i == 21) LSA_TL(14);
       tc::fence_after_sync();
       const uint32_t s_addr = tmem_base + lane_addr + kColS + b * kSBuf;
       uint32_t v[32];
@@ -375,6 +383,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
           v[j] = __float_as_uint(keep + __shfl_xor_sync(0xffffffffu, give, 16));
         }
       }
+      if (tid == 0 && i == 20) LSA_TL(11);
       // logits in log2 units, ragged tail masked
       const int n_valid = n_tot - (tile_begin + i) * kTileKeys - kHalfKeys * hi;   // keys of this lane's half that exist
       float mx = -INFINITY;
@@ -422,6 +431,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
         pk[j] = pack_bf16(p0, p1);
       }
       l_run += sum;
+      if (tid == 0 && i == 20) LSA_TL(12);
       {
         // The A operand of P V sits in tensor memory, in the lanes of the accumulator it feeds: both lanes of a
         // row need all 64 keys, so the two halves are swapped in, then written as 32 columns of packed bf16.
@@ -438,6 +448,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       }
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(smem_u32(&sm.p_ready[b]));
+      if (tid == 0 && i == 20) LSA_TL(13);
     }
     if (tid == 0) LSA_TL(5);
     // ---- epilogue: O / l
