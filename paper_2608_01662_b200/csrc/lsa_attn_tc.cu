@@ -69,6 +69,11 @@ constexpr int kAtomBytes = 64 * 128;         // 64 rows x 128 bytes
 constexpr int kHalfKeys = 32;
 
 constexpr int kSoftmaxWarps = 4, kMmaWarps = 4, kLoadWarps = 4;
+#ifndef LSA_PV_ISSUERS
+#define LSA_PV_ISSUERS 4
+#endif
+constexpr int kPvIssuers = LSA_PV_ISSUERS;   // 4: one per 128 value dims; 2: one per 256 (N = 256 MMAs; measured 6 % slower:
+                                             // an M = 64 MMA of N = 256 takes twice the time of N = 128, and two threads issue everything)
 constexpr int kThreadsAttnTc = 32 * (kSoftmaxWarps + kMmaWarps + kLoadWarps);
 constexpr uint32_t kTmemColsAttn = 512;
 constexpr int kKBufs = 3;                    // 64-key tile buffers in shared memory
@@ -116,11 +121,11 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     tc::mbar_init(smem_u32(&sm.q_tmem), kSoftmaxWarps);
     for (int b = 0; b < kKBufs; ++b) {
       tc::mbar_init(smem_u32(&sm.k_full[b]), 32 * kLoadWarps);
-      tc::mbar_init(smem_u32(&sm.k_empty[b]), kMmaWarps);
+      tc::mbar_init(smem_u32(&sm.k_empty[b]), kPvIssuers);
     }
     for (int b = 0; b < 2; ++b) {
       tc::mbar_init(smem_u32(&sm.s_full[b]), 2);
-      tc::mbar_init(smem_u32(&sm.pv_done[b]), kMmaWarps);
+      tc::mbar_init(smem_u32(&sm.pv_done[b]), kPvIssuers);
       tc::mbar_init(smem_u32(&sm.p_ready[b]), kSoftmaxWarps);
     }
     tc::fence_mbar_init();
@@ -258,14 +263,14 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
 #else
       constexpr uint32_t idesc_qk = tc::idesc_bf16(kH, kTileKeys, 0, 0);
 #endif
-      constexpr uint32_t idesc_pv = tc::idesc_bf16(kH, 128, 0, 1);   // B = V read MN-major
+      constexpr uint32_t idesc_pv = tc::idesc_bf16(kH, kPvIssuers == 4 ? 128 : 256, 0, 1);   // B = V read MN-major
       bool ok = tc::mbar_wait(smem_u32(&sm.q_full), 0, p.status) && tc::mbar_wait(smem_u32(&sm.q_tmem), 0, p.status);
       if (x == 0) LSA_TL(2);
       // Descriptors are built once; inside the loops only the start-address word moves (one add per operand).
       constexpr uint32_t kBufBytes = kAtoms * kAtomBytes;
       const uint64_t dqr = tc::smem_desc_sw128(smem_u32(sm.q_rope), 16, 1024);
       const uint64_t dk0 = tc::smem_desc_sw128(smem_u32(sm.k), 16, 1024);           // K-major view (Q K^T)
-      const uint64_t dv0 = tc::desc_advance(tc::smem_desc_sw128(smem_u32(sm.k), kAtomBytes, 1024), 2 * x * kAtomBytes);  // MN-major view (P V)
+      const uint64_t dv0 = tc::desc_advance(tc::smem_desc_sw128(smem_u32(sm.k), kAtomBytes, 1024), (kPvIssuers == 4 ? 2 : 4) * x * kAtomBytes);  // MN-major view (P V)
       constexpr uint32_t kLane16 = 16u << 16;
       // Q K^T (issuers 0 and 1): chain x = dims 256x .. 256x+255 with Q from tensor memory (lane half x), plus two of
       // the four rope steps with Q from shared memory; its partial sum goes to lane half x of the S buffer
@@ -273,8 +278,8 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       const uint32_t s_dst = tmem_base + (x & 1) * kLane16 + kColS;
       // P V (all four issuers): value dims 128x .. 128x+127 = columns 128*(x&1) .. of the accumulator in lane half
       // x>>1; P is read from the same lane half
-      const uint32_t o_dst = tmem_base + (x >> 1) * kLane16 + (x & 1) * 128;
-      const uint32_t p_src = tmem_base + (x >> 1) * kLane16 + kColS;
+      const uint32_t o_dst = kPvIssuers == 4 ? tmem_base + (x >> 1) * kLane16 + (x & 1) * 128 : tmem_base + (x & 1) * kLane16;
+      const uint32_t p_src = tmem_base + (kPvIssuers == 4 ? (x >> 1) : (x & 1)) * kLane16 + kColS;
       auto issue_qk = [&](int i) {
         tc::fence_after_sync();
         const uint32_t d = s_dst + (i & 1) * kSBuf;
@@ -299,7 +304,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       };
       const bool does_qk = x < 2;
       // Two in-order queues, "next Q K^T" (at most one tile ahead of the softmax it feeds) and "next P V".
-      int qk_next = does_qk ? 0 : n_tiles, pv_next = 0;
+      int qk_next = does_qk ? 0 : n_tiles, pv_next = x < kPvIssuers ? 0 : n_tiles;
       long long t_idle = clock64();
       uint32_t spins = 0;
       while (ok && pv_next < n_tiles) {
