@@ -345,12 +345,24 @@ def main():
                    "l2": "inputs larger than L2 (per-layer q and out are GBs); no flush" if not decode
                          else "KV pools are GBs per layer, far larger than L2; no flush"},
         "clocks": clocks.summary(), "gpu_launches": int(launches), "kernels": kernels,
-        "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "decode": decode_line,
+        "roofline": with_nominal(roofline), "e2e": e2e, "cpu_baseline": cpu, "decode": decode_line,
     }
     print(json.dumps(line))
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+NOMINAL_BF16_TFLOPS, NOMINAL_HBM_GBS = 2250.0, 8000.0   # dense bf16 and HBM3e data-sheet figures, for context
+
+
+def with_nominal(roofline):
+    """Adds the fraction of the nominal (data-sheet) peak beside the fraction of the measured one."""
+    if roofline is not None:
+        nominal = NOMINAL_HBM_GBS if roofline["bound"] == "hbm" else NOMINAL_BF16_TFLOPS
+        roofline["peak_nominal"] = nominal
+        roofline["frac_of_nominal"] = roofline["achieved"] / nominal
+    return roofline
 
 
 def decode_attn_launch_us(wl, rounds=10):
@@ -433,10 +445,10 @@ def measure_decode(cfg, dev, peaks, steps=50, warmup=10):
             "config": {"workload": cfg.name, "batch": cfg.batch, "R": cfg.R, "ctx": [cfg.ctx_lo, cfg.ctx_hi],
                        "l2": "KV pools are GBs per layer, far larger than L2; no flush"},
             "kernels_us_per_step": {k: v[0] / steps * 1e3 for k, v in prof.items() if v[1] > 0},
-            "roofline": {"kernel": "sparse_attn_tc_kernel", "bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"],
-                         "unit": "GB/s", "frac": a / peaks["hbm_gbs"], "traffic": None,
-                         "peak_source": peaks["source"], "launch_us": attn_us,
-                         "timing": "one event pair around 10 x R back-to-back launches"},
+            "roofline": with_nominal({"kernel": "sparse_attn_tc_kernel", "bound": "hbm", "achieved": a,
+                                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": a / peaks["hbm_gbs"],
+                                      "traffic": None, "peak_source": peaks["source"], "launch_us": attn_us,
+                                      "timing": "one event pair around 10 x R back-to-back launches"}),
             "running_loop": running}
 
 
