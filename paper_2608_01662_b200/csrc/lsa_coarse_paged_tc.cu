@@ -84,6 +84,8 @@ coarse_score_paged_tc_kernel(const __grid_constant__ CUtensorMap map_km, const _
   const int spp = p.P / p.B;                       // sub-blocks per page: 8, 16 or 32
   sh.spp_shift = 31 - __clz(spp);
   if (tc::status_raised(p.status)) return;
+  pdl_wait();                 // the cached lengths may come from the previous kernel of the stream (lsa_append)
+  pdl_launch_dependents();
 
   // ---- this block's share of the tile list
   int my_tiles = 0;
@@ -317,9 +319,9 @@ cudaError_t launch_coarse_paged_tc(const IndexArgs& a, cudaStream_t st, int64_t*
   int64_t blocks = 2 * sm_count_of_current_device();
   if (blocks > max_tiles) blocks = max_tiles;
   if (blocks < 1) blocks = 1;
-  coarse_score_paged_tc_kernel<<<static_cast<unsigned>(blocks), kThreadsCp, smem, st>>>(map_km, map_q, a);
+  e = launch_pdl(coarse_score_paged_tc_kernel, dim3(static_cast<unsigned>(blocks)), dim3(kThreadsCp), smem, st, map_km, map_q, a);
   ++*n_launch;
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace lsa

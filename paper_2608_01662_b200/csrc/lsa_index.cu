@@ -348,6 +348,8 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
   auto& sm = *reinterpret_cast<FineSmem<HI, DI>*>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int qi = blockIdx.x;
+  pdl_wait();
+  pdl_launch_dependents();
   int64_t t, n_key;
   const int32_t* pt = nullptr;
   if (p.paged) {
@@ -519,6 +521,8 @@ __global__ void __launch_bounds__(kSelThreads) fine_topk_kernel(IndexArgs p) {
   __shared__ int32_t pages[kMaxPages];
   __shared__ SelectScratch sc;
   const int qi = blockIdx.x, tid = threadIdx.x;
+  pdl_wait();
+  pdl_launch_dependents();
   const int32_t* fp = p.fine_pages + qi * (kMaxPages + 1);
   const int nP = fp[kMaxPages];
   if (nP == 0) return;   // no candidates: the scoring kernel has written the empty result
@@ -585,6 +589,8 @@ __global__ void __launch_bounds__(kConvertThreads) convert_kernel(int S, int W, 
                                                      int32_t* __restrict__ rows_out, int32_t* __restrict__ n_rows_out,
                                                      int32_t* __restrict__ runs_out) {
   const int qi = blockIdx.x, tid = threadIdx.x;
+  pdl_wait();
+  pdl_launch_dependents();
   const int64_t t = paged ? ctx_len[qi] - 1 : q_pos0 + qi;
   const int32_t* pt = paged ? page_table + qi * pt_stride : nullptr;
   const int n_sink = static_cast<int>(min64(S, t + 1));
@@ -803,6 +809,8 @@ constexpr int kAppendThreads = 128;
 __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a) {
   const int b = blockIdx.x, tid = threadIdx.x;
   const int DI = a.DI, U = DI / 8;
+  pdl_wait();
+  pdl_launch_dependents();
   const int64_t pos = a.ctx_len[b];
   const int64_t phys = a.page_table[b * a.pt_stride + pos / a.kv_page];
   const int64_t row = phys * a.kv_page + pos % a.kv_page;
@@ -943,9 +951,9 @@ cudaError_t launch_coarse(const IndexArgs& a, cudaStream_t st, int64_t* n_launch
 
 cudaError_t launch_append(const AppendArgs& a, cudaStream_t st, int64_t* n_launch) {
   if (a.batch == 0) return cudaSuccess;
-  append_kernel<<<a.batch, kAppendThreads, 0, st>>>(a);
+  const cudaError_t e = launch_pdl(append_kernel, dim3(a.batch), dim3(kAppendThreads), 0, st, a);
   ++*n_launch;
-  return cudaGetLastError();
+  return e;
 }
 
 cudaError_t launch_block_minmax(int DI, int key_e4m3, int B, const void* k_idx, const float* k_scale, int64_t n_key,
@@ -989,11 +997,13 @@ static cudaError_t launch_fine_t(const IndexArgs& a, cudaStream_t st, int64_t* n
   cudaError_t e = set_smem(fine_select_kernel<HI, DI, E4M3>, smem);
   if (e != cudaSuccess) return e;
   const int parts = a.fine_parts > 1 ? a.fine_parts : 1;
-  fine_select_kernel<HI, DI, E4M3><<<dim3(a.n_query, parts), kThreads, smem, st>>>(a);
+  e = launch_pdl(fine_select_kernel<HI, DI, E4M3>, dim3(a.n_query, parts), dim3(kThreads), smem, st, a);
+  if (e != cudaSuccess) return e;
   ++*n_launch;
   e = cudaGetLastError();
   if (e != cudaSuccess || parts == 1) return e;
-  fine_topk_kernel<<<a.n_query, kSelThreads, 0, st>>>(a);
+  e = launch_pdl(fine_topk_kernel, dim3(a.n_query), dim3(kSelThreads), 0, st, a);
+  if (e != cudaSuccess) return e;
   ++*n_launch;
   return cudaGetLastError();
 }
@@ -1003,7 +1013,8 @@ cudaError_t launch_fine_select(const IndexArgs& a, cudaStream_t st, int64_t* n_l
   if (fine_tc_supported(a)) {
     cudaError_t e = launch_fine_select_tc(a, st, n_launch);
     if (e != cudaSuccess || a.fine_parts <= 1) return e;
-    fine_topk_kernel<<<a.n_query, kSelThreads, 0, st>>>(a);
+    e = launch_pdl(fine_topk_kernel, dim3(a.n_query), dim3(kSelThreads), 0, st, a);
+    if (e != cudaSuccess) return e;
     ++*n_launch;
     return cudaGetLastError();
   }
@@ -1036,10 +1047,10 @@ cudaError_t launch_convert(int S, int W, int Ksp, int paged, int kv_page, const 
                            int64_t pt_stride, const int32_t* ctx_len, int32_t* rows_out, int32_t* n_rows_out,
                            int32_t* runs_out, cudaStream_t st, int64_t* n_launch) {
   if (n_query == 0) return cudaSuccess;
-  convert_kernel<<<n_query, kConvertThreads, 0, st>>>(S, W, Ksp, paged, kv_page, sparse_idx, n_sparse, q_pos0, page_table,
-                                          pt_stride, ctx_len, rows_out, n_rows_out, runs_out);
+  const cudaError_t e = launch_pdl(convert_kernel, dim3(n_query), dim3(kConvertThreads), 0, st, S, W, Ksp, paged, kv_page, sparse_idx,
+                                   n_sparse, q_pos0, page_table, pt_stride, ctx_len, rows_out, n_rows_out, runs_out);
   ++*n_launch;
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace lsa
