@@ -152,7 +152,8 @@ int pick_split(int sm_count, int batch, int max_rows, bool tc_kernel) {
 int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w, const void* k_idx,
               const float* k_scale, const void* kmean, int64_t q_pos0, int64_t n_query, int64_t n_key,
               const int32_t* page_table, int64_t pt_stride, const int32_t* ctx_len, int batch,
-              int32_t* sparse_idx, int32_t* n_sparse, int32_t* pages_out) {
+              int32_t* sparse_idx, int32_t* n_sparse, int32_t* pages_out, int32_t* rows_out = nullptr,
+              int32_t* n_rows_out = nullptr) {
   const int64_t nq = p->paged ? batch : n_query;
   if (nq == 0) return LSA_OK;
   const int64_t n_key_max = p->paged ? pt_stride * p->kv_page : n_key;
@@ -175,6 +176,8 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
     a.page_scores = reinterpret_cast<float*>(c->ws + l.page_scores); a.ps_ld = l.ps_ld;
     a.sparse_idx = sparse_idx + q0 * p->k_sparse; a.n_sparse = n_sparse + q0;
     a.pages_out = pages_out ? pages_out + q0 * p->keep_pages : nullptr;
+    a.rows_out = p->paged ? rows_out : nullptr;   // a5 fused into the last selection kernel (decode)
+    a.n_rows_out = n_rows_out;
     a.status = status_word(c);
     a.fine_parts = 1;
     if (p->paged) {
@@ -230,6 +233,13 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
                                            : lsa::launch_coarse(a, c->stream, &c->launches);
       });
     if (e == cudaSuccess) e = timed(c, LSA_K_FINE_SELECT, [&] { return lsa::launch_fine_select(a, c->stream, &c->launches); });
+    if (e == cudaSuccess && a.rows_out != nullptr && a.fine_parts <= 1)
+      // only the split fine stage writes the cache rows itself (in its top-K kernel)
+      e = timed(c, LSA_K_CONVERT, [&] {
+        return lsa::launch_convert(p->k_sink, p->k_swa, p->k_sparse, p->paged, p->kv_page, a.sparse_idx, a.n_sparse, a.q_pos0,
+                                   a.n_query, page_table, pt_stride, ctx_len, a.rows_out, a.n_rows_out, nullptr, c->stream,
+                                   &c->launches);
+      });
     if (e != cudaSuccess) return cuda_fail(c, e);
   }
   return LSA_OK;
@@ -454,10 +464,12 @@ int lsa_append(lsa_ctx* c, const lsa_params* p, const void* k_new, void* k_idx, 
   return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
 }
 
-int lsa_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w, const void* k_idx,
-              const float* k_scale, const void* kmean, int64_t q_pos0, int64_t n_query, int64_t n_key,
-              const int32_t* page_table, int64_t page_table_stride, const int32_t* ctx_len, int batch,
-              int32_t* sparse_idx, int32_t* n_sparse, int32_t* pages_out) {
+// lsa_index with its argument checks; rows_out / n_rows_out (paged caches): also write what lsa_convert would
+static int index_checked(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w, const void* k_idx,
+                         const float* k_scale, const void* kmean, int64_t q_pos0, int64_t n_query, int64_t n_key,
+                         const int32_t* page_table, int64_t page_table_stride, const int32_t* ctx_len, int batch,
+                         int32_t* sparse_idx, int32_t* n_sparse, int32_t* pages_out, int32_t* rows_out,
+                         int32_t* n_rows_out) {
   if (c == nullptr) return LSA_ERR_ARG;
   int r = check_params(p, true, false);
   if (r != LSA_OK) return r;
@@ -472,7 +484,15 @@ int lsa_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
   }
   if (!aligned16(q_idx) || !aligned16(w) || !aligned16(k_idx) || (kmean && !aligned16(kmean))) return LSA_ERR_SHAPE;
   return run_index(c, p, q_idx, w, k_idx, k_scale, kmean, q_pos0, n_query, n_key, page_table, page_table_stride,
-                   ctx_len, batch, sparse_idx, n_sparse, pages_out);
+                   ctx_len, batch, sparse_idx, n_sparse, pages_out, rows_out, n_rows_out);
+}
+
+int lsa_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w, const void* k_idx,
+              const float* k_scale, const void* kmean, int64_t q_pos0, int64_t n_query, int64_t n_key,
+              const int32_t* page_table, int64_t page_table_stride, const int32_t* ctx_len, int batch,
+              int32_t* sparse_idx, int32_t* n_sparse, int32_t* pages_out) {
+  return index_checked(c, p, q_idx, w, k_idx, k_scale, kmean, q_pos0, n_query, n_key, page_table, page_table_stride,
+                       ctx_len, batch, sparse_idx, n_sparse, pages_out, nullptr, nullptr);
 }
 
 int lsa_select(lsa_ctx* c, const lsa_params* p, const float* scores, int64_t ld_scores, const int32_t* cand_pos,
@@ -551,22 +571,19 @@ int lsa_layer_group(lsa_ctx* c, const lsa_params* p, const void* q_idx, const fl
   if (p->n_layers <= 0 || q == nullptr || k == nullptr || v == nullptr || out == nullptr) return LSA_ERR_ARG;
   for (int i = 0; i < p->n_layers; ++i)
     if (q[i] == nullptr || k[i] == nullptr || v[i] == nullptr || out[i] == nullptr) return LSA_ERR_ARG;
-  r = lsa_index(c, p, q_idx, w, k_idx, k_scale, kmean, q_pos0, n_query, n_key, page_table, page_table_stride,
-                ctx_len, batch, sparse_idx, n_sparse, nullptr);
-  if (r != LSA_OK) return r;
-  const int32_t* rows = nullptr;
-  const int32_t* n_rows = nullptr;
+  // paged caches: the index -> cache-row conversion (a5) rides in the indexer's last kernel
+  int32_t* rows = nullptr;
+  int32_t* n_rows = nullptr;
   if (p->paged) {
+    if (page_table_stride <= 0 || batch <= 0) return LSA_ERR_ARG;
     const WsLayout l = ws_layout(p, batch, page_table_stride * p->kv_page, batch);
     if (c->ws == nullptr || l.total > c->ws_bytes) return LSA_ERR_WORKSPACE;
-    int32_t* rows_w = reinterpret_cast<int32_t*>(c->ws + l.rows);
-    int32_t* n_rows_w = reinterpret_cast<int32_t*>(c->ws + l.n_rows);
-    r = lsa_convert(c, p, sparse_idx, n_sparse, q_pos0, n_query, page_table, page_table_stride, ctx_len, batch,
-                    rows_w, n_rows_w, nullptr);
-    if (r != LSA_OK) return r;
-    rows = rows_w;
-    n_rows = n_rows_w;
+    rows = reinterpret_cast<int32_t*>(c->ws + l.rows);
+    n_rows = reinterpret_cast<int32_t*>(c->ws + l.n_rows);
   }
+  r = index_checked(c, p, q_idx, w, k_idx, k_scale, kmean, q_pos0, n_query, n_key, page_table, page_table_stride,
+                    ctx_len, batch, sparse_idx, n_sparse, nullptr, rows, n_rows);
+  if (r != LSA_OK) return r;
   for (int i = 0; i < p->n_layers; ++i) {
     r = lsa_sparse_attn(c, p, q[i], k[i], v[i], ld_k, ld_v, sparse_idx, n_sparse, rows, n_rows, q_pos0, n_query,
                         n_key, ctx_len, batch, out[i], lse ? lse[i] : nullptr);

@@ -25,6 +25,9 @@ struct IndexArgs {
   int32_t* sparse_idx;    // [n_query, Ksp]
   int32_t* n_sparse;
   int32_t* pages_out;     // optional [n_query, M]
+  // optional, paged caches: a5 fused into the last selection kernel (what lsa_convert would write)
+  int32_t* rows_out;      // [n_query, S + Ksp + W] physical cache rows, -1 padded
+  int32_t* n_rows_out;    // [n_query]
   // split fine stage (few queries, many SMs): the scoring blocks leave their results here for the top-K kernel
   int fine_parts;         // 1: fused kernel; >1: blocks per query in the scoring kernel
   uint32_t* fine_keys;    // [n_query, 4096] order-preserving keys of the candidate slots (0 = not a candidate)

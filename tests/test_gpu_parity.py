@@ -193,6 +193,19 @@ def test_paged_decode_row_splits(cuda_device, n_split):
     m.assert_ok(pu.TOL_FP8)
 
 
+def test_paged_decode_large_batch(cuda_device):
+    """More sequences than twice the SM count: the fine stage runs unsplit (one block per sequence selects by itself)
+    and the cache rows come from the separate conversion kernel."""
+    cfg = SMALL_DEC.replace(name="dec_wide", batch=320, ctx_lo=700, ctx_hi=1600, M=8, Ksp=256, R=1, seed=19)
+    wl = DecodeWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.step()
+    assert wl.ctx.status() == 0
+    m = pu.check_decode(wl, [0, 1, 17, 150, 318, 319])
+    print(cfg.name, m.summary())
+    m.assert_ok(pu.TOL_FP8)
+
+
 def test_decode_split_count_is_checked(cuda_device):
     cfg = SMALL_DEC
     if cfg.H != 64:
