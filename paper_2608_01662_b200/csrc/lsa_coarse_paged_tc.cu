@@ -6,10 +6,11 @@
 // 2 x SM-count resident blocks takes an equal contiguous share of it (every block derives the same partition from the
 // cached lengths; nothing is scheduled dynamically).  Inside a block:
 //
-//   warp 0      producer: for each tile, looks up the physical page of each of its logical pages and issues one TMA box
+//   warps 0, 6-8  producers: for each tile, look up the physical page of each of its logical pages and issue one TMA box
 //               per page and 64-dim half (the sub-blocks of a page are consecutive rows of the mean cache) into a
-//               two-deep ring; when its share crosses into the next sequence, fetches that sequence's query heads
-//               (TMA) and head weights into the other of two query slots
+//               two-deep ring.  A box is 1 KB and a TMA instruction costs its issuing warp some eighty cycles, so the
+//               32 boxes of a tile are spread over four warps.  When the block's share crosses into the next sequence,
+//               warp 0 fetches that sequence's query heads (TMA) and head weights into the other of two query slots
 //   warp 1      one thread issues 8 x tcgen05.mma (M128 N64 K16) per tile into one of two TMEM accumulators
 //   warps 2-5   epilogue: one thread = one sub-block row: sum_j w_j relu(acc_j), then the sum over the page's
 //               sub-blocks (Eq. 9) with warp shuffles, page score to global
@@ -25,7 +26,8 @@ constexpr int kTile = 128;                  // sub-block rows per tile
 constexpr int kAtomA = kTile * 128;         // one 64-dim column block of a tile
 constexpr int kAtomQ = kHI * 128;
 constexpr int kStages = 2;                  // two blocks share an SM: four tiles (128 KB) in flight per SM
-constexpr int kThreadsCp = 192;
+constexpr int kThreadsCp = 288;             // warps 0, 6, 7, 8: producers; 1: MMA; 2-5: epilogue
+constexpr int kProducerWarps = 4;
 constexpr int kMaxBatchCp = 2048;           // cached lengths kept in shared memory
 constexpr uint32_t kTmemColsCp = 128;       // two accumulators of 64 columns
 
@@ -152,16 +154,20 @@ coarse_score_paged_tc_kernel(const __grid_constant__ CUtensorMap map_km, const _
   Walker wk;
   wk.start(sm.ctx, sh, sm.first_seq, sm.first_tile);
 
-  if (warp == 0) {
-    // ================= producer =================
+  const int pw = warp == 0 ? 0 : warp - 5;   // producer number of warps 0, 6, 7, 8
+  if (warp == 0 || warp >= 6) {
+    // ================= producers =================
     const int pages_per_tile = kTile >> sh.spp_shift;    // 16, 8 or 4
     const int n_loads = pages_per_tile * 2;              // one box per page and 64-dim half
+    const int per_warp = n_loads / kProducerWarps;       // 8, 4 or 2 boxes per producer warp
+    const int box = pw * per_warp + lane;                // the box this lane issues (lanes below per_warp)
+    const bool issues = lane < per_warp;
     const int box_bytes = spp * 128;
     auto first_row = [&](int seq, int tile) -> int {     // physical row of the box this lane fetches
       const int n_sub = (sm.ctx[seq] + sh.B - 1) / sh.B;
-      const int sub0 = tile * kTile + ((lane >> 1) << sh.spp_shift);
+      const int sub0 = tile * kTile + ((box >> 1) << sh.spp_shift);
       // pages past the cached length are never eligible: any mapped rows will do, the epilogue drops them
-      return (lane < n_loads && sub0 < n_sub) ? p.page_table[seq * p.pt_stride + (sub0 >> sh.spp_shift)] << sh.spp_shift : 0;
+      return (issues && sub0 < n_sub) ? p.page_table[seq * p.pt_stride + (sub0 >> sh.spp_shift)] << sh.spp_shift : 0;
     };
     int n_q = 0;
     bool new_seq = true;
@@ -174,7 +180,7 @@ coarse_score_paged_tc_kernel(const __grid_constant__ CUtensorMap map_km, const _
       new_seq = wk.next(sm.ctx, sh, batch);
       if (i + 1 < n_tiles) row_next = first_row(wk.seq, wk.tile);   // look-ups of the next tile: off the critical path
       bool ok = true;
-      if (was_new) {
+      if (was_new && pw == 0) {
         // query heads and head weights of this sequence into slot n_q & 1
         const int slot = n_q & 1;
         if (lane == 0) ok = tc::mbar_wait(smem_u32(&sm.q_empty[slot]), ((n_q >> 1) & 1) ^ 1, p.status);
@@ -191,11 +197,12 @@ coarse_score_paged_tc_kernel(const __grid_constant__ CUtensorMap map_km, const _
       }
       if (lane == 0) {
         ok = tc::mbar_wait(smem_u32(&sm.empty[s]), ((i / kStages) & 1) ^ 1, p.status);
-        if (ok) tc::mbar_expect_tx(smem_u32(&sm.full[s]), 2 * kAtomA);
+        // one arrival per tile, by producer 0; bytes the other producers' boxes complete before it are counted all the same
+        if (ok && pw == 0) tc::mbar_expect_tx(smem_u32(&sm.full[s]), 2 * kAtomA);
       }
       if (!__shfl_sync(0xffffffffu, ok, 0)) break;
-      if (lane < n_loads)
-        tc::tma_load_2d(smem_u32(sm.a[s][lane & 1]) + (lane >> 1) * box_bytes, &map_km, (lane & 1) * 64, row, smem_u32(&sm.full[s]));
+      if (issues)
+        tc::tma_load_2d(smem_u32(sm.a[s][box & 1]) + (box >> 1) * box_bytes, &map_km, (box & 1) * 64, row, smem_u32(&sm.full[s]));
     }
   } else if (warp == 1) {
     // ================= MMA issuer =================
@@ -227,7 +234,7 @@ coarse_score_paged_tc_kernel(const __grid_constant__ CUtensorMap map_km, const _
         if (new_seq || i + 1 == n_tiles) tc::umma_commit(smem_u32(&sm.q_empty[slot]));   // last tile of its sequence here
       }
     }
-  } else {
+  } else if (warp < 6) {
     // ================= epilogue warps =================
     const int quarter = warp & 3;          // warps 2-5 own TMEM lanes 32*quarter .. +31
     const int r = 32 * quarter + lane;     // sub-block row of the tile
