@@ -295,7 +295,8 @@ LSA_API int lsa_layer_group(lsa_ctx* ctx, const lsa_params* p, const void* q_idx
  * q_idx_host, w_host, q_host[r], out_host[r] are host pointers; caches (k_idx, k_scale, kmean, k[r], v[r])
  * stay device-resident.  The queries are processed in passes of `stage_queries`; each pass copies its
  * slice of q_idx, w and q[r] to the device staging buffers, runs the group on it and copies out[r] back;
- * copies of the next pass overlap the kernels of the current one on two internal streams.
+ * copies in, kernels and copies out of consecutive passes overlap on two internal streams (the copy-in of pass i+2
+ * starts as soon as the kernels of pass i have read their inputs).
  * stage[2] are two caller-owned device staging areas of lsa_host_stage_bytes() bytes each. */
 LSA_API int lsa_layer_group_host(lsa_ctx* ctx, const lsa_params* p, const void* q_idx_host, const float* w_host,
                          const void* k_idx, const float* k_scale, const void* kmean, int64_t n_query,

@@ -639,14 +639,16 @@ int lsa_layer_group_host(lsa_ctx* c, const lsa_params* p, const void* q_idx_host
     for (int l = 0; l < R; ++l) { d_o[l] = base + off; off += align_up(static_cast<size_t>(sq) * b_o, 256); }
     int32_t* d_idx = reinterpret_cast<int32_t*>(base + off); off += align_up(static_cast<size_t>(sq) * p->k_sparse * 4, 256);
     int32_t* d_n = reinterpret_cast<int32_t*>(base + off);
-    // stage s is free once the copy-out of pass i-2 has drained it
-    if (i >= 2) e = cudaStreamWaitEvent(c->copy_in, c->ev_out[s], 0);
+    // The input half of stage s is free once the kernels of pass i-2 have read it; its output half only once the
+    // copy-out of pass i-2 has drained it, which the kernels of this pass (not its copy-in) have to wait for.
+    if (i >= 2) e = cudaStreamWaitEvent(c->copy_in, c->ev_done[s], 0);
     if (e == cudaSuccess) e = cudaMemcpyAsync(d_qi, static_cast<const uint8_t*>(q_idx_host) + q0 * b_qi, n * b_qi, cudaMemcpyHostToDevice, c->copy_in);
     if (e == cudaSuccess) e = cudaMemcpyAsync(d_w, reinterpret_cast<const uint8_t*>(w_host) + q0 * b_w, n * b_w, cudaMemcpyHostToDevice, c->copy_in);
     for (int l = 0; l < R && e == cudaSuccess; ++l)
       e = cudaMemcpyAsync(const_cast<void*>(d_q[l]), static_cast<const uint8_t*>(q_host[l]) + q0 * b_q, n * b_q, cudaMemcpyHostToDevice, c->copy_in);
     if (e == cudaSuccess) e = cudaEventRecord(c->ev_in[s], c->copy_in);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(c->stream, c->ev_in[s], 0);
+    if (e == cudaSuccess && i >= 2) e = cudaStreamWaitEvent(c->stream, c->ev_out[s], 0);
     if (e != cudaSuccess) break;
     r = lsa_layer_group(c, p, d_qi, reinterpret_cast<const float*>(d_w), k_idx, k_scale, kmean, q0, n, n_key, nullptr,
                         0, nullptr, 1, d_q, k, v, ld_k, ld_v, d_o, nullptr, d_idx, d_n);

@@ -242,6 +242,30 @@ def test_convert_lists_physical_rows(cuda_device):
         assert r[3] <= n_sp + cfg.W // cfg.kv_page + 3
 
 
+# ---------------------------------------------------------------- host-buffer entry point
+def test_layer_group_from_host_buffers_equals_device_run(cuda_device):
+    """lsa_layer_group_host (queries in pinned host memory, staged through the device in passes, copies overlapping
+    kernels) returns the bytes of the device-resident run, for a pass size that leaves a ragged last pass and needs
+    every staging buffer several times."""
+    cfg = SMALL_FP8.replace(name="host_small", L=5000, R=2, seed=23)
+    wl = PrefillWorkload(cfg, cuda_device, with_lse=False)
+    wl.prepare()
+    wl.step()
+    torch.cuda.synchronize()
+    sq = 768
+    stage = [torch.empty(binding.host_stage_bytes(wl.params, sq), dtype=torch.uint8, device=cuda_device) for _ in range(2)]
+    q_idx_h, w_h = wl.q_idx.cpu().pin_memory(), wl.w.cpu().pin_memory()
+    q_h = [q.cpu().pin_memory() for q in wl.q]
+    out_h = [torch.zeros(o.shape, dtype=o.dtype).pin_memory() for o in wl.out]
+    for _ in range(2):   # twice: the second call reuses events and staging areas left by the first
+        wl.ctx.layer_group_host(q_idx_h, w_h, wl.keys["k"], wl.keys.get("scale"), wl.kmean, wl.n_query, wl.n_key, q_h,
+                                wl.k, wl.v, out_h, sq, stage)
+        torch.cuda.synchronize()
+        assert wl.ctx.status() == 0
+        for oh, o in zip(out_h, wl.out):
+            assert torch.equal(oh, o.cpu())
+
+
 # ---------------------------------------------------------------- decode-step cache maintenance
 def test_append_tokens_then_decode(cuda_device):
     """37 decode steps of cache maintenance (crossing sub-block and page boundaries): the stored codes and scales are
