@@ -42,6 +42,8 @@ def parse_args():
     ap.add_argument("--attn-tc", type=int, default=-1, help="override LSA_TUNE_ATTN_TC (0 or 1)")
     ap.add_argument("--seq-len", type=int, default=0, help="override the prefill length L of the config (profiling sweeps)")
     ap.add_argument("--q-tail", type=int, default=0, help="score only the last N queries of the sequence")
+    ap.add_argument("--batch", type=int, default=0, help="override the decode batch of the config (small profiling captures)")
+    ap.add_argument("--layers", type=int, default=0, help="override R, the layers per group (small profiling captures)")
     ap.add_argument("--flat", action="store_true", help="hi_enable = 0: flat indexer (Eq. 7) instead of the hierarchy")
     ap.add_argument("--attn-split", type=int, default=0, help="override LSA_TUNE_ATTN_SPLIT (decode row splits)")
     ap.add_argument("--coarse-groups", type=int, default=0, help="override LSA_TUNE_COARSE_GROUPS (1 or 2)")
@@ -129,6 +131,9 @@ def attn_bytes_per_launch(cfg, positions):
 # (profiles/sparse_attn_tc_cfg3_16k.md: dram__bytes_read.sum 1.346437 GB + dram__bytes_write.sum 1.041851 GB).
 # Traffic there is q + out (the KV latent stays in L2), so it scales with the number of queries of a launch.
 NCU_ATTN_DRAM_BYTES_PER_QUERY = (1.346437e9 + 1.041851e9) / 16384
+# Decode: DRAM bytes of one attention launch per sequence, from the ncu capture at batch 16
+# (profiles/sparse_attn_tc_cfg4_decode_batch16.md: dram__bytes_read.sum 43.94 MB + dram__bytes_write.sum 0.45 MB).
+NCU_DECODE_ATTN_DRAM_BYTES_PER_SEQ = (43939584 + 450048) / 16
 
 
 def measured_peaks():
@@ -222,6 +227,10 @@ def main():
         kw = dict(q_pos0=cfg.L - cfg.q_chunk, n_query=cfg.q_chunk)
     if args.seq_len:
         cfg = cfg.replace(L=args.seq_len)
+    if args.batch:
+        cfg = cfg.replace(batch=args.batch)
+    if args.layers:
+        cfg = cfg.replace(R=args.layers)
     if args.flat:
         cfg = cfg.replace(hi_enable=False)
     if args.q_tail:
@@ -298,7 +307,10 @@ def main():
             attn_us = decode_attn_launch_us(wl)
             a = attn_bytes_per_launch(cfg, positions) / (attn_us * 1e-6) / 1e9
             roofline = {"kernel": "sparse_attn_tc_kernel", "bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"],
-                        "unit": "GB/s", "frac": a / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                        "unit": "GB/s", "frac": a / peaks["hbm_gbs"],
+                        "traffic": NCU_DECODE_ATTN_DRAM_BYTES_PER_SEQ * cfg.batch,
+                        "traffic_source": "ncu capture at batch 16, scaled by sequences per launch",
+                        "algorithmic_bytes": attn_bytes_per_launch(cfg, positions), "peak_source": peaks["source"],
                         "launch_ms": attn_us * 1e-3, "timing": "one event pair around 10 x R back-to-back launches"}
         else:
             a = attn_flops_per_launch(cfg, positions) / dur_s / 1e12
@@ -447,7 +459,10 @@ def measure_decode(cfg, dev, peaks, steps=50, warmup=10):
             "kernels_us_per_step": {k: v[0] / steps * 1e3 for k, v in prof.items() if v[1] > 0},
             "roofline": with_nominal({"kernel": "sparse_attn_tc_kernel", "bound": "hbm", "achieved": a,
                                       "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": a / peaks["hbm_gbs"],
-                                      "traffic": None, "peak_source": peaks["source"], "launch_us": attn_us,
+                                      "traffic": NCU_DECODE_ATTN_DRAM_BYTES_PER_SEQ * cfg.batch,
+                                      "traffic_source": "ncu capture at batch 16, scaled by sequences per launch",
+                                      "algorithmic_bytes": attn_bytes_per_launch(cfg, positions),
+                                      "peak_source": peaks["source"], "launch_us": attn_us,
                                       "timing": "one event pair around 10 x R back-to-back launches"}),
             "running_loop": running}
 
