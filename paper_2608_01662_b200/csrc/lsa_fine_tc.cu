@@ -75,6 +75,18 @@ __global__ void __launch_bounds__(kFineThreads, 2) fine_select_tc_kernel(const _
   }
   if (tc::status_raised(p.status)) return;   // an earlier block of this launch gave up on a wait
 
+  // query heads (K-major, 128B swizzle) and head weights: asynchronous copies that land during the page selection
+  {
+    const uint8_t* qg = reinterpret_cast<const uint8_t*>(p.q_idx) + static_cast<int64_t>(qi) * kHI * kDI * 2;
+#pragma unroll
+    for (int k = 0; k < kHI * 16 / kFineThreads; ++k) {
+      const int e = tid + k * kFineThreads, r = e >> 4, c = e & 15;
+      cp_async16(smem_u32(sm.q[c >> 3]) + r * 128 + (((c & 7) ^ (r & 7)) << 4), qg + e * 16, 16);
+    }
+    if (tid < kHI / 4) cp_async16(smem_u32(&sm.w[tid * 4]), p.w + static_cast<int64_t>(qi) * kHI + tid * 4, 16);
+    cp_async_commit();
+  }
+
   // ---- a2: pages that survive the coarse stage
   const int p0 = static_cast<int>(lo / p.P), p1 = static_cast<int>(hi / p.P);
   const int nE = p1 - p0 + 1;
@@ -108,16 +120,7 @@ __global__ void __launch_bounds__(kFineThreads, 2) fine_select_tc_kernel(const _
     tc::tmem_alloc(smem_u32(&sm.tmem_slot), kTmemColsFine);
     tc::tmem_relinquish();
   }
-  // query heads (K-major, 128B swizzle) and head weights
-  {
-    const uint8_t* qg = reinterpret_cast<const uint8_t*>(p.q_idx) + static_cast<int64_t>(qi) * kHI * kDI * 2;
-    for (int e = tid; e < kHI * 16; e += kFineThreads) {
-      const int r = e >> 4, c = e & 15;
-      *reinterpret_cast<uint4*>(sm.q[c >> 3] + r * 128 + (((c & 7) ^ (r & 7)) << 4)) =
-          *reinterpret_cast<const uint4*>(qg + e * 16);
-    }
-    if (tid < kHI) sm.w[tid] = p.w[static_cast<int64_t>(qi) * kHI + tid];
-  }
+  cp_async_wait<0>();   // query heads and weights, requested before the page selection
   tc::fence_proxy_async();
   tc::fence_before_sync();
   __syncthreads();   // pages, q, w, barriers and the TMEM base are visible
