@@ -3,7 +3,7 @@
 // Items i = 0..n-1 carry a 32-bit key (larger = better, 0 = absent) and appear in ascending id
 // order.  The k items that are largest under (key descending, i ascending) are written in
 // ascending i.  Four 8-bit histogram passes find the k-th largest key T; everything above T is
-// taken, and of the items equal to T the first (k - #above) in index order.
+// taken, and of the items equal to T the first (k - #above) in index order.  Three block barriers per pass.
 #pragma once
 
 #include "lsa_common.cuh"
@@ -29,78 +29,76 @@ template <class KeyF, class IdF>
 __device__ int block_select_topk(KeyF key, IdF id, int n, int k, int* out, SelectScratch& sc) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-  // ---- how many items are present
-  uint32_t cnt = 0;
-  for (int i = tid; i < n; i += kSelThreads) cnt += key(i) != 0u;
-  cnt = __reduce_add_sync(0xffffffffu, cnt);
-  if (lane == 0) sc.warp_gt[warp] = cnt;
-  __syncthreads();
-  if (tid == 0) {
-    uint32_t s = 0;
-    for (int w = 0; w < kSelWarps; ++w) s += sc.warp_gt[w];
-    sc.n_valid = s;
-  }
-  __syncthreads();
-  const int n_valid = static_cast<int>(sc.n_valid);
+  // ---- radix select: four 8-bit passes from the top byte down.  A pass counts the digits of the keys that still
+  // match the prefix into per-warp histograms (zero between passes: every thread clears the bins it has just summed);
+  // then thread t sums bin 255 - t over the warps, the block scans those sums from the top bin down (warp shuffles
+  // plus one exchange of warp totals), and the thread whose bin holds the k-th key publishes the new prefix.  The
+  // first pass also yields the number of keys present (its grand total): with k or fewer, everything is taken.
   uint32_t T = 0;      // take keys > T ...
   int need_eq = 0;     // ... and the first need_eq keys == T
-  if (k <= 0 || n_valid == 0) {
-    for (int i = tid; i < k; i += kSelThreads) out[i] = -1;
-    __syncthreads();
-    return 0;
-  }
-  if (n_valid > k) {
+  for (int i = tid; i < kSelWarps * 256; i += kSelThreads) (&sc.hist[0][0])[i] = 0;
+  if (tid == 0) sc.n_valid = 0;
+  __syncthreads();
+  int n_valid = 0;
+  {
     uint32_t prefix = 0, mask = 0;
-    uint32_t remaining = static_cast<uint32_t>(k);
+    uint32_t remaining = static_cast<uint32_t>(k > 0 ? k : 0);
+    bool take_all = false;
 #pragma unroll 1
     for (int shift = 24; shift >= 0; shift -= 8) {
-      for (int i = tid; i < kSelWarps * 256; i += kSelThreads) (&sc.hist[0][0])[i] = 0;
-      __syncthreads();
       for (int i = tid; i < n; i += kSelThreads) {
         const uint32_t kk = key(i);
         if (kk != 0u && (kk & mask) == prefix) atomicAdd(&sc.hist[warp][(kk >> shift) & 255u], 1u);
       }
       __syncthreads();
-      if (warp == 0) {
-        // lane l owns bins 255-8l .. 248-8l (descending); find the bin where the running count
-        // from the top reaches `remaining`
-        uint32_t mine[8], tot = 0;
+      // bin 255 - tid: its count over all warps, cleared for the next pass
+      const int bin = 255 - tid;
+      uint32_t cnt = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int b = 255 - 8 * lane - j;
-          uint32_t s = 0;
+      for (int w = 0; w < kSelWarps; ++w) {
+        cnt += sc.hist[w][bin];
+        sc.hist[w][bin] = 0;
+      }
+      uint32_t incl = cnt;
 #pragma unroll
-          for (int w = 0; w < kSelWarps; ++w) s += sc.hist[w][b];
-          mine[j] = s;
-          tot += s;
-        }
-        uint32_t incl = tot;
+      for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += v;
+      }
+      if (lane == 31) sc.warp_gt[warp] = incl;   // this warp's 32 bins
+      __syncthreads();
+      uint32_t before = 0, total = 0;
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-          const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
-          if (lane >= d) incl += v;
-        }
-        const uint32_t excl = incl - tot;
-        if (excl < remaining && remaining <= incl) {
-          uint32_t run = excl;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            if (run < remaining && remaining <= run + mine[j]) {
-              sc.prefix = prefix | (static_cast<uint32_t>(255 - 8 * lane - j) << shift);
-              sc.remaining = remaining - run;
-            }
-            run += mine[j];
-          }
-        }
+      for (int w = 0; w < kSelWarps; ++w) {
+        const uint32_t v = sc.warp_gt[w];
+        before += w < warp ? v : 0u;
+        total += v;
+      }
+      incl += before;
+      const uint32_t excl = incl - cnt;
+      if (shift == 24) {
+        n_valid = static_cast<int>(total);
+        take_all = n_valid <= k || k <= 0;
+      }
+      if (!take_all && excl < remaining && remaining <= incl) {   // exactly one thread
+        sc.prefix = prefix | (static_cast<uint32_t>(bin) << shift);
+        sc.remaining = remaining - excl;
       }
       __syncthreads();
+      if (take_all) break;   // uniform: every thread computed the same total
       prefix = sc.prefix;
       remaining = sc.remaining;
       mask |= 255u << shift;
-      __syncthreads();
     }
-    T = prefix;
-    need_eq = static_cast<int>(remaining);
+    if (!take_all) {
+      T = prefix;
+      need_eq = static_cast<int>(remaining);
+    }
+  }
+  if (k <= 0 || n_valid == 0) {
+    for (int i = tid; i < k; i += kSelThreads) out[i] = -1;
+    __syncthreads();
+    return 0;
   }
 
   // ---- ordered compaction: warp w owns the contiguous index range [w*per, (w+1)*per)
