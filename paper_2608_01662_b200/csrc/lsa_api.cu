@@ -33,6 +33,8 @@ namespace {
 constexpr size_t kStatusBytes = 256;
 constexpr int kMaxSplit = 16;
 constexpr int kProfPairs = 4096;
+constexpr int64_t kFusedBudget = 4096;        // candidate tokens per query the fused fine kernels keep in shared memory
+constexpr int64_t kMaxBudget = 262144;        // largest recall budget M * P of the large-budget path
 constexpr int64_t kFlatFusedMaxKeys = 4096;   // caches up to this length: the fused fine kernel scores every eligible page
 
 // Runs `launch` (a callable returning cudaError_t), bracketed by an event pair of class `cat` when
@@ -71,7 +73,11 @@ int check_params(const lsa_params* p, bool need_index, bool need_attn) {
     if (p->page % p->sub_block != 0) return LSA_ERR_SHAPE;
     const int spp = p->page / p->sub_block;
     if (spp != 8 && spp != 16 && spp != 32) return LSA_ERR_SHAPE;
-    if (static_cast<int64_t>(p->keep_pages) * p->page > 4096) return LSA_ERR_SHAPE;
+    const int64_t budget = static_cast<int64_t>(p->keep_pages) * p->page;
+    if (budget > kFusedBudget) {
+      // larger recall budgets: contiguous caches and the 64-head, 128-dim indexer only (scores go through the workspace)
+      if (p->paged || p->n_heads_idx != 64 || p->d_idx != 128 || budget > kMaxBudget || budget % 128 != 0) return LSA_ERR_SHAPE;
+    }
     if (p->k_sparse > 4096 || p->k_sparse % 4 != 0) return LSA_ERR_SHAPE;
     if (p->paged && p->kv_page != p->page) return LSA_ERR_SHAPE;
     if (p->pooling != LSA_POOL_MEAN && p->pooling != LSA_POOL_MINMAX) return LSA_ERR_ARG;
@@ -88,6 +94,7 @@ int check_params(const lsa_params* p, bool need_index, bool need_attn) {
 // Workspace map.  All offsets are multiples of 256 bytes.
 struct WsLayout {
   size_t page_scores, rows, n_rows, part_out, part_lse, fine_keys, fine_pages, wide_keys, total;
+  size_t big_pages, big_np, big_scores, big_pos;   // large recall budget (M * P > 4096): page lists, scores, positions
   int ps_ld, rows_ld;
 };
 
@@ -117,6 +124,17 @@ WsLayout ws_layout(const lsa_params* p, int64_t n_query, int64_t n_key_max, int 
     // e4m3 codes widened to bf16 once per call: dense scoring of the flat indexer, TMA source of the fine stage
     l.wide_keys = off;
     off += align_up(static_cast<size_t>(n_key_max) * p->d_idx * 2, 256);
+  }
+  const int64_t budget = static_cast<int64_t>(p->keep_pages) * p->page;
+  if (!flat && !p->paged && budget > kFusedBudget) {
+    l.big_pages = off;
+    off += align_up(static_cast<size_t>(nq) * p->keep_pages * sizeof(int32_t), 256);
+    l.big_np = off;
+    off += align_up(static_cast<size_t>(nq) * sizeof(int32_t), 256);
+    l.big_scores = off;
+    off += align_up(static_cast<size_t>(nq) * budget * sizeof(float), 256);
+    l.big_pos = off;
+    off += align_up(static_cast<size_t>(nq) * budget * sizeof(int32_t), 256);
   }
   const int P = p->page > 0 ? p->page : 64;
   // hierarchical: one score per page; flat: one score per token
@@ -232,6 +250,23 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
         return lsa::coarse_tc_supported(a) ? lsa::launch_coarse_tc(a, c->tune[LSA_TUNE_COARSE_GROUPS], c->stream, &c->launches)
                                            : lsa::launch_coarse(a, c->stream, &c->launches);
       });
+    if (e == cudaSuccess && l.big_scores != 0) {
+      // recall budget beyond one block's shared memory: page list, fine scores through the workspace, standalone top-K
+      if (!lsa::fine_big_supported(a)) return LSA_ERR_SHAPE;
+      int32_t* pages_ws = reinterpret_cast<int32_t*>(c->ws + l.big_pages);
+      int32_t* np_ws = reinterpret_cast<int32_t*>(c->ws + l.big_np);
+      float* sc_ws = reinterpret_cast<float*>(c->ws + l.big_scores);
+      int32_t* pos_ws = reinterpret_cast<int32_t*>(c->ws + l.big_pos);
+      const int64_t budget = static_cast<int64_t>(p->keep_pages) * p->page;
+      e = timed(c, LSA_K_FINE_SELECT, [&] { return lsa::launch_fine_big(a, pages_ws, np_ws, sc_ws, pos_ws, c->stream, &c->launches); });
+      if (e == cudaSuccess)
+        e = timed(c, LSA_K_SELECT, [&] {
+          return lsa::launch_select(sc_ws, budget, pos_ws, nullptr, a.q_pos0, a.n_query, budget, p->k_sparse, 1, p->k_sink,
+                                    p->k_swa, a.sparse_idx, a.n_sparse, c->stream, &c->launches);
+        });
+      if (e != cudaSuccess) return cuda_fail(c, e);
+      continue;
+    }
     if (e == cudaSuccess) e = timed(c, LSA_K_FINE_SELECT, [&] { return lsa::launch_fine_select(a, c->stream, &c->launches); });
     if (e == cudaSuccess && a.rows_out != nullptr && a.fine_parts <= 1)
       // only the split fine stage writes the cache rows itself (in its top-K kernel)

@@ -44,11 +44,13 @@ def test_host_only_entry_points():
 def test_bad_parameters_return_codes():
     import pytest
     cfg = CONFIGS["cfg2"]
-    for bad in (cfg.replace(P=96), cfg.replace(B=3), cfg.replace(M=128), cfg.replace(Ksp=2050), cfg.replace(H=32),
-                cfg.replace(d_I=96)):
+    # M * P: 8192 is served by the large-budget path; 2^19 tokens, an odd multiple of 64, or the 8-head indexer are not
+    for bad in (cfg.replace(P=96), cfg.replace(B=3), cfg.replace(M=8192), cfg.replace(M=129), cfg.replace(Ksp=2050),
+                cfg.replace(H=32), cfg.replace(d_I=96), CONFIGS["cfg1"].replace(M=128), CONFIGS["cfg4"].replace(M=128)):
         with pytest.raises(binding.LsaError) as e:
             binding.workspace_bytes(binding.make_params(bad), 16, 1024)
         assert e.value.code == -2
+    assert binding.workspace_bytes(binding.make_params(cfg.replace(M=128)), 16, 1024) > 16 * 128 * 64 * 8
     p = binding.make_params(cfg)
     p.struct_size = 12
     with pytest.raises(binding.LsaError) as e:

@@ -242,6 +242,32 @@ def test_convert_lists_physical_rows(cuda_device):
         assert r[3] <= n_sp + cfg.W // cfg.kv_page + 3
 
 
+# ---------------------------------------------------------------- recall budgets beyond 4096 tokens
+@pytest.mark.parametrize("base", ["fp8", "bf16"])
+def test_large_recall_budget(cuda_device, base):
+    """M * P = 8192 candidate tokens per query (twice what the fused fine kernel holds): page list, fine scores through
+    the workspace and the standalone top-K give the oracle's pages and tokens, in one pass and in query chunks."""
+    src = CONFIGS["cfg3"] if base == "fp8" else CONFIGS["cfg2"]
+    cfg = src.replace(name=f"big_{base}", L=20000, P=64, M=128, Ksp=1024, W=384, R=1, seed=27, q_chunk=0)
+    wl = PrefillWorkload(cfg, cuda_device)
+    wl.prepare()
+    pages = torch.full((wl.n_query, cfg.M), -7, dtype=torch.int32, device=cuda_device)
+    wl.index(pages)
+    assert wl.ctx.status() == 0
+    qs = pu.boundary_queries(cfg, 0, cfg.L, 40, seed=3)
+    m = pu.check_prefill(wl, qs, check_attention=False, pages=pages)
+    print(cfg.name, m.summary())
+    assert m.summary()["mean_overlap"] >= pu.MIN_OVERLAP and m.summary()["page_sets_differ"] == 0
+    whole = wl.sparse_idx.clone()
+    del wl
+    wl2 = PrefillWorkload(cfg.replace(q_chunk=3000), cuda_device)
+    wl2.prepare()
+    wl2.step()
+    assert torch.equal(wl2.sparse_idx, whole)
+    m2 = pu.check_prefill(wl2, qs[-6:], check_attention=True)
+    m2.assert_ok(pu.TOL_FP8 if base == "fp8" else pu.TOL_BF16)
+
+
 # ---------------------------------------------------------------- host-buffer entry point
 def test_layer_group_from_host_buffers_equals_device_run(cuda_device):
     """lsa_layer_group_host (queries in pinned host memory, staged through the device in passes, copies overlapping
