@@ -42,6 +42,7 @@ def parse_args():
     ap.add_argument("--attn-tc", type=int, default=-1, help="override LSA_TUNE_ATTN_TC (0 or 1)")
     ap.add_argument("--seq-len", type=int, default=0, help="override the prefill length L of the config (profiling sweeps)")
     ap.add_argument("--q-tail", type=int, default=0, help="score only the last N queries of the sequence")
+    ap.add_argument("--keep-pages", type=int, default=0, help="override M, the pages recalled by the coarse stage (recall-budget sweeps)")
     ap.add_argument("--batch", type=int, default=0, help="override the decode batch of the config (small profiling captures)")
     ap.add_argument("--layers", type=int, default=0, help="override R, the layers per group (small profiling captures)")
     ap.add_argument("--flat", action="store_true", help="hi_enable = 0: flat indexer (Eq. 7) instead of the hierarchy")
@@ -227,6 +228,8 @@ def main():
         kw = dict(q_pos0=cfg.L - cfg.q_chunk, n_query=cfg.q_chunk)
     if args.seq_len:
         cfg = cfg.replace(L=args.seq_len)
+    if args.keep_pages:
+        cfg = cfg.replace(M=args.keep_pages)
     if args.batch:
         cfg = cfg.replace(batch=args.batch)
     if args.layers:
