@@ -46,9 +46,17 @@ __device__ int block_select_topk(KeyF key, IdF id, int n, int k, int* out, Selec
     bool take_all = false;
 #pragma unroll 1
     for (int shift = 24; shift >= 0; shift -= 8) {
-      for (int i = tid; i < n; i += kSelThreads) {
-        const uint32_t kk = key(i);
-        if (kk != 0u && (kk & mask) == prefix) atomicAdd(&sc.hist[warp][(kk >> shift) & 255u], 1u);
+      // four keys per thread and step: when the keys come from global memory the loads are in flight together
+      for (int i0 = tid; i0 < n; i0 += 4 * kSelThreads) {
+        uint32_t kk[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = i0 + u * kSelThreads;
+          kk[u] = i < n ? key(i) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (kk[u] != 0u && (kk[u] & mask) == prefix) atomicAdd(&sc.hist[warp][(kk[u] >> shift) & 255u], 1u);
       }
       __syncthreads();
       // bin 255 - tid: its count over all warps, cleared for the next pass
@@ -105,10 +113,18 @@ __device__ int block_select_topk(KeyF key, IdF id, int n, int k, int* out, Selec
   const int per = ((n + kSelWarps - 1) / kSelWarps + 31) & ~31;
   const int begin = warp * per, end = min(n, begin + per);
   uint32_t gt = 0, eq = 0;
-  for (int i = begin + lane; i < end; i += 32) {
-    const uint32_t kk = key(i);
-    gt += kk > T;
-    eq += (kk == T) & (kk != 0u);
+  for (int i0 = begin + lane; i0 < end; i0 += 4 * 32) {
+    uint32_t kk[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + 32 * u;
+      kk[u] = i < end ? key(i) : 0u;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      gt += kk[u] > T;
+      eq += (kk[u] == T) & (kk[u] != 0u);
+    }
   }
   gt = __reduce_add_sync(0xffffffffu, gt);
   eq = __reduce_add_sync(0xffffffffu, eq);
