@@ -1,28 +1,34 @@
 // a6 on the 5th-generation tensor cores: sparse attention (Eq. 3) for the MLA latent shape
 // (H = 64 heads, d_qk = 576, d_v = 512, the value is the first 512 dims of the key row).
 //
-// One thread block = one query (or one split of one sequence's rows in decode).  Its 64 heads are the M = 64
-// rows of every MMA; the attended cache rows stream through two 64-key shared tiles:
+// One thread block = one query (or one row split of one sequence in decode).  Its 64 heads are the M = 64
+// rows of every MMA; the attended cache rows stream through a ring of three 64-key shared tiles:
 //
-//   warps 5-8   gather: rows [sink | sparse | window] -> 128B-swizzled K-major tiles with coalesced 16-byte
-//               cp.async (all four warps on each tile), completion through an mbarrier
-//   warp 4      one thread issues every tcgen05.mma.  Back-to-back MMAs into one accumulator run far below
-//               the pipe's rate at these small shapes, so each product is cut into two independent
-//               accumulation chains that alternate instruction by instruction:
-//                 S = Q K^T   two partial sums of 18 K-steps each (M64 N64 K16)
-//                 O += P V    value dims 0-255 and 256-511 (M64 N256 K16 x 4 each); V is the key tile read
-//                             MN-major, so each cache row is fetched once
-//               The thread takes whichever of "next Q K^T" / "next P V" is ready.
-//   warps 0-3   softmax: tcgen05.ld of both partial sums, add, running max with lazy rescaling of O, exp2,
-//               fp32 row sums, P as bf16 -> tensor memory (A operand of P V); at the end O / l -> bf16
+//   warps 8-11  gather: rows [sink | sparse | window] -> 128B-swizzled K-major tiles with coalesced 16-byte
+//               cp.async, up to three tiles in flight, each handed over through an mbarrier when it has landed.
+//               Q arrives the same way: its rope dims (512-575) stay in shared memory as an MMA operand, dims 0-511
+//               are staged in the last tile buffer for the softmax warps
+//   warps 4-7   one thread each issues tcgen05.mma.  Back-to-back MMAs into one accumulator run far below the
+//               pipe's rate at these small shapes, so each product is cut into independent accumulation chains:
+//                 S = Q K^T   issuers 0 and 1: dims 0-255 / 256-511 with Q from tensor memory (16 steps of M64 N64
+//                             K16 each) plus two rope steps with Q from shared memory; the two partial sums land in
+//                             the two lane halves of the S buffer
+//                 O += P V    all four issuers: value dims 128x .. 128x+127 (M64 N128 K16 x 4 per tile) with P from
+//                             tensor memory; V is the key tile read MN-major, so each cache row is fetched once
+//               A thread takes whichever of "next Q K^T" / "next P V" is ready.
+//   warps 0-3   softmax: move Q to tensor memory once; per tile tcgen05.ld of both partial sums, add, running max
+//               with lazy rescaling of O, exp2, fp32 row sums, P as bf16 -> tensor memory (A operand of P V); at the
+//               end O / l through shared memory to global in whole rows
 //
-// An M = 64 accumulator occupies 16 of the 32 lanes of each TMEM quarter, so two of them share a column range:
+// An M = 64 accumulator occupies 16 of the 32 lanes of each TMEM quarter, so two of them share a column range.  All
+// 512 columns are in use:
 //   columns   0-255   O[:, 0:256] in lanes 0-15, O[:, 256:512] in lanes 16-31
-//   columns 256-383   S buffers 0 and 1 (64 columns each): the first chain's partial sum in lanes 0-15, the second's in
-//                     lanes 16-31.  Lanes l and l+16 of a softmax warp share head row l: they swap halves, so
-//                     lane l finishes keys 0-31 and lane l+16 keys 32-63 of the tile.
-//   columns 384-447   P buffers 0 and 1 (32 columns = 64 bf16 each), one copy per lane half, because an MMA reads
-//                     its TMEM operand from the lanes its accumulator lives in
+//   columns 256-383   Q[:, 0:512] as packed bf16: dims 0-255 in lanes 0-15, dims 256-511 in lanes 16-31 (an MMA reads
+//                     its TMEM operand from the lanes its accumulator lives in)
+//   columns 384-511   S buffers 0 and 1 (64 columns each): the first chain's partial sum in lanes 0-15, the second's in
+//                     lanes 16-31.  Lanes l and l+16 of a softmax warp share head row l: they swap halves, so lane l
+//                     finishes keys 0-31 and lane l+16 keys 32-63 of the tile.  P (32 columns = 64 bf16, one copy
+//                     per lane half) overwrites the first half of the S buffer it came from.
 #include <cstdio>
 #include <cstdlib>
 

@@ -2,6 +2,10 @@
 // fine token scores on the recalled pages (a3, Eq. 11) and top-K_sparse (a4, Eq. 12), the standalone
 // selection (Eq. 2/7) and the streaming-aware conversion of an index set to cache rows (a5, Sec. 3.1).
 //
+// The scoring kernels of this file are the `mma.sync` forms: they serve the 8-head indexer, paged fine scoring and
+// the MinMax variant; the 64-head indexer's coarse and contiguous fine stages run on tcgen05 (lsa_coarse_tc.cu,
+// lsa_coarse_paged_tc.cu, lsa_fine_tc.cu, lsa_fine_big_tc.cu).  Also here: the append-token cache maintenance.
+//
 // Scoring tiles put 128 keys (or mean keys) on the M axis of the tensor-core tile and the H_I heads of
 // one query on the N axis, so that the ReLU / head-weight / head-sum epilogue of Eq. 1 runs inside one
 // thread quad and one number per key leaves the tile.
