@@ -26,8 +26,8 @@ Pins (tests/test_oracle_*.py) check every function against something outside
 this file: brute-force loops, full sorts, torch/scipy library routines, closed
 forms and the equivalences the paper states.  No function here is unpinned.
 
-Readings taken where the paper is silent are listed in the design doc; the ones that
-matter for the arithmetic are repeated in the docstrings below.
+Readings taken where the paper is silent, and that matter for the arithmetic, are
+stated in the docstrings below.
 """
 from __future__ import annotations
 
