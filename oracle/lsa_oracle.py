@@ -10,7 +10,10 @@ first widened exactly to float64).  Positions are 0-indexed; the paper writes
 them 1-indexed.  One function per step, in the paper's order:
 
   e4m3_decode, dequant_keys      stored fp8 keys -> real values (FP8 indexer, Sec. 2.2)
+  e4m3_encode, quantize_token    real key -> stored fp8 code and per-token scale (fp32 decision)
   block_means                    per-dimension sub-block mean keys (Sec. 3.3, stage 1)
+  block_minmax, page_scores_minmax   the MinMax pooling variant (Eq. 13)
+  append_token                   cache maintenance of one decode step (new key, its sub-block mean)
   indexer_scores                 Eq. 1 / Eq. 11
   page_scores                    Eq. 9
   top_k                          arg-topK with the total order (score desc, id asc)
