@@ -206,6 +206,30 @@ def test_paged_decode_large_batch(cuda_device):
     m.assert_ok(pu.TOL_FP8)
 
 
+def test_decode_step_replays_from_a_cuda_graph(cuda_device):
+    """lsa_layer_group on a side stream makes no synchronising call: a decode step captures into a CUDA graph, and
+    the replay writes the bytes of the eager step."""
+    side = torch.cuda.Stream(device=cuda_device)
+    with torch.cuda.stream(side):
+        wl = DecodeWorkload(SMALL_DEC, cuda_device)
+        wl.prepare()
+        wl.step()
+        wl.step()
+        side.synchronize()
+        want = [o.clone() for o in wl.out] + [wl.sparse_idx.clone()]
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            wl.step()
+        for o in wl.out:
+            o.zero_()
+        wl.sparse_idx.zero_()
+        graph.replay()
+        side.synchronize()
+        assert wl.ctx.status() == 0
+        for a, b in zip(want, wl.out + [wl.sparse_idx]):
+            assert torch.equal(a, b)
+
+
 def test_decode_split_count_is_checked(cuda_device):
     cfg = SMALL_DEC
     if cfg.H != 64:
