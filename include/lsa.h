@@ -33,7 +33,7 @@
  *   indexer  (H_I, d_I) in {(8,64), (64,128)};  page P in {64,128,256}, sub_block B with P/B in
  *            {8,16,32};  k_sparse <= 4096, multiple of 4;  recall budget keep_pages*P <= 4096, or, for the
  *            (64,128) indexer on contiguous caches, any multiple of 128 up to 262144 (the candidates' scores
- *            then pass through the workspace: 8 bytes per candidate and query of a pass, see q_chunk)
+ *            then pass through the workspace: 4 bytes per candidate and query of a pass, see q_chunk)
  *   attention (H, d_qk, d_v) in {(16,128,128), (64,576,512)}
  *   paged mode needs kv_page == page.
  */

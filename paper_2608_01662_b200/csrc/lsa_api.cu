@@ -94,7 +94,7 @@ int check_params(const lsa_params* p, bool need_index, bool need_attn) {
 // Workspace map.  All offsets are multiples of 256 bytes.
 struct WsLayout {
   size_t page_scores, rows, n_rows, part_out, part_lse, fine_keys, fine_pages, wide_keys, total;
-  size_t big_pages, big_np, big_scores, big_pos;   // large recall budget (M * P > 4096): page lists, scores, positions
+  size_t big_pages, big_np, big_keys;   // large recall budget (M * P > 4096): page lists and the candidates' keys
   int ps_ld, rows_ld;
 };
 
@@ -131,10 +131,8 @@ WsLayout ws_layout(const lsa_params* p, int64_t n_query, int64_t n_key_max, int 
     off += align_up(static_cast<size_t>(nq) * p->keep_pages * sizeof(int32_t), 256);
     l.big_np = off;
     off += align_up(static_cast<size_t>(nq) * sizeof(int32_t), 256);
-    l.big_scores = off;
-    off += align_up(static_cast<size_t>(nq) * budget * sizeof(float), 256);
-    l.big_pos = off;
-    off += align_up(static_cast<size_t>(nq) * budget * sizeof(int32_t), 256);
+    l.big_keys = off;
+    off += align_up(static_cast<size_t>(nq) * budget * sizeof(uint32_t), 256);
   }
   const int P = p->page > 0 ? p->page : 64;
   // hierarchical: one score per page; flat: one score per token
@@ -250,20 +248,13 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
         return lsa::coarse_tc_supported(a) ? lsa::launch_coarse_tc(a, c->tune[LSA_TUNE_COARSE_GROUPS], c->stream, &c->launches)
                                            : lsa::launch_coarse(a, c->stream, &c->launches);
       });
-    if (e == cudaSuccess && l.big_scores != 0) {
-      // recall budget beyond one block's shared memory: page list, fine scores through the workspace, standalone top-K
+    if (e == cudaSuccess && l.big_keys != 0) {
+      // recall budget beyond one block's shared memory: page lists, fine scores through the workspace, top-K over them
       if (!lsa::fine_big_supported(a)) return LSA_ERR_SHAPE;
-      int32_t* pages_ws = reinterpret_cast<int32_t*>(c->ws + l.big_pages);
-      int32_t* np_ws = reinterpret_cast<int32_t*>(c->ws + l.big_np);
-      float* sc_ws = reinterpret_cast<float*>(c->ws + l.big_scores);
-      int32_t* pos_ws = reinterpret_cast<int32_t*>(c->ws + l.big_pos);
-      const int64_t budget = static_cast<int64_t>(p->keep_pages) * p->page;
-      e = timed(c, LSA_K_FINE_SELECT, [&] { return lsa::launch_fine_big(a, pages_ws, np_ws, sc_ws, pos_ws, c->stream, &c->launches); });
-      if (e == cudaSuccess)
-        e = timed(c, LSA_K_SELECT, [&] {
-          return lsa::launch_select(sc_ws, budget, pos_ws, nullptr, a.q_pos0, a.n_query, budget, p->k_sparse, 1, p->k_sink,
-                                    p->k_swa, a.sparse_idx, a.n_sparse, c->stream, &c->launches);
-        });
+      e = timed(c, LSA_K_FINE_SELECT, [&] {
+        return lsa::launch_fine_big(a, reinterpret_cast<int32_t*>(c->ws + l.big_pages), reinterpret_cast<int32_t*>(c->ws + l.big_np),
+                                    reinterpret_cast<uint32_t*>(c->ws + l.big_keys), c->stream, &c->launches);
+      });
       if (e != cudaSuccess) return cuda_fail(c, e);
       continue;
     }

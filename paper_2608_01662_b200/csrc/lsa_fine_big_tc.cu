@@ -6,10 +6,11 @@
 //                           (Eq. 10; the exact radix select, reading the scores from global memory) into a page list
 //   fine_scores_tc_kernel   a3: the fine scores (Eq. 11) of the listed pages on tcgen05 as in lsa_fine_tc.cu (TMA key
 //                           tiles of 128 tokens from the bf16 rows, M128 N64 K16, epilogue sum_j w_j relu(.) x scale),
-//                           but the scores and the positions they belong to go to global memory: a block covers a run
-//                           of a query's tiles, several blocks share a query
+//                           but the scores go to global memory as order-preserving keys (0 = not a candidate): a block
+//                           covers a run of a query's tiles, several blocks share a query
 //
-// a4 then runs as the standalone top-K (select_kernel) over the M * P scores of each query with their positions.
+//   select_keys_kernel      a4: the exact radix top-K_sparse over each query's keys; a slot's position comes from the page
+//                           list, so only the keys (4 bytes per candidate) travel through memory
 #include "lsa_internal.h"
 #include "lsa_select.cuh"
 #include "lsa_tc.cuh"
@@ -66,8 +67,7 @@ struct FineBigSmem {
 
 __global__ void __launch_bounds__(kThreadsBig, 2)
 fine_scores_tc_kernel(const __grid_constant__ CUtensorMap map, IndexArgs p, const int32_t* __restrict__ pages_ws,
-                      const int32_t* __restrict__ n_pages_ws, float* __restrict__ scores, int32_t* __restrict__ cand_pos,
-                      int64_t ld) {
+                      const int32_t* __restrict__ n_pages_ws, uint32_t* __restrict__ keys, int64_t ld) {
   extern __shared__ uint8_t smem_raw[];
   FineBigSmem& sm = *reinterpret_cast<FineBigSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -82,10 +82,9 @@ fine_scores_tc_kernel(const __grid_constant__ CUtensorMap map, IndexArgs p, cons
   const int tile_end = min(tiles_all, tile_begin + kTilesPerBlockBig);
   const int tiles_live = min(tile_end, (n_slots + kTile - 1) / kTile);  // tiles that hold listed pages
   const int32_t* pages = pages_ws + static_cast<int64_t>(qi) * p.M;
-  float* srow = scores + static_cast<int64_t>(qi) * ld;
-  int32_t* prow = cand_pos + static_cast<int64_t>(qi) * ld;
+  uint32_t* krow = keys + static_cast<int64_t>(qi) * ld;
   // slots past the listed pages: marked absent for the top-K
-  for (int c = max(tile_begin, tiles_live) * kTile + tid; c < tile_end * kTile; c += kThreadsBig) prow[c] = -1;
+  for (int c = max(tile_begin, tiles_live) * kTile + tid; c < tile_end * kTile; c += kThreadsBig) krow[c] = 0u;
   const int n_tiles = tiles_live - tile_begin;
   if (n_tiles <= 0) return;
   if (tc::status_raised(p.status)) return;
@@ -189,13 +188,35 @@ fine_scores_tc_kernel(const __grid_constant__ CUtensorMap map, IndexArgs p, cons
         a0 = fmaf(ww.z, fmaxf(__uint_as_float(v[4 * j + 2]), 0.f), a0);
         a1 = fmaf(ww.w, fmaxf(__uint_as_float(v[4 * j + 3]), 0.f), a1);
       }
-      srow[c] = (a0 + a1) * sc;
-      prow[c] = cand ? static_cast<int32_t>(pos) : -1;   // outside the scoring range: absent
+      krow[c] = cand ? score_key((a0 + a1) * sc) : 0u;   // order-preserving key; outside the scoring range: absent
     }
   }
   tc::fence_before_sync();
   __syncthreads();
   if (warp == 1) tc::tmem_dealloc(tmem_base, kTmemColsBig);
+}
+
+// ---- a4 over the keys of a query's listed pages: slot c of the row is token pages[c / P] * P + c % P
+__global__ void __launch_bounds__(kSelThreads) select_keys_kernel(IndexArgs p, const int32_t* __restrict__ pages_ws,
+                                                                  const int32_t* __restrict__ n_pages_ws,
+                                                                  const uint32_t* __restrict__ keys, int64_t ld) {
+  __shared__ SelectScratch sc;
+  __shared__ int32_t pages[1024];
+  const int qi = blockIdx.x, tid = threadIdx.x;
+  const int pshift = 31 - __clz(p.P);
+  const int nP = n_pages_ws[qi];
+  const bool cached = p.M <= 1024;
+  const int32_t* pg = pages_ws + static_cast<int64_t>(qi) * p.M;
+  if (cached) {
+    for (int i = tid; i < nP; i += kSelThreads) pages[i] = pg[i];
+    __syncthreads();
+    pg = pages;
+  }
+  const uint32_t* krow = keys + static_cast<int64_t>(qi) * ld;
+  const int n_sel = block_select_topk([&](int i) { return krow[i]; },
+                                      [&](int i) { return (pg[i >> pshift] << pshift) + (i & (p.P - 1)); }, nP << pshift, p.Ksp,
+                                      p.sparse_idx + static_cast<int64_t>(qi) * p.Ksp, sc);
+  if (tid == 0) p.n_sparse[qi] = n_sel;
 }
 
 }  // namespace
@@ -207,9 +228,10 @@ bool fine_big_supported(const IndexArgs& a) {
          tma_available();
 }
 
-// pages_ws int32 [n_query, M], n_pages_ws int32 [n_query], scores fp32 and cand_pos int32 [n_query, M * P]
-cudaError_t launch_fine_big(const IndexArgs& a, int32_t* pages_ws, int32_t* n_pages_ws, float* scores, int32_t* cand_pos,
-                            cudaStream_t st, int64_t* n_launch) {
+// pages_ws int32 [n_query, M], n_pages_ws int32 [n_query], keys uint32 [n_query, M * P]; three launches: page lists,
+// fine scores as order-preserving keys, top-K_sparse
+cudaError_t launch_fine_big(const IndexArgs& a, int32_t* pages_ws, int32_t* n_pages_ws, uint32_t* keys, cudaStream_t st,
+                            int64_t* n_launch) {
   if (a.n_query == 0) return cudaSuccess;
   page_topm_kernel<<<a.n_query, kSelThreads, 0, st>>>(a, pages_ws, n_pages_ws);
   ++*n_launch;
@@ -223,7 +245,11 @@ cudaError_t launch_fine_big(const IndexArgs& a, int32_t* pages_ws, int32_t* n_pa
   if (e != cudaSuccess) return e;
   const int64_t ld = static_cast<int64_t>(a.M) * a.P;
   const unsigned parts = static_cast<unsigned>((ld / kTile + kTilesPerBlockBig - 1) / kTilesPerBlockBig);
-  fine_scores_tc_kernel<<<dim3(a.n_query, parts), kThreadsBig, smem, st>>>(map, a, pages_ws, n_pages_ws, scores, cand_pos, ld);
+  fine_scores_tc_kernel<<<dim3(a.n_query, parts), kThreadsBig, smem, st>>>(map, a, pages_ws, n_pages_ws, keys, ld);
+  ++*n_launch;
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  select_keys_kernel<<<a.n_query, kSelThreads, 0, st>>>(a, pages_ws, n_pages_ws, keys, ld);
   ++*n_launch;
   return cudaGetLastError();
 }

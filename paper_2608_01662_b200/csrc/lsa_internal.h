@@ -94,10 +94,10 @@ cudaError_t launch_fine_select(const IndexArgs& a, cudaStream_t st, int64_t* n_l
 bool fine_tc_supported(const IndexArgs& a);
 cudaError_t launch_fine_select_tc(const IndexArgs& a, cudaStream_t st, int64_t* n_launch);
 // Recall budgets M * P > 4096 (contiguous caches, H_I = 64, d_I = 128): page top-M into pages_ws [n_query, M] /
-// n_pages_ws [n_query], then fine scores and their positions into scores / cand_pos [n_query, M * P] for launch_select
+// n_pages_ws [n_query], fine scores as keys [n_query, M * P], top-K_sparse into a.sparse_idx / a.n_sparse
 bool fine_big_supported(const IndexArgs& a);
-cudaError_t launch_fine_big(const IndexArgs& a, int32_t* pages_ws, int32_t* n_pages_ws, float* scores, int32_t* cand_pos,
-                            cudaStream_t st, int64_t* n_launch);
+cudaError_t launch_fine_big(const IndexArgs& a, int32_t* pages_ws, int32_t* n_pages_ws, uint32_t* keys, cudaStream_t st,
+                            int64_t* n_launch);
 cudaError_t launch_select(const float* scores, int64_t ld, const int32_t* cand_pos, const float* pos_scale,
                           int64_t q_pos0, int n_query, int64_t n_cand, int k, int apply_range, int S, int W,
                           int32_t* idx_out, int32_t* n_out, cudaStream_t st, int64_t* n_launch);

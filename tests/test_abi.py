@@ -50,7 +50,7 @@ def test_bad_parameters_return_codes():
         with pytest.raises(binding.LsaError) as e:
             binding.workspace_bytes(binding.make_params(bad), 16, 1024)
         assert e.value.code == -2
-    assert binding.workspace_bytes(binding.make_params(cfg.replace(M=128)), 16, 1024) > 16 * 128 * 64 * 8
+    assert binding.workspace_bytes(binding.make_params(cfg.replace(M=128)), 16, 1024) > 16 * 128 * 64 * 4
     p = binding.make_params(cfg)
     p.struct_size = 12
     with pytest.raises(binding.LsaError) as e:
