@@ -307,14 +307,8 @@ def main():
     if attn_n > 0:
         dur_s = attn_ms / attn_n * 1e-3
         if decode:
-            attn_us = decode_attn_launch_us(wl)
-            a = attn_bytes_per_launch(cfg, positions) / (attn_us * 1e-6) / 1e9
-            roofline = {"kernel": "sparse_attn_tc_kernel", "bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"],
-                        "unit": "GB/s", "frac": a / peaks["hbm_gbs"],
-                        "traffic": NCU_DECODE_ATTN_DRAM_BYTES_PER_SEQ * cfg.batch,
-                        "traffic_source": "ncu capture at batch 16, scaled by sequences per launch",
-                        "algorithmic_bytes": attn_bytes_per_launch(cfg, positions), "peak_source": peaks["source"],
-                        "launch_ms": attn_us * 1e-3, "timing": "one event pair around 10 x R back-to-back launches"}
+            roofline = decode_attn_roofline(cfg, prof, args.steps, positions, peaks)
+            roofline["single_layer_launch_us"] = decode_attn_launch_us(wl)
         else:
             a = attn_flops_per_launch(cfg, positions) / dur_s / 1e12
             roofline = {"kernel": "sparse_attn_tc_kernel" if cfg.H == 64 else "sparse_attn_kernel", "bound": "tensor", "achieved": a,
@@ -380,6 +374,26 @@ def with_nominal(roofline):
     return roofline
 
 
+def decode_attn_roofline(cfg, prof, steps, positions, peaks):
+    """Decode roofline of the attention launch as lsa_layer_group issues it: on the MLA shape one launch covers the R
+    layers of the group (each with its own multi-GB cache, so nothing is found in L2), timed by the library's event
+    pair around it inside the timed steps.  `single_layer_launch_us` is the same kernel launched per layer
+    (lsa_sparse_attn back to back), for comparison."""
+    attn_ms, attn_n = prof["sparse_attn"]
+    launches_per_step = attn_n / steps
+    layers_per_launch = cfg.R / launches_per_step
+    launch_us = attn_ms / attn_n * 1e3
+    bytes_per_launch = attn_bytes_per_launch(cfg, positions) * layers_per_launch
+    a = bytes_per_launch / (launch_us * 1e-6) / 1e9
+    return with_nominal({"kernel": "sparse_attn_tc_kernel", "bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": a / peaks["hbm_gbs"],
+                         "traffic": NCU_DECODE_ATTN_DRAM_BYTES_PER_SEQ * cfg.batch * layers_per_launch,
+                         "traffic_source": "ncu capture at batch 16, one layer, scaled by sequences and layers per launch",
+                         "algorithmic_bytes": bytes_per_launch, "peak_source": peaks["source"], "launch_us": launch_us,
+                         "layers_per_launch": layers_per_launch,
+                         "timing": "library event pair around the launch inside the timed steps"})
+
+
 def decode_attn_launch_us(wl, rounds=10):
     """Average device time of one decode attention launch (a6 with its split merge), timed with one CUDA event pair
     around rounds x R back-to-back lsa_sparse_attn calls on the physical row lists lsa_convert wrote.  Each layer
@@ -435,8 +449,8 @@ def measure_decode(cfg, dev, peaks, steps=50, warmup=10):
     prof = wl.ctx.profile_read()
     wl.ctx.profile_enable(False)
     positions = wl.ctx_len.cpu().numpy().astype(np.int64) - 1
-    attn_us = decode_attn_launch_us(wl)
-    a = attn_bytes_per_launch(cfg, positions) / (attn_us * 1e-6) / 1e9
+    roofline = decode_attn_roofline(cfg, prof, steps, positions, peaks)
+    roofline["single_layer_launch_us"] = decode_attn_launch_us(wl)
     # running loop: every step first appends one token per sequence (indexer key quantised, sub-block mean updated,
     # one latent row per layer), then runs the group on the grown caches
     k_new = (torch.randn((cfg.batch, cfg.d_I), device=dev) / cfg.d_I ** 0.5).to(torch.bfloat16)
@@ -460,13 +474,7 @@ def measure_decode(cfg, dev, peaks, steps=50, warmup=10):
             "config": {"workload": cfg.name, "batch": cfg.batch, "R": cfg.R, "ctx": [cfg.ctx_lo, cfg.ctx_hi],
                        "l2": "KV pools are GBs per layer, far larger than L2; no flush"},
             "kernels_us_per_step": {k: v[0] / steps * 1e3 for k, v in prof.items() if v[1] > 0},
-            "roofline": with_nominal({"kernel": "sparse_attn_tc_kernel", "bound": "hbm", "achieved": a,
-                                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": a / peaks["hbm_gbs"],
-                                      "traffic": NCU_DECODE_ATTN_DRAM_BYTES_PER_SEQ * cfg.batch,
-                                      "traffic_source": "ncu capture at batch 16, scaled by sequences per launch",
-                                      "algorithmic_bytes": attn_bytes_per_launch(cfg, positions),
-                                      "peak_source": peaks["source"], "launch_us": attn_us,
-                                      "timing": "one event pair around 10 x R back-to-back launches"}),
+            "roofline": roofline,
             "running_loop": running}
 
 

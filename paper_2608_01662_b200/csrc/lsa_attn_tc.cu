@@ -113,7 +113,14 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
   extern __shared__ uint8_t smem_raw[];
   AttnTcSmem& sm = *reinterpret_cast<AttnTcSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int qi = blockIdx.x, split = blockIdx.y;
+  const int qi = blockIdx.x, split = blockIdx.y, layer = blockIdx.z;
+  // this layer's tensors (a launch may cover several layers of a group: same rows, different caches)
+  const void* const q_ptr = p.q_l[layer];
+  const void* const k_ptr = p.k_l[layer];
+  void* const out_ptr = p.out_l[layer];
+  float* const lse_ptr = p.lse_l[layer];
+  float* const part_out = p.part_out + static_cast<int64_t>(layer) * p.n_query * p.n_split * kH * kDV;
+  float* const part_lse = p.part_lse + static_cast<int64_t>(layer) * p.n_query * p.n_split * kH;
 
   const bool clustered = p.n_split > 1;
   const bool dead = tc::status_raised(p.status);   // an earlier block of this launch (or an earlier launch) gave up on a wait
@@ -185,7 +192,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       // Q of this query: the rope part (dims 512-575) stays in shared memory as an MMA operand; dims 0-511 are staged
       // in the last key buffer (64 rows x 1024 B, 16-byte chunks swizzled by row) for the softmax warps, which move
       // them to tensor memory.  The copies share the first cp.async group, handed over with the first key tile.
-      const uint8_t* qg = reinterpret_cast<const uint8_t*>(p.q) + static_cast<int64_t>(qi) * kH * kDQK * 2;
+      const uint8_t* qg = reinterpret_cast<const uint8_t*>(q_ptr) + static_cast<int64_t>(qi) * kH * kDQK * 2;
       for (int e = lt; e < kH * 8; e += 32 * kLoadWarps) {
         const int r = e >> 3, c = e & 7;
         cp_async16(smem_u32(sm.q_rope) + r * 128 + ((c ^ (r & 7)) << 4), qg + r * kDQK * 2 + 512 * 2 + c * 16, 16);
@@ -202,7 +209,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     // and the 72 16-byte chunks of that row are copied by consecutive lanes (coalesced 512-byte requests).
     const int lw = lt >> 5;
     constexpr int kRowsPerWarp = kTileKeys / kLoadWarps;
-    const uint8_t* kg = reinterpret_cast<const uint8_t*>(p.k);
+    const uint8_t* kg = reinterpret_cast<const uint8_t*>(k_ptr);
     auto my_key_row = [&](int i) -> int32_t {
       return (i < n_tiles && lane < kRowsPerWarp) ? row_of((tile_begin + i) * kTileKeys + kRowsPerWarp * lw + lane) : -1;
     };
@@ -500,7 +507,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
         }
       }
       __syncwarp();
-      uint8_t* dst = reinterpret_cast<uint8_t*>(reinterpret_cast<__nv_bfloat16*>(p.out) + static_cast<int64_t>(qi) * kH * kDV);
+      uint8_t* dst = reinterpret_cast<uint8_t*>(reinterpret_cast<__nv_bfloat16*>(out_ptr) + static_cast<int64_t>(qi) * kH * kDV);
       constexpr int kChunksPerRow = kRowBytes / 16;
 #pragma unroll 4
       for (int e = lane; e < 16 * kChunksPerRow; e += 32) {   // this warp's 16 rows
@@ -508,7 +515,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
         *reinterpret_cast<uint4*>(dst + static_cast<int64_t>(r) * kRowBytes + cc * 16) =
             *reinterpret_cast<const uint4*>(stage + r * kPitch + cc * 16);
       }
-      if (hi == 0 && p.lse != nullptr) p.lse[static_cast<int64_t>(qi) * kH + row] = lse2 / kLog2eTc;
+      if (hi == 0 && lse_ptr != nullptr) lse_ptr[static_cast<int64_t>(qi) * kH + row] = lse2 / kLog2eTc;
     } else {
       // partial result of a split: normalised fp32 rows in the key buffers (padded against bank conflicts)
       constexpr int kPitchPart = kDV * 4 + 16;
@@ -531,7 +538,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       }
       if (hi == 0) {
         sm.lse_own[row] = lse2;
-        p.part_lse[(static_cast<int64_t>(qi) * p.n_split + split) * kH + row] = lse2;
+        part_lse[(static_cast<int64_t>(qi) * p.n_split + split) * kH + row] = lse2;
       }
     }
   }
@@ -550,7 +557,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     constexpr int kRowChunks = kDV / 4;   // 16-byte chunks of an fp32 row
     const uint8_t* stage = &sm.k[0][0][0];
     // rows owned by the other blocks -> global scratch, consecutive threads on consecutive chunks
-    float* mine = p.part_out + (static_cast<int64_t>(qi) * n + split) * kH * kDV;
+    float* mine = part_out + (static_cast<int64_t>(qi) * n + split) * kH * kDV;
     for (int e = tid; e < (kH - rows_per) * kRowChunks; e += kThreadsAttnTc) {
       const int fr = e / kRowChunks, cc = e % kRowChunks;
       const int r = fr < row0 ? fr : fr + rows_per;
@@ -568,7 +575,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     float my_l = -INFINITY;
     if (k_of < 3 && rl_mine < rows_per && j_of < n)
       my_l = j_of == split ? sm.lse_own[row0 + rl_mine]
-                           : __ldcg(p.part_lse + (static_cast<int64_t>(qi) * n + j_of) * kH + row0 + rl_mine);
+                           : __ldcg(part_lse + (static_cast<int64_t>(qi) * n + j_of) * kH + row0 + rl_mine);
     float m = my_l;
 #pragma unroll
     for (int d = 1; d < 8; d <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
@@ -577,9 +584,9 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
 #pragma unroll
     for (int d = 1; d < 8; d <<= 1) den += __shfl_xor_sync(0xffffffffu, den, d);
     wgt = den > 0.f ? wgt / den : 0.f;
-    if (p.lse != nullptr && j_of == 0 && k_of < 3 && rl_mine < rows_per)
-      p.lse[static_cast<int64_t>(qi) * kH + row0 + rl_mine] = den > 0.f ? (m + log2f(den)) / kLog2eTc : -INFINITY;
-    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + (static_cast<int64_t>(qi) * kH + row0) * kDV;
+    if (lse_ptr != nullptr && j_of == 0 && k_of < 3 && rl_mine < rows_per)
+      lse_ptr[static_cast<int64_t>(qi) * kH + row0 + rl_mine] = den > 0.f ? (m + log2f(den)) / kLog2eTc : -INFINITY;
+    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(out_ptr) + (static_cast<int64_t>(qi) * kH + row0) * kDV;
     for (int k = 0; k < 3; ++k) {
       const int rl = warp + kWarps * k;   // warp-uniform
       if (rl >= rows_per) break;
@@ -593,7 +600,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
 #pragma unroll
           for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const float4*>(stage + (row0 + rl) * kPitchPart + (lane + 32 * u) * 16);
         } else {
-          const float4* src = reinterpret_cast<const float4*>(p.part_out + ((static_cast<int64_t>(qi) * n + j) * kH + row0 + rl) * kDV);
+          const float4* src = reinterpret_cast<const float4*>(part_out + ((static_cast<int64_t>(qi) * n + j) * kH + row0 + rl) * kDV);
 #pragma unroll
           for (int u = 0; u < 4; ++u) v[u] = __ldcg(src + lane + 32 * u);
         }
@@ -655,17 +662,23 @@ bool attn_tc_supported(const AttnArgs& a) {
   return a.H == kH && a.DQK == kDQK && a.DV == kDV && a.v == a.k && a.ld_v == a.ld_k;
 }
 
-cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t st, int64_t* n_launch) {
-  if (a.n_query == 0) return cudaSuccess;
+cudaError_t launch_attn_tc(const AttnArgs& a_in, cudaStream_t st, int64_t* n_launch) {
+  if (a_in.n_query == 0) return cudaSuccess;
+  AttnArgs a = a_in;
+  if (a.n_layers <= 1) {   // one layer: the plain fields are the whole description
+    a.n_layers = 1;
+    a.q_l[0] = a.q; a.k_l[0] = a.k; a.out_l[0] = a.out; a.lse_l[0] = a.lse;
+  }
+  if (a.n_layers > 8) return cudaErrorInvalidValue;
   const size_t smem = sizeof(AttnTcSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(sparse_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
   if (a.n_split <= 1) {
-    sparse_attn_tc_kernel<<<dim3(a.n_query, 1), kThreadsAttnTc, smem, st>>>(a);
+    sparse_attn_tc_kernel<<<dim3(a.n_query, 1, a.n_layers), kThreadsAttnTc, smem, st>>>(a);
   } else {
     if (!attn_tc_split_ok(a.n_split)) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(a.n_query, a.n_split);
+    cfg.gridDim = dim3(a.n_query, a.n_split, a.n_layers);
     cfg.blockDim = dim3(kThreadsAttnTc);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
