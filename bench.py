@@ -35,7 +35,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--e2e-steps", type=int, default=2)
-    ap.add_argument("--cpu-queries", type=int, default=24)
+    ap.add_argument("--cpu-queries", type=int, default=256,
+                    help="queries the CPU oracle is timed on for the cpu_baseline leg (about 10 s of host work at cfg3)")
     ap.add_argument("--no-decode", action="store_true", help="skip the cfg4 decode side measurement of the default run")
     ap.add_argument("--phase", default="group", choices=["group", "index"],
                     help="group: whole lsa_layer_group step; index: indexer only (no attention tensors are allocated; for profiling)")
