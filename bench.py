@@ -308,8 +308,7 @@ def main():
     if attn_n > 0:
         dur_s = attn_ms / attn_n * 1e-3
         if decode:
-            roofline = decode_attn_roofline(cfg, prof, args.steps, positions, peaks)
-            roofline["single_layer_launch_us"] = decode_attn_launch_us(wl)
+            roofline = decode_attn_roofline(cfg, prof, decode_attn_launch_us(wl), positions, peaks)
         else:
             a = attn_flops_per_launch(cfg, positions) / dur_s / 1e12
             roofline = {"kernel": "sparse_attn_tc_kernel" if cfg.H == 64 else "sparse_attn_kernel", "bound": "tensor", "achieved": a,
@@ -375,24 +374,21 @@ def with_nominal(roofline):
     return roofline
 
 
-def decode_attn_roofline(cfg, prof, steps, positions, peaks):
-    """Decode roofline of the attention launch as lsa_layer_group issues it: on the MLA shape one launch covers the R
-    layers of the group (each with its own multi-GB cache, so nothing is found in L2), timed by the library's event
-    pair around it inside the timed steps.  `single_layer_launch_us` is the same kernel launched per layer
-    (lsa_sparse_attn back to back), for comparison."""
+def decode_attn_roofline(cfg, prof, launch_us, positions, peaks):
+    """Decode roofline of one attention launch (one layer of the group; the layers run one after another because each
+    layer's query depends on the layer before).  `launch_us` comes from one event pair around many back-to-back
+    launches (decode_attn_launch_us); `launch_us_in_step` is the library's event pair around each launch inside
+    lsa_layer_group, which adds front-end time to a launch this short."""
     attn_ms, attn_n = prof["sparse_attn"]
-    launches_per_step = attn_n / steps
-    layers_per_launch = cfg.R / launches_per_step
-    launch_us = attn_ms / attn_n * 1e3
-    bytes_per_launch = attn_bytes_per_launch(cfg, positions) * layers_per_launch
+    bytes_per_launch = attn_bytes_per_launch(cfg, positions)
     a = bytes_per_launch / (launch_us * 1e-6) / 1e9
     return with_nominal({"kernel": "sparse_attn_tc_kernel", "bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": a / peaks["hbm_gbs"],
-                         "traffic": NCU_DECODE_ATTN_DRAM_BYTES_PER_SEQ * cfg.batch * layers_per_launch,
-                         "traffic_source": "ncu capture at batch 16, one layer, scaled by sequences and layers per launch",
+                         "traffic": NCU_DECODE_ATTN_DRAM_BYTES_PER_SEQ * cfg.batch,
+                         "traffic_source": "ncu capture at batch 16, scaled by sequences per launch",
                          "algorithmic_bytes": bytes_per_launch, "peak_source": peaks["source"], "launch_us": launch_us,
-                         "layers_per_launch": layers_per_launch,
-                         "timing": "library event pair around the launch inside the timed steps"})
+                         "launch_us_in_step": attn_ms / attn_n * 1e3,
+                         "timing": "one event pair around 10 x R back-to-back launches, each layer on its own cache"})
 
 
 def decode_attn_launch_us(wl, rounds=10):
@@ -450,8 +446,7 @@ def measure_decode(cfg, dev, peaks, steps=50, warmup=10):
     prof = wl.ctx.profile_read()
     wl.ctx.profile_enable(False)
     positions = wl.ctx_len.cpu().numpy().astype(np.int64) - 1
-    roofline = decode_attn_roofline(cfg, prof, steps, positions, peaks)
-    roofline["single_layer_launch_us"] = decode_attn_launch_us(wl)
+    roofline = decode_attn_roofline(cfg, prof, decode_attn_launch_us(wl), positions, peaks)
     # running loop: every step first appends one token per sequence (indexer key quantised, sub-block mean updated,
     # one latent row per layer), then runs the group on the grown caches
     k_new = (torch.randn((cfg.batch, cfg.d_I), device=dev) / cfg.d_I ** 0.5).to(torch.bfloat16)

@@ -286,8 +286,8 @@ LSA_API int lsa_merge(lsa_ctx* ctx, const lsa_params* p, int n_parts, const void
  * index set.  q/k/v/out/lse are HOST arrays of R device pointers (lse or its entries may be NULL).
  * kmean must already hold the means (lsa_block_means) — the cache is maintained per sequence, not per
  * group.  sparse_idx / n_sparse are caller buffers, returned filled for inspection.
- * Paged mode with the (64, 576, 512) attention shape and R <= 8: the conversion rides in the indexer's last kernel and
- * the R layers attend in one launch (the split knob LSA_TUNE_ATTN_SPLIT, when set, keeps one launch per layer). */
+ * Paged mode: the conversion rides in the indexer's last kernel.  The layers are never launched side by side: in a
+ * model the query of layer r + 1 is computed from the output of layer r. */
 LSA_API int lsa_layer_group(lsa_ctx* ctx, const lsa_params* p, const void* q_idx, const float* w,
                     const void* k_idx, const float* k_scale, const void* kmean, int64_t q_pos0,
                     int64_t n_query, int64_t n_key, const int32_t* page_table, int64_t page_table_stride,

@@ -274,19 +274,10 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
 int run_attn(lsa_ctx* c, const lsa_params* p, const void* q, const void* k, const void* v, int64_t ld_k,
              int64_t ld_v, const int32_t* sparse_idx, const int32_t* n_sparse, const int32_t* rows,
              const int32_t* n_rows, int64_t q_pos0, int64_t n_query, const int32_t* ctx_len, int batch,
-             void* out, float* lse, const lsa::AttnArgs* layers = nullptr) {
-  // layers: n_layers and the per-layer arrays of a launch that covers several layers of a group (decode, tcgen05
-  // kernel); q, k, v, out, lse are then those of the first layer
+             void* out, float* lse) {
   const int64_t nq = p->paged ? batch : n_query;
   if (nq == 0) return LSA_OK;
   lsa::AttnArgs a{};
-  const int n_layers = layers ? layers->n_layers : 1;
-  if (layers) {
-    a.n_layers = n_layers;
-    for (int i = 0; i < n_layers; ++i) {
-      a.q_l[i] = layers->q_l[i]; a.k_l[i] = layers->k_l[i]; a.out_l[i] = layers->out_l[i]; a.lse_l[i] = layers->lse_l[i];
-    }
-  }
   a.H = p->n_heads; a.DQK = p->d_qk; a.DV = p->d_v; a.S = p->k_sink; a.W = p->k_swa; a.Ksp = p->k_sparse;
   a.paged = p->paged; a.sm_scale = p->sm_scale;
   a.q = q; a.k = k; a.v = v; a.ld_k = ld_k; a.ld_v = ld_v;
@@ -298,11 +289,9 @@ int run_attn(lsa_ctx* c, const lsa_params* p, const void* q, const void* k, cons
   if (p->paged) {
     const WsLayout l = ws_layout(p, nq, 0, batch);
     if (c->ws == nullptr || l.total > c->ws_bytes) return LSA_ERR_WORKSPACE;
-    // a launch over several layers has batch * n_layers independent sequences to spread over the SMs
     a.n_split = c->tune[LSA_TUNE_ATTN_SPLIT] > 0 ? c->tune[LSA_TUNE_ATTN_SPLIT]
-                                                 : pick_split(c->sm_count, batch * n_layers, a.rows_ld, use_tc);
+                                                 : pick_split(c->sm_count, batch, a.rows_ld, use_tc);
     if (use_tc && !lsa::attn_tc_split_ok(a.n_split)) return LSA_ERR_ARG;
-    if (n_layers * a.n_split > kMaxSplit) return LSA_ERR_ARG;   // the partials of all layers share the split scratch
     a.part_out = reinterpret_cast<float*>(c->ws + l.part_out);
     a.part_lse = reinterpret_cast<float*>(c->ws + l.part_lse);
   }
@@ -622,23 +611,8 @@ int lsa_layer_group(lsa_ctx* c, const lsa_params* p, const void* q_idx, const fl
   r = index_checked(c, p, q_idx, w, k_idx, k_scale, kmean, q_pos0, n_query, n_key, page_table, page_table_stride,
                     ctx_len, batch, sparse_idx, n_sparse, nullptr, rows, n_rows);
   if (r != LSA_OK) return r;
-  // Decode on the MLA shape: the layers of the group read the same rows of different caches, so they go out as one
-  // launch (grid.z = layer): twice as many independent blocks need no row splits, and the blocks' prologues and
-  // epilogues no longer fall together across the whole GPU.
-  if (p->paged && p->n_layers > 1 && p->n_layers <= 8 && c->tune[LSA_TUNE_ATTN_TC] && p->n_heads == 64) {
-    lsa::AttnArgs layers{};
-    layers.n_layers = p->n_layers;
-    bool same_shape = true;
-    for (int i = 0; i < p->n_layers; ++i) {
-      layers.q_l[i] = q[i]; layers.k_l[i] = k[i]; layers.out_l[i] = out[i]; layers.lse_l[i] = lse ? lse[i] : nullptr;
-      same_shape = same_shape && v[i] == k[i] && aligned16(q[i]) && aligned16(k[i]) && aligned16(out[i]);
-    }
-    if (same_shape && ld_v == ld_k && ld_k >= p->d_qk && ld_k % 8 == 0 &&
-        p->n_layers * pick_split(c->sm_count, batch * p->n_layers, p->k_sink + p->k_sparse + p->k_swa, true) <= kMaxSplit &&
-        c->tune[LSA_TUNE_ATTN_SPLIT] == 0)
-      return run_attn(c, p, q[0], k[0], v[0], ld_k, ld_v, sparse_idx, n_sparse, rows, n_rows, q_pos0, n_query, ctx_len, batch,
-                      out[0], lse ? lse[0] : nullptr, &layers);
-  }
+  // The layers run one after another on the stream: in a model the query of layer r + 1 is computed from the output of
+  // layer r, so they are never launched side by side.
   for (int i = 0; i < p->n_layers; ++i) {
     r = lsa_sparse_attn(c, p, q[i], k[i], v[i], ld_k, ld_v, sparse_idx, n_sparse, rows, n_rows, q_pos0, n_query,
                         n_key, ctx_len, batch, out[i], lse ? lse[i] : nullptr);

@@ -113,14 +113,13 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
   extern __shared__ uint8_t smem_raw[];
   AttnTcSmem& sm = *reinterpret_cast<AttnTcSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int qi = blockIdx.x, split = blockIdx.y, layer = blockIdx.z;
-  // this layer's tensors (a launch may cover several layers of a group: same rows, different caches)
-  const void* const q_ptr = p.q_l[layer];
-  const void* const k_ptr = p.k_l[layer];
-  void* const out_ptr = p.out_l[layer];
-  float* const lse_ptr = p.lse_l[layer];
-  float* const part_out = p.part_out + static_cast<int64_t>(layer) * p.n_query * p.n_split * kH * kDV;
-  float* const part_lse = p.part_lse + static_cast<int64_t>(layer) * p.n_query * p.n_split * kH;
+  const int qi = blockIdx.x, split = blockIdx.y;
+  const void* const q_ptr = p.q;
+  const void* const k_ptr = p.k;
+  void* const out_ptr = p.out;
+  float* const lse_ptr = p.lse;
+  float* const part_out = p.part_out;
+  float* const part_lse = p.part_lse;
 
   const bool clustered = p.n_split > 1;
   const bool dead = tc::status_raised(p.status);   // an earlier block of this launch (or an earlier launch) gave up on a wait
@@ -662,23 +661,17 @@ bool attn_tc_supported(const AttnArgs& a) {
   return a.H == kH && a.DQK == kDQK && a.DV == kDV && a.v == a.k && a.ld_v == a.ld_k;
 }
 
-cudaError_t launch_attn_tc(const AttnArgs& a_in, cudaStream_t st, int64_t* n_launch) {
-  if (a_in.n_query == 0) return cudaSuccess;
-  AttnArgs a = a_in;
-  if (a.n_layers <= 1) {   // one layer: the plain fields are the whole description
-    a.n_layers = 1;
-    a.q_l[0] = a.q; a.k_l[0] = a.k; a.out_l[0] = a.out; a.lse_l[0] = a.lse;
-  }
-  if (a.n_layers > 8) return cudaErrorInvalidValue;
+cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t st, int64_t* n_launch) {
+  if (a.n_query == 0) return cudaSuccess;
   const size_t smem = sizeof(AttnTcSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(sparse_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
   if (a.n_split <= 1) {
-    sparse_attn_tc_kernel<<<dim3(a.n_query, 1, a.n_layers), kThreadsAttnTc, smem, st>>>(a);
+    sparse_attn_tc_kernel<<<dim3(a.n_query, 1, 1), kThreadsAttnTc, smem, st>>>(a);
   } else {
     if (!attn_tc_split_ok(a.n_split)) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(a.n_query, a.n_split, a.n_layers);
+    cfg.gridDim = dim3(a.n_query, a.n_split, 1);
     cfg.blockDim = dim3(kThreadsAttnTc);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;

@@ -55,13 +55,6 @@ struct AttnArgs {
   int n_split;            // >1: partial results in part_out / part_lse, merged afterwards
   float* part_out;        // fp32 [n_query, n_split, H, DV]
   float* part_lse;        // fp32 [n_query, n_split, H]
-  // Several layers of a group in one launch of the tcgen05 kernel (grid.z = layer; same row lists, each layer its own
-  // q / cache / out): entry 0 repeats q, k, out, lse above; partials of layer z follow those of layer z-1.
-  int n_layers;           // 1..8
-  const void* q_l[8];
-  const void* k_l[8];
-  void* out_l[8];
-  float* lse_l[8];
   int* status;
 };
 
