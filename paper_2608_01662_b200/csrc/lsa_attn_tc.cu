@@ -105,11 +105,14 @@ __device__ __forceinline__ void cluster_sync_all() {
 }
 // With n_split > 1 the kernel must be launched with clusters of (1, n_split, 1) blocks: the splits of one sequence
 // are co-scheduled and merge their partial results themselves (no second kernel).  Block s finishes heads
-// [s * 64 / n_split, (s + 1) * 64 / n_split): every block keeps its own share of the rows in shared memory and writes
-// the other rows (normalised, fp32) and all its log-sum-exps to the global scratch, where they stay in L2; after one
-// cluster barrier the owner of a row combines its own part with the others'.  (Distributed shared memory moved the
+// [s * 64 / n_split, (s + 1) * 64 / n_split): every block stages its rows (normalised, fp32) in shared memory, keeps its
+// own share there and sends the other rows (one bulk copy per row) and all its log-sum-exps to the global scratch, where
+// they stay in L2; after one cluster barrier the owner of a row combines its own part with the others'.  (Distributed shared memory moved the
 // same rows at about a quarter of the L2 path's rate, so it carries nothing here.)
-__global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnArgs p) {
+//
+// q_tma != 0: q_map describes q as a bf16 matrix [n_query * 64, 576] and Q arrives as nine TMA boxes; otherwise the
+// gather warps copy it with cp.async.
+__global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, int q_tma, AttnArgs p) {
   extern __shared__ uint8_t smem_raw[];
   AttnTcSmem& sm = *reinterpret_cast<AttnTcSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -129,7 +132,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
   if (tid == 0) {
     LSA_TL(0);
     LSA_WALL(0);
-    tc::mbar_init(smem_u32(&sm.q_full), 32 * kLoadWarps);
+    tc::mbar_init(smem_u32(&sm.q_full), q_tma ? 1 : 32 * kLoadWarps);
     tc::mbar_init(smem_u32(&sm.q_tmem), kSoftmaxWarps);
     for (int b = 0; b < kKBufs; ++b) {
       tc::mbar_init(smem_u32(&sm.k_full[b]), 32 * kLoadWarps);
@@ -155,6 +158,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
   // draining; what earlier kernels wrote is read only from here on.  The next kernel's blocks may be placed from now.
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (tid == 0) LSA_TL(13);
 
   // ---- this query's row list (same conventions as the mma.sync kernel)
   const int64_t t = p.paged ? static_cast<int64_t>(p.ctx_len[qi]) - 1 : p.q_pos0 + qi;
@@ -189,19 +193,28 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     const int lt = tid - 32 * (kSoftmaxWarps + kMmaWarps);   // 0..127
     {
       // Q of this query: the rope part (dims 512-575) stays in shared memory as an MMA operand; dims 0-511 are staged
-      // in the last key buffer (64 rows x 1024 B, 16-byte chunks swizzled by row) for the softmax warps, which move
-      // them to tensor memory.  The copies share the first cp.async group, handed over with the first key tile.
-      const uint8_t* qg = reinterpret_cast<const uint8_t*>(q_ptr) + static_cast<int64_t>(qi) * kH * kDQK * 2;
-      for (int e = lt; e < kH * 8; e += 32 * kLoadWarps) {
-        const int r = e >> 3, c = e & 7;
-        cp_async16(smem_u32(sm.q_rope) + r * 128 + ((c ^ (r & 7)) << 4), qg + r * kDQK * 2 + 512 * 2 + c * 16, 16);
-      }
+      // in the last key buffer for the softmax warps, which move them to tensor memory.  As TMA boxes they complete
+      // q_full by themselves; as cp.async copies they form the first group, handed over with the first key tile.
+      // Both ways leave dims 64a .. 64a+63 of the 64 rows in column block a of that buffer, 128-byte swizzled.
       const uint32_t stage = smem_u32(sm.k[kKBufs - 1]);
-      for (int e = lt; e < kH * 64; e += 32 * kLoadWarps) {
-        const int r = e >> 6, c = e & 63;
-        cp_async16(stage + r * 1024 + ((c ^ (r & 7)) << 4), qg + r * kDQK * 2 + c * 16, 16);
+      if (q_tma) {
+        if (lt == 0) {
+          tc::mbar_expect_tx(smem_u32(&sm.q_full), kH * kDQK * 2);
+          for (int a = 0; a < kAtoms; ++a)
+            tc::tma_load_2d(a < 8 ? stage + a * kAtomBytes : smem_u32(sm.q_rope), &q_map, a * 64, qi * kH, smem_u32(&sm.q_full));
+        }
+      } else {
+        const uint8_t* qg = reinterpret_cast<const uint8_t*>(q_ptr) + static_cast<int64_t>(qi) * kH * kDQK * 2;
+        for (int e = lt; e < kH * 8; e += 32 * kLoadWarps) {
+          const int r = e >> 3, c = e & 7;
+          cp_async16(smem_u32(sm.q_rope) + r * 128 + ((c ^ (r & 7)) << 4), qg + r * kDQK * 2 + 512 * 2 + c * 16, 16);
+        }
+        for (int e = lt; e < kH * 64; e += 32 * kLoadWarps) {
+          const int r = e >> 6, c = e & 63;
+          cp_async16(stage + (c >> 3) * kAtomBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4), qg + r * kDQK * 2 + c * 16, 16);
+        }
+        cp_async_commit();
       }
-      cp_async_commit();
     }
     // Every gather warp works on every tile: warp w copies rows 16w .. 16w+15, so a freed buffer is refilled by all
     // four warps at once.  Lanes 0-15 look up the cache row of their key once; the row number is then broadcast
@@ -216,11 +229,12 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     // Copies of up to three tiles are in flight: a tile is handed to the MMA issuers (k_full) when its cp.async group
     // has landed, which is looked at after the next tile's copies are issued, or at once when no buffer is free.
     int first_pend = 0, n_pend = 0;   // tiles first_pend .. first_pend + n_pend - 1 are issued but not handed over
-    bool q_handed = false;
+    bool q_handed = q_tma != 0;       // TMA completes q_full by itself
     auto hand_over_q = [&]() {        // call after a wait that covers the first group
       tc::fence_proxy_async();
       tc::mbar_arrive(smem_u32(&sm.q_full));
       q_handed = true;
+      if (lt == 0) LSA_TL(15);
     };
     auto hand_over_oldest = [&]() {
       if (n_pend >= 3) cp_async_wait<2>();
@@ -257,6 +271,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
           cp_async16(smem_u32(sm.k[b][c >> 3]) + r * 128 + (((c & 7) ^ (r & 7)) << 4), src + c * 16, nb);
       }
       cp_async_commit();
+      if (lt == 0 && i == 0) LSA_TL(14);
       ++n_pend;
       if (n_pend == kKBufs) hand_over_oldest();
       my_row = next_row;
@@ -326,7 +341,6 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
           if (tc::mbar_test(smem_u32(&sm.k_full[qk_next % kKBufs]), (qk_next / kKBufs) & 1) &&
               tc::mbar_test(smem_u32(&sm.pv_done[qk_next & 1]), ((qk_next >> 1) & 1) ^ 1)) {
             if (x == 0 && qk_next == 0) LSA_TL(3);
-            if (x == 0 && qk_next == 22) LSA_TL(15);
             issue_qk(qk_next++);
             did = true;
           }
@@ -358,14 +372,14 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     {
       // Q[row, 256*hi : 256*hi+256] from the staging buffer -> 128 columns of this lane, in the order the tensor core
       // reads an A operand (two consecutive dims per 32-bit column)
-      const uint8_t* qs = sm.k[kKBufs - 1][0] + row * 1024;
+      const uint8_t* qs = sm.k[kKBufs - 1][0] + row * 128;
 #pragma unroll 1
       for (int part = 0; part < 2; ++part) {
         uint32_t w[64];
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
           const int c = 32 * hi + 16 * part + j;
-          const uint4 u = *reinterpret_cast<const uint4*>(qs + ((c ^ (row & 7)) << 4));
+          const uint4 u = *reinterpret_cast<const uint4*>(qs + (c >> 3) * kAtomBytes + (((c & 7) ^ (row & 7)) << 4));
           w[4 * j] = u.x; w[4 * j + 1] = u.y; w[4 * j + 2] = u.z; w[4 * j + 3] = u.w;
         }
         tc::tmem_st64(tmem_base + lane_addr + kColQ + part * 64, w);
@@ -383,7 +397,6 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
       if (!ok) break;
       if (tid == 0 && i == 0) LSA_TL(4);
       if (tid == 0 && i == 20) LSA_TL(10);
-      if (tid == 0 && i == 21) LSA_TL(14);
       tc::fence_after_sync();
       const uint32_t s_addr = tmem_base + lane_addr + kColS + b * kSBuf;
       uint32_t v[32];
@@ -539,6 +552,18 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
         sm.lse_own[row] = lse2;
         part_lse[(static_cast<int64_t>(qi) * p.n_split + split) * kH + row] = lse2;
       }
+      // Rows that another block of the cluster finishes go to the global scratch as soon as this warp has staged them:
+      // one bulk copy per row (2 KB), issued by the lane that holds the row's first half, while the other softmax warps
+      // are still staging.
+      tc::fence_proxy_async();
+      __syncwarp();
+      const int rows_per = kH / p.n_split;
+      if (hi == 0 && row / rows_per != split) {
+        float* dst = part_out + ((static_cast<int64_t>(qi) * p.n_split + split) * kH + row) * kDV;
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                     :: "l"(dst), "r"(smem_u32(stage + row * kPitchPart)), "n"(kDV * 4) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      }
     }
   }
   if (tid == 0) LSA_TL(8);
@@ -553,22 +578,30 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     const int rows_per = kH / n;
     const int row0 = split * rows_per;
     constexpr int kPitchPart = kDV * 4 + 16;
-    constexpr int kRowChunks = kDV / 4;   // 16-byte chunks of an fp32 row
     const uint8_t* stage = &sm.k[0][0][0];
-    // rows owned by the other blocks -> global scratch, consecutive threads on consecutive chunks
-    float* mine = part_out + (static_cast<int64_t>(qi) * n + split) * kH * kDV;
-    for (int e = tid; e < (kH - rows_per) * kRowChunks; e += kThreadsAttnTc) {
-      const int fr = e / kRowChunks, cc = e % kRowChunks;
-      const int r = fr < row0 ? fr : fr + rows_per;
-      *reinterpret_cast<float4*>(mine + r * kDV + cc * 4) = *reinterpret_cast<const float4*>(stage + r * kPitchPart + cc * 16);
+    if (warp < kSoftmaxWarps) {   // the threads that sent rows wait until they are written (not only read out of shared memory)
+      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+      __threadfence();
     }
-    __threadfence();
     if (tid == 0) LSA_TL(10);
     cluster_sync_all();   // every block of the cluster has written its rows
     if (tid == 0) LSA_TL(11);
     // Warp w finishes rows w, w + 12, ... of this block's share (at most three).  Lane 8k + j first fetches the
     // log-sum-exp of split j for the warp's k-th row, so that all of them are in flight together.
     constexpr int kWarps = kThreadsAttnTc / 32;
+    // two splits (the usual decode case): the peer's parts of all of this warp's rows are requested before the first is used
+    float4 pre[3][4];
+    if (n == 2) {
+#pragma unroll
+      for (int k = 0; k < 3; ++k) {
+        const int rl = warp + kWarps * k;
+        if (rl < rows_per) {
+          const float4* src = reinterpret_cast<const float4*>(part_out + ((static_cast<int64_t>(qi) * 2 + (split ^ 1)) * kH + row0 + rl) * kDV);
+#pragma unroll
+          for (int u = 0; u < 4; ++u) pre[k][u] = __ldcg(src + lane + 32 * u);
+        }
+      }
+    }
     const int k_of = lane >> 3, j_of = lane & 7;
     const int rl_mine = warp + kWarps * k_of;
     float my_l = -INFINITY;
@@ -586,34 +619,39 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(AttnA
     if (lse_ptr != nullptr && j_of == 0 && k_of < 3 && rl_mine < rows_per)
       lse_ptr[static_cast<int64_t>(qi) * kH + row0 + rl_mine] = den > 0.f ? (m + log2f(den)) / kLog2eTc : -INFINITY;
     __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(out_ptr) + (static_cast<int64_t>(qi) * kH + row0) * kDV;
+#pragma unroll
     for (int k = 0; k < 3; ++k) {
       const int rl = warp + kWarps * k;   // warp-uniform
-      if (rl >= rows_per) break;
-      float4 acc[4];
+      if (rl < rows_per) {
+        float4 acc[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int j = 0; j < n; ++j) {
-        const float w = __shfl_sync(0xffffffffu, wgt, 8 * k + j);
-        float4 v[4];
-        if (j == split) {
+        for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int j = 0; j < n; ++j) {
+          const float w = __shfl_sync(0xffffffffu, wgt, 8 * k + j);
+          float4 v[4];
+          if (j == split) {
 #pragma unroll
-          for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const float4*>(stage + (row0 + rl) * kPitchPart + (lane + 32 * u) * 16);
-        } else {
-          const float4* src = reinterpret_cast<const float4*>(part_out + ((static_cast<int64_t>(qi) * n + j) * kH + row0 + rl) * kDV);
+            for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const float4*>(stage + (row0 + rl) * kPitchPart + (lane + 32 * u) * 16);
+          } else if (n == 2) {
 #pragma unroll
-          for (int u = 0; u < 4; ++u) v[u] = __ldcg(src + lane + 32 * u);
+            for (int u = 0; u < 4; ++u) v[u] = pre[k][u];
+          } else {
+            const float4* src = reinterpret_cast<const float4*>(part_out + ((static_cast<int64_t>(qi) * n + j) * kH + row0 + rl) * kDV);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[u] = __ldcg(src + lane + 32 * u);
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            acc[u].x += w * v[u].x; acc[u].y += w * v[u].y; acc[u].z += w * v[u].z; acc[u].w += w * v[u].w;
+          }
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          acc[u].x += w * v[u].x; acc[u].y += w * v[u].y; acc[u].z += w * v[u].z; acc[u].w += w * v[u].w;
+          uint2 o;
+          o.x = pack_bf16(acc[u].x, acc[u].y);
+          o.y = pack_bf16(acc[u].z, acc[u].w);
+          *reinterpret_cast<uint2*>(out + static_cast<int64_t>(rl) * kDV + (lane + 32 * u) * 4) = o;
         }
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        uint2 o;
-        o.x = pack_bf16(acc[u].x, acc[u].y);
-        o.y = pack_bf16(acc[u].z, acc[u].w);
-        *reinterpret_cast<uint2*>(out + static_cast<int64_t>(rl) * kDV + (lane + 32 * u) * 4) = o;
       }
     }
     if (tid == 0) LSA_TL(12);
@@ -666,8 +704,11 @@ cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t st, int64_t* n_launch
   const size_t smem = sizeof(AttnTcSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(sparse_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
+  CUtensorMap q_map{};
+  const int q_tma = (reinterpret_cast<uintptr_t>(a.q) & 15u) == 0 &&
+                    make_map_bf16_rows(&q_map, a.q, kDQK, static_cast<uint64_t>(a.n_query) * kH, kH);
   if (a.n_split <= 1) {
-    sparse_attn_tc_kernel<<<dim3(a.n_query, 1, 1), kThreadsAttnTc, smem, st>>>(a);
+    sparse_attn_tc_kernel<<<dim3(a.n_query, 1, 1), kThreadsAttnTc, smem, st>>>(q_map, q_tma, a);
   } else {
     if (!attn_tc_split_ok(a.n_split)) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg{};
@@ -684,7 +725,7 @@ cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t st, int64_t* n_launch
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    e = cudaLaunchKernelEx(&cfg, sparse_attn_tc_kernel, a);
+    e = cudaLaunchKernelEx(&cfg, sparse_attn_tc_kernel, q_map, q_tma, a);
     if (e != cudaSuccess) {
       if (getenv("LSA_DEBUG")) fprintf(stderr, "[lsa] cluster launch (%d x %d blocks) failed: %s\n", a.n_query, a.n_split, cudaGetErrorString(e));
       return e;

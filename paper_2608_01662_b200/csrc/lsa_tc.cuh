@@ -218,5 +218,6 @@ bool tma_available();
 // Tensor map of a bf16 matrix [rows, 128] row-major: box = 64 columns x box_rows rows, 128-byte swizzle, zero fill
 // outside.  `base` must be 16-byte aligned.
 bool make_map_bf16_128(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows);
+bool make_map_bf16_rows(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint32_t box_rows);
 
 }  // namespace lsa
