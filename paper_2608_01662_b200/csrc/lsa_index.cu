@@ -12,6 +12,21 @@
 #include "lsa_internal.h"
 #include "lsa_select.cuh"
 
+#ifdef LSA_TIMELINE
+// Debug build only: SM-clock stamps of the fine kernel's phases per block, read back with lsa_debug_timeline_fine.
+__device__ long long g_tl_fine[1024 * 8];
+#define LSA_TLF(k)                                                              \
+  do {                                                                          \
+    const unsigned blk_ = blockIdx.x + gridDim.x * blockIdx.y;                  \
+    if (threadIdx.x == 0 && blk_ < 1024) g_tl_fine[blk_ * 8 + (k)] = clock64(); \
+  } while (0)
+extern "C" __attribute__((visibility("default"))) int lsa_debug_timeline_fine(long long* host, int n_blocks) {
+  return cudaMemcpyFromSymbol(host, g_tl_fine, sizeof(long long) * 8 * (n_blocks < 1024 ? n_blocks : 1024)) == cudaSuccess ? 0 : -1;
+}
+#else
+#define LSA_TLF(k)
+#endif
+
 namespace lsa {
 
 namespace {
@@ -405,17 +420,20 @@ struct FineSmem {
   uint32_t keys[kMaxSlots];
   float scale[2][kTileRows];   // per-token key scales of the tile in flight (e4m3 keys)
   int32_t pages[kMaxPages];
+  int32_t phys[kMaxPages];     // where each selected page lives in the cache (page-table entry; the page itself when contiguous)
   SelectScratch sel;
 };
 
 template <int HI, int DI, bool E4M3>
-__global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
+__global__ void __launch_bounds__(kThreads, 2) fine_select_kernel(IndexArgs p) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   auto& sm = *reinterpret_cast<FineSmem<HI, DI>*>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int qi = blockIdx.x;
+  LSA_TLF(0);
   pdl_wait();
   pdl_launch_dependents();
+  LSA_TLF(1);
   int64_t t, n_key;
   const int32_t* pt = nullptr;
   if (p.paged) {
@@ -450,6 +468,7 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
       // the six passes of the radix select then run out of shared memory
       for (int i = tid; i < nE; i += kThreads) sm.keys[i] = score_key(ps[i]);
       __syncthreads();
+      LSA_TLF(7);
       nP = block_select_topk([&](int i) { return sm.keys[i]; }, [&](int i) { return p0 + i; }, nE, p.M, sm.pages, sm.sel);
     } else {
       nP = block_select_topk([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M,
@@ -459,11 +478,15 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
     nP = nE;  // host guarantees nE <= kMaxSlots / P here
     for (int i = tid; i < nP; i += kThreads) sm.pages[i] = p0 + i;
   }
+  LSA_TLF(2);
   // ---- query heads and weights -> shared
   load_q_async<HI, DI>(smem_u32(sm.q), reinterpret_cast<const __nv_bfloat16*>(p.q_idx) + static_cast<int64_t>(qi) * HI * DI);
   if (tid < HI / 4) cp_async16(smem_u32(&sm.w[tid * 4]), p.w + static_cast<int64_t>(qi) * HI + tid * 4, 16);
   cp_async_commit();
   __syncthreads();  // sm.pages visible
+  // one page-table lookup per selected page, not one per copied chunk
+  for (int i = tid; i < nP; i += kThreads) sm.phys[i] = p.paged ? pt[sm.pages[i]] : sm.pages[i];
+  __syncthreads();
   if (out_pages && part == 0) for (int i = tid; i < p.M; i += kThreads) out_pages[i] = i < nP ? sm.pages[i] : -1;
   if (n_parts > 1 && part == 0) {
     int32_t* fp = p.fine_pages + qi * (kMaxPages + 1);
@@ -478,9 +501,7 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
   const int n_tiles = max(0, min(n_tiles_all, tile0 + tiles_per) - tile0);
   const int pshift = 31 - __clz(p.P);
   auto slot_pos = [&](int c) -> int64_t { return static_cast<int64_t>(sm.pages[c >> pshift]) * p.P + (c & (p.P - 1)); };
-  auto phys_row = [&](int64_t pos) -> int64_t {
-    return p.paged ? static_cast<int64_t>(pt[pos >> pshift]) * p.P + (pos & (p.P - 1)) : pos;
-  };
+  auto slot_row = [&](int c) -> int64_t { return static_cast<int64_t>(sm.phys[c >> pshift]) * p.P + (c & (p.P - 1)); };
   const uint8_t* kbase = reinterpret_cast<const uint8_t*>(p.k_idx);
 
   // Tile loaders.  bf16 keys go global -> shared asynchronously; e4m3 keys are read into registers one
@@ -488,16 +509,19 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
   constexpr int U = DI / 8;                           // 16-byte bf16 units per row
   constexpr int CU = DI / 16;                         // 16-byte code units per row (e4m3)
   constexpr int kCodePerThread = kTileRows * CU / kThreads;
-  uint4 staged[E4M3 ? kCodePerThread : 1];
-  float staged_scale = 0.f;
-  auto issue_tile = [&](int tile, int buf) {
+  // e4m3: kDepth tiles are in flight in registers (a gathered tile takes several microseconds to arrive from a
+  // multi-GB cache; one tile ahead left the loop waiting on it)
+  constexpr int kDepth = E4M3 ? 3 : 1;
+  uint4 staged_all[kDepth][E4M3 ? kCodePerThread : 1];
+  float staged_scale_all[kDepth];
+  auto issue_tile = [&](int tile, int buf, uint4* staged, float& staged_scale) {
     if constexpr (E4M3) {
       if (tid < kTileRows) {   // this row's scale travels with the tile instead of being fetched after the MMAs
         const int c = tile * kTileRows + tid;
         staged_scale = 0.f;
         if (c < n_slots) {
           const int64_t pos = slot_pos(c);
-          if (pos < n_key) staged_scale = p.k_scale[phys_row(pos)];
+          if (pos < n_key) staged_scale = p.k_scale[slot_row(c)];
         }
       }
 #pragma unroll
@@ -507,7 +531,7 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
         uint4 v = make_uint4(0, 0, 0, 0);
         if (c < n_slots) {
           const int64_t pos = slot_pos(c);
-          if (pos < n_key) v = *reinterpret_cast<const uint4*>(kbase + phys_row(pos) * DI + u * 16);
+          if (pos < n_key) v = *reinterpret_cast<const uint4*>(kbase + slot_row(c) * DI + u * 16);
         }
         staged[j] = v;
       }
@@ -521,13 +545,13 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
           pos = slot_pos(c);
           ok = pos < n_key;
         }
-        cp_async16(smem_u32(sm.a[buf]) + swz<DI * 2>(r, u), kbase + (ok ? phys_row(pos) : 0) * DI * 2 + u * 16,
+        cp_async16(smem_u32(sm.a[buf]) + swz<DI * 2>(r, u), kbase + (ok ? slot_row(c) : 0) * DI * 2 + u * 16,
                    ok ? 16 : 0);
       }
       cp_async_commit();
     }
   };
-  auto land_tile = [&](int buf) {
+  auto land_tile = [&](int buf, const uint4* staged, float staged_scale) {
     if constexpr (E4M3) {
       if (tid < kTileRows) sm.scale[buf][tid] = staged_scale;
 #pragma unroll
@@ -541,13 +565,22 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
     }
   };
 
-  if (n_tiles > 0) issue_tile(tile0, 0);
-  for (int tile = tile0; tile < tile0 + n_tiles; ++tile) {
-    const int buf = (tile - tile0) & 1;
-    land_tile(buf);
+#pragma unroll
+  for (int d = 0; d < kDepth; ++d)
+    if (d < n_tiles) issue_tile(tile0 + d, d & 1, staged_all[d], staged_scale_all[d]);
+  for (int base = 0; base < n_tiles; base += kDepth) {
+#pragma unroll
+   for (int d = 0; d < kDepth; ++d) {
+    const int it = base + d;           // block-uniform
+    if (it >= n_tiles) break;
+    const int tile = tile0 + it;
+    const int buf = it & 1;
+    land_tile(buf, staged_all[d], staged_scale_all[d]);
     cp_async_wait<0>();
     __syncthreads();  // tile `tile` (and, first time, q/w) in shared; buffer buf^1 free
-    if (tile + 1 < tile0 + n_tiles) issue_tile(tile + 1, buf ^ 1);
+    if (it == 0) LSA_TLF(3);
+    if (it == 3) LSA_TLF(4);
+    if (it + kDepth < n_tiles) issue_tile(tile + kDepth, (it + kDepth) & 1, staged_all[d], staged_scale_all[d]);
     uint32_t a[DI / 16][4];
     load_a_frags<DI>(a, smem_u32(sm.a[buf]));
     float s_lo, s_hi;
@@ -568,13 +601,16 @@ __global__ void __launch_bounds__(kThreads) fine_select_kernel(IndexArgs p) {
         }
       }
     }
+   }
   }
   __syncthreads();
+  LSA_TLF(5);
   if (n_parts > 1) {
     // hand this block's share of the candidate keys to the top-K kernel
     uint32_t* fk = p.fine_keys + static_cast<int64_t>(qi) * kMaxSlots;
     const int c0 = tile0 * kTileRows, c1 = min(n_slots, (tile0 + n_tiles) * kTileRows);
     for (int c = c0 + tid; c < c1; c += kThreads) fk[c] = sm.keys[c];
+    LSA_TLF(6);
     return;
   }
   const int n_sel = block_select_topk([&](int i) { return sm.keys[i]; },
