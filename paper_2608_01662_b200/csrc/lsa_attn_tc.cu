@@ -4,8 +4,9 @@
 // One thread block = one query (or one row split of one sequence in decode).  Its 64 heads are the M = 64
 // rows of every MMA; the attended cache rows stream through a ring of three 64-key shared tiles:
 //
-//   warps 8-11  gather: rows [sink | sparse | window] -> 128B-swizzled K-major tiles with coalesced 16-byte
-//               cp.async, up to three tiles in flight, each handed over through an mbarrier when it has landed.
+//   warps 8-11  gather: rows [window | sink | sparse] (or the caller's row list) -> 128B-swizzled K-major tiles with
+//               coalesced 16-byte cp.async, up to three tiles in flight, each handed over through an mbarrier when it
+//               has landed; tiles of 64 consecutive window rows come as nine TMA boxes instead.
 //               Q arrives the same way: its rope dims (512-575) stay in shared memory as an MMA operand, dims 0-511
 //               are staged in the last tile buffer for the softmax warps
 //   warps 4-7   one thread each issues tcgen05.mma.  Back-to-back MMAs into one accumulator run far below the
@@ -111,8 +112,11 @@ __device__ __forceinline__ void cluster_sync_all() {
 // same rows at about a quarter of the L2 path's rate, so it carries nothing here.)
 //
 // q_tma != 0: q_map describes q as a bf16 matrix [n_query * 64, 576] and Q arrives as nine TMA boxes; otherwise the
-// gather warps copy it with cp.async.
-__global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, int q_tma, AttnArgs p) {
+// gather warps copy it with cp.async.  k_tma != 0 (contiguous caches only): k_map describes the cache rows, and key
+// tiles that lie wholly inside the window, 64 consecutive rows, arrive as nine TMA boxes as well.
+__global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, int q_tma,
+                                                                            const __grid_constant__ CUtensorMap k_map, int k_tma,
+                                                                            AttnArgs p) {
   extern __shared__ uint8_t smem_raw[];
   AttnTcSmem& sm = *reinterpret_cast<AttnTcSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -162,7 +166,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
 
   // ---- this query's row list (same conventions as the mma.sync kernel)
   const int64_t t = p.paged ? static_cast<int64_t>(p.ctx_len[qi]) - 1 : p.q_pos0 + qi;
-  int n_sink = 0, n_sp = 0, n_tot;
+  int n_sink = 0, n_sp = 0, n_win = 0, n_tot;
   int64_t win0 = 0;
   const int32_t* rows = nullptr;
   if (p.rows != nullptr) {
@@ -171,16 +175,19 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
   } else {
     n_sink = static_cast<int>(min64(p.S, t + 1));
     win0 = max64(p.S, t - p.W + 1);
+    n_win = static_cast<int>(max64(0, t - win0 + 1));
     n_sp = p.n_sparse[qi];
-    n_tot = n_sink + n_sp + static_cast<int>(max64(0, t - win0 + 1));
+    n_tot = n_sink + n_sp + n_win;
   }
   const int32_t* sp = p.sparse_idx ? p.sparse_idx + static_cast<int64_t>(qi) * p.Ksp : nullptr;
+  // Without a row list the keys are visited as [window | sink | sparse] (the order within one softmax is free): the
+  // window is a run of consecutive cache rows, so its whole tiles need no per-row addressing.
   auto row_of = [&](int i) -> int32_t {
     if (i >= n_tot) return -1;
     if (rows) return rows[i];
-    if (i < n_sink) return i;
-    if (i < n_sink + n_sp) return sp[i - n_sink];
-    return static_cast<int32_t>(win0 + (i - n_sink - n_sp));
+    if (i < n_win) return static_cast<int32_t>(win0 + i);
+    if (i < n_win + n_sink) return i - n_win;
+    return sp[i - n_win - n_sink];
   };
   const int tiles_all = (n_tot + kTileKeys - 1) / kTileKeys;
   const int tiles_per = (tiles_all + p.n_split - 1) / p.n_split;
@@ -222,8 +229,11 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
     const int lw = lt >> 5;
     constexpr int kRowsPerWarp = kTileKeys / kLoadWarps;
     const uint8_t* kg = reinterpret_cast<const uint8_t*>(k_ptr);
+    auto tile_by_tma = [&](int i) -> bool {   // block-uniform
+      return k_tma && rows == nullptr && (tile_begin + i + 1) * kTileKeys <= n_win;
+    };
     auto my_key_row = [&](int i) -> int32_t {
-      return (i < n_tiles && lane < kRowsPerWarp) ? row_of((tile_begin + i) * kTileKeys + kRowsPerWarp * lw + lane) : -1;
+      return (i < n_tiles && lane < kRowsPerWarp && !tile_by_tma(i)) ? row_of((tile_begin + i) * kTileKeys + kRowsPerWarp * lw + lane) : -1;
     };
     int32_t my_row = my_key_row(0);
     // Copies of up to three tiles are in flight: a tile is handed to the MMA issuers (k_full) when its cp.async group
@@ -260,15 +270,26 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       }
       while (n_pend > 0 && !__all_sync(0xffffffffu, tc::mbar_test(smem_u32(&sm.k_empty[b]), par))) hand_over_oldest();
       if (!__all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.k_empty[b]), par, p.status))) break;
+      if (tile_by_tma(i)) {
+        // 64 consecutive window rows: nine boxes that complete k_full by byte count; the (empty) cp.async group
+        // below keeps the hand-over bookkeeping the same for both kinds of tile
+        if (lt == 0) {
+          tc::mbar_expect_tx_only(smem_u32(&sm.k_full[b]), kAtoms * kAtomBytes);
+          const int row0 = static_cast<int>(win0) + (tile_begin + i) * kTileKeys;
+          for (int a = 0; a < kAtoms; ++a)
+            tc::tma_load_2d(smem_u32(sm.k[b][a]), &k_map, a * 64, row0, smem_u32(&sm.k_full[b]));
+        }
+      } else {
 #pragma unroll 4
-      for (int rr = 0; rr < kRowsPerWarp; ++rr) {
-        const int32_t row = __shfl_sync(0xffffffffu, my_row, rr);
-        const int r = kRowsPerWarp * lw + rr;
-        const uint8_t* src = kg + static_cast<int64_t>(row >= 0 ? row : 0) * p.ld_k * 2;
-        const int nb = row >= 0 ? 16 : 0;
+        for (int rr = 0; rr < kRowsPerWarp; ++rr) {
+          const int32_t row = __shfl_sync(0xffffffffu, my_row, rr);
+          const int r = kRowsPerWarp * lw + rr;
+          const uint8_t* src = kg + static_cast<int64_t>(row >= 0 ? row : 0) * p.ld_k * 2;
+          const int nb = row >= 0 ? 16 : 0;
 #pragma unroll
-        for (int c = lane; c < 72; c += 32)
-          cp_async16(smem_u32(sm.k[b][c >> 3]) + r * 128 + (((c & 7) ^ (r & 7)) << 4), src + c * 16, nb);
+          for (int c = lane; c < 72; c += 32)
+            cp_async16(smem_u32(sm.k[b][c >> 3]) + r * 128 + (((c & 7) ^ (r & 7)) << 4), src + c * 16, nb);
+        }
       }
       cp_async_commit();
       if (lt == 0 && i == 0) LSA_TL(14);
@@ -518,14 +539,14 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
           *reinterpret_cast<uint4*>(my_stage + (c + 8 * j) * 2) = w4;
         }
       }
+      tc::fence_proxy_async();
       __syncwarp();
       uint8_t* dst = reinterpret_cast<uint8_t*>(reinterpret_cast<__nv_bfloat16*>(out_ptr) + static_cast<int64_t>(qi) * kH * kDV);
-      constexpr int kChunksPerRow = kRowBytes / 16;
-#pragma unroll 4
-      for (int e = lane; e < 16 * kChunksPerRow; e += 32) {   // this warp's 16 rows
-        const int r = 16 * quarter + e / kChunksPerRow, cc = e % kChunksPerRow;
-        *reinterpret_cast<uint4*>(dst + static_cast<int64_t>(r) * kRowBytes + cc * 16) =
-            *reinterpret_cast<const uint4*>(stage + r * kPitch + cc * 16);
+      if (hi == 0) {   // one bulk copy per row, issued by the lane that staged the row's first half
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                     :: "l"(dst + static_cast<int64_t>(row) * kRowBytes), "r"(smem_u32(stage + row * kPitch)), "n"(kRowBytes) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the staging buffer must outlive the copy
       }
       if (hi == 0 && lse_ptr != nullptr) lse_ptr[static_cast<int64_t>(qi) * kH + row] = lse2 / kLog2eTc;
     } else {
@@ -704,11 +725,14 @@ cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t st, int64_t* n_launch
   const size_t smem = sizeof(AttnTcSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(sparse_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
-  CUtensorMap q_map{};
+  CUtensorMap q_map{}, k_map{};
   const int q_tma = (reinterpret_cast<uintptr_t>(a.q) & 15u) == 0 &&
                     make_map_bf16_rows(&q_map, a.q, kDQK, static_cast<uint64_t>(a.n_query) * kH, kH);
+  // contiguous cache: the last query sees rows 0 .. q_pos0 + n_query - 1, so the cache holds at least that many
+  const int k_tma = !a.paged && a.rows == nullptr && a.ld_k % 8 == 0 && (reinterpret_cast<uintptr_t>(a.k) & 15u) == 0 &&
+                    make_map_bf16_rows(&k_map, a.k, static_cast<uint64_t>(a.ld_k), static_cast<uint64_t>(a.q_pos0 + a.n_query), kTileKeys);
   if (a.n_split <= 1) {
-    sparse_attn_tc_kernel<<<dim3(a.n_query, 1, 1), kThreadsAttnTc, smem, st>>>(q_map, q_tma, a);
+    sparse_attn_tc_kernel<<<dim3(a.n_query, 1, 1), kThreadsAttnTc, smem, st>>>(q_map, q_tma, k_map, k_tma, a);
   } else {
     if (!attn_tc_split_ok(a.n_split)) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg{};
@@ -725,7 +749,7 @@ cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t st, int64_t* n_launch
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    e = cudaLaunchKernelEx(&cfg, sparse_attn_tc_kernel, q_map, q_tma, a);
+    e = cudaLaunchKernelEx(&cfg, sparse_attn_tc_kernel, q_map, q_tma, k_map, k_tma, a);
     if (e != cudaSuccess) {
       if (getenv("LSA_DEBUG")) fprintf(stderr, "[lsa] cluster launch (%d x %d blocks) failed: %s\n", a.n_query, a.n_split, cudaGetErrorString(e));
       return e;
