@@ -157,6 +157,26 @@ def test_prefill_query_window_with_offset_matches_whole_run(cuda_device):
     assert torch.equal(chunked.sparse_idx, full.sparse_idx) and torch.equal(chunked.out[0], full.out[0])
 
 
+def test_attention_on_cache_rows_with_padding(cuda_device):
+    """The latent cache may be a view of wider rows (ld_k > d_qk): same output as on packed rows, both where key tiles
+    are whole window runs and where they are gathered row by row."""
+    cfg = SMALL_MLA.replace(R=1)
+    wl = PrefillWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.step()
+    assert wl.ctx.status() == 0
+    packed = wl.k[0]
+    wide = torch.zeros((packed.shape[0], cfg.d_qk + 64), dtype=packed.dtype, device=cuda_device)
+    wide[:, :cfg.d_qk] = packed
+    wide[:, cfg.d_qk:] = 7.0                                           # must never be read
+    view = wide[:, :cfg.d_qk]
+    assert view.stride(0) == cfg.d_qk + 64
+    out = torch.empty_like(wl.out[0])
+    wl.ctx.sparse_attn(wl.q[0], view, view, wl.sparse_idx, wl.n_sparse, 0, wl.n_query, wl.n_key, out)
+    assert wl.ctx.status() == 0
+    assert torch.equal(out, wl.out[0])
+
+
 def test_runs_are_deterministic(cuda_device):
     wl = PrefillWorkload(SMALL_FP8, cuda_device)
     wl.prepare()
