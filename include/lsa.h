@@ -123,8 +123,11 @@ LSA_API int64_t lsa_launch_count(lsa_ctx* ctx);
  *   LSA_TUNE_ATTN_TC        1 (default): MLA-shape attention on tcgen05.mma; 0: the mma.sync kernel
  *   LSA_TUNE_ATTN_SPLIT     row splits per sequence in paged attention: 0 (default) = chosen by the wave cost model,
  *                           1..16 = fixed (the tcgen05 kernel merges its splits inside a thread-block cluster and
- *                           accepts 1, 2, 4 or 8; other values make lsa_sparse_attn return LSA_ERR_ARG there) */
-enum { LSA_TUNE_COARSE_GROUPS = 0, LSA_TUNE_ATTN_TC, LSA_TUNE_ATTN_SPLIT, LSA_TUNE_COUNT };
+ *                           accepts 1, 2, 4 or 8; other values make lsa_sparse_attn return LSA_ERR_ARG there)
+ *   LSA_TUNE_ATTN_PV_WAIT   prefill on the tcgen05 attention kernel.  0 (default): the Q K^T of a tile follows the P V that
+ *                           frees its accumulator in the issuing thread's program order; 1: it waits for that P V's
+ *                           completion barrier (slower, same bits).  Paged calls always wait. */
+enum { LSA_TUNE_COARSE_GROUPS = 0, LSA_TUNE_ATTN_TC, LSA_TUNE_ATTN_SPLIT, LSA_TUNE_ATTN_PV_WAIT, LSA_TUNE_COUNT };
 LSA_API int lsa_tune(lsa_ctx* ctx, int knob, int value);
 
 /* Per-kernel timing.  While enabled, every kernel-launching call records a CUDA event pair on the

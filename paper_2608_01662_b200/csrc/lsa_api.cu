@@ -285,6 +285,8 @@ int run_attn(lsa_ctx* c, const lsa_params* p, const void* q, const void* k, cons
   a.rows_ld = p->k_sink + p->k_sparse + p->k_swa;
   a.q_pos0 = q_pos0; a.n_query = static_cast<int>(nq); a.ctx_len = ctx_len; a.out = out; a.lse = lse;
   a.n_split = 1; a.status = status_word(c);
+  a.qk_waits_pv = c->tune[LSA_TUNE_ATTN_PV_WAIT];
+  a.pv_issuers = p->paged ? 4 : 2;   // decode waits on HBM gathers, prefill on the tensor pipe
   const bool use_tc = c->tune[LSA_TUNE_ATTN_TC] && lsa::attn_tc_supported(a);
   if (p->paged) {
     const WsLayout l = ws_layout(p, nq, 0, batch);
@@ -400,6 +402,7 @@ int lsa_tune(lsa_ctx* c, int knob, int value) {
   if (c == nullptr || knob < 0 || knob >= LSA_TUNE_COUNT) return LSA_ERR_ARG;
   if (knob == LSA_TUNE_COARSE_GROUPS && value != 1 && value != 2) return LSA_ERR_ARG;
   if (knob == LSA_TUNE_ATTN_SPLIT && (value < 0 || value > kMaxSplit)) return LSA_ERR_ARG;
+  if (knob == LSA_TUNE_ATTN_PV_WAIT && value != 0 && value != 1) return LSA_ERR_ARG;
   c->tune[knob] = value;
   return LSA_OK;
 }

@@ -9,14 +9,25 @@
 //               has landed; tiles of 64 consecutive window rows come as nine TMA boxes instead.
 //               Q arrives the same way: its rope dims (512-575) stay in shared memory as an MMA operand, dims 0-511
 //               are staged in the last tile buffer for the softmax warps
-//   warps 4-7   one thread each issues tcgen05.mma.  Back-to-back MMAs into one accumulator run far below the
-//               pipe's rate at these small shapes, so each product is cut into independent accumulation chains:
-//                 S = Q K^T   issuers 0 and 1: dims 0-255 / 256-511 with Q from tensor memory (16 steps of M64 N64
-//                             K16 each) plus two rope steps with Q from shared memory; the two partial sums land in
-//                             the two lane halves of the S buffer
-//                 O += P V    all four issuers: value dims 128x .. 128x+127 (M64 N128 K16 x 4 per tile) with P from
-//                             tensor memory; V is the key tile read MN-major, so each cache row is fetched once
-//               A thread takes whichever of "next Q K^T" / "next P V" is ready.
+//   warps 4-7   one thread each issues tcgen05.mma.  Back-to-back MMAs into one accumulator run far below the pipe's
+//               rate at these small shapes, so each product is cut into independent accumulation chains:
+//                 S = Q K^T   issuers 0 and 1: dims 256x .. 256x+255 with Q from tensor memory (16 steps of M64 N64
+//                             K16) plus two rope steps with Q from shared memory; the partial sum of issuer x lands in
+//                             lane half x of the S buffer
+//                 O += P V    with P from tensor memory; V is the key tile read MN-major, so each cache row is fetched
+//                             once.  Two layouts (AttnArgs::pv_issuers):
+//                             2 (prefill)  issuer x: value dims 256x .. 256x+255 (M64 N256 K16 x 4 per tile), P from lane
+//                                          half x, O in lane half x: an issuer owns everything in its lane half
+//                             4 (decode)   issuer x: value dims 128x .. 128x+127 (M64 N128 K16 x 4 per tile)
+//               A thread takes whichever of "next Q K^T" / "next P V" is ready.  The S buffer of tile i+1 still holds
+//               P of tile i-1 in its first columns.  With four issuers Q K^T(i+1) waits for the completion barrier of
+//               P V(i-1); the P V issuers that do no Q K^T release a key buffer as early as possible, which is what a
+//               decode step, waiting on HBM gathers, needs.  With two issuers the P V that reads those columns and the
+//               Q K^T that overwrites them are issued by the same thread, in that order, and touch only that thread's
+//               lane half, so the tensor core's in-order execution of one thread's MMAs keeps them apart: Q K^T(i+1)
+//               is queued right behind P V(i-1) and the pipe never idles for a barrier round trip between them (4 % of
+//               a prefill step).  AttnArgs::qk_waits_pv (tuning knob LSA_TUNE_ATTN_PV_WAIT) brings the barrier back;
+//               both ways give the same bits, which a test checks.
 //   warps 0-3   softmax: move Q to tensor memory once; per tile tcgen05.ld of both partial sums, add, running max
 //               with lazy rescaling of O, exp2, fp32 row sums, P as bf16 -> tensor memory (A operand of P V); at the
 //               end O / l through shared memory to global in whole rows
@@ -76,11 +87,6 @@ constexpr int kAtomBytes = 64 * 128;         // 64 rows x 128 bytes
 constexpr int kHalfKeys = 32;
 
 constexpr int kSoftmaxWarps = 4, kMmaWarps = 4, kLoadWarps = 4;
-#ifndef LSA_PV_ISSUERS
-#define LSA_PV_ISSUERS 4
-#endif
-constexpr int kPvIssuers = LSA_PV_ISSUERS;   // 4: one per 128 value dims; 2: one per 256 (N = 256 MMAs; measured 6 % slower:
-                                             // an M = 64 MMA of N = 256 takes twice the time of N = 128, and two threads issue everything)
 constexpr int kThreadsAttnTc = 32 * (kSoftmaxWarps + kMmaWarps + kLoadWarps);
 constexpr uint32_t kTmemColsAttn = 512;
 constexpr int kKBufs = 3;                    // 64-key tile buffers in shared memory
@@ -128,6 +134,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
   float* const part_out = p.part_out;
   float* const part_lse = p.part_lse;
 
+  const int n_pv = p.pv_issuers == 4 ? 4 : 2;   // threads that issue P V (see the header: 2 = lane-half ownership)
   const bool clustered = p.n_split > 1;
   const bool dead = tc::status_raised(p.status);   // an earlier block of this launch (or an earlier launch) gave up on a wait
   if (dead && !clustered) return;
@@ -140,11 +147,11 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
     tc::mbar_init(smem_u32(&sm.q_tmem), kSoftmaxWarps);
     for (int b = 0; b < kKBufs; ++b) {
       tc::mbar_init(smem_u32(&sm.k_full[b]), 32 * kLoadWarps);
-      tc::mbar_init(smem_u32(&sm.k_empty[b]), kPvIssuers);
+      tc::mbar_init(smem_u32(&sm.k_empty[b]), n_pv);
     }
     for (int b = 0; b < 2; ++b) {
       tc::mbar_init(smem_u32(&sm.s_full[b]), 2);
-      tc::mbar_init(smem_u32(&sm.pv_done[b]), kPvIssuers);
+      tc::mbar_init(smem_u32(&sm.pv_done[b]), n_pv);
       tc::mbar_init(smem_u32(&sm.p_ready[b]), kSoftmaxWarps);
     }
     tc::fence_mbar_init();
@@ -311,14 +318,14 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
 #else
       constexpr uint32_t idesc_qk = tc::idesc_bf16(kH, kTileKeys, 0, 0);
 #endif
-      constexpr uint32_t idesc_pv = tc::idesc_bf16(kH, kPvIssuers == 4 ? 128 : 256, 0, 1);   // B = V read MN-major
+      const uint32_t idesc_pv = n_pv == 4 ? tc::idesc_bf16(kH, 128, 0, 1) : tc::idesc_bf16(kH, 256, 0, 1);   // B = V read MN-major
       bool ok = tc::mbar_wait(smem_u32(&sm.q_full), 0, p.status) && tc::mbar_wait(smem_u32(&sm.q_tmem), 0, p.status);
       if (x == 0) LSA_TL(2);
       // Descriptors are built once; inside the loops only the start-address word moves (one add per operand).
       constexpr uint32_t kBufBytes = kAtoms * kAtomBytes;
       const uint64_t dqr = tc::smem_desc_sw128(smem_u32(sm.q_rope), 16, 1024);
       const uint64_t dk0 = tc::smem_desc_sw128(smem_u32(sm.k), 16, 1024);           // K-major view (Q K^T)
-      const uint64_t dv0 = tc::desc_advance(tc::smem_desc_sw128(smem_u32(sm.k), kAtomBytes, 1024), (kPvIssuers == 4 ? 2 : 4) * x * kAtomBytes);  // MN-major view (P V)
+      const uint64_t dv0 = tc::desc_advance(tc::smem_desc_sw128(smem_u32(sm.k), kAtomBytes, 1024), (n_pv == 4 ? 2 : 4) * x * kAtomBytes);  // MN-major view (P V)
       constexpr uint32_t kLane16 = 16u << 16;
       // Q K^T (issuers 0 and 1): chain x = dims 256x .. 256x+255 with Q from tensor memory (lane half x), plus two of
       // the four rope steps with Q from shared memory; its partial sum goes to lane half x of the S buffer
@@ -326,8 +333,8 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       const uint32_t s_dst = tmem_base + (x & 1) * kLane16 + kColS;
       // P V (all four issuers): value dims 128x .. 128x+127 = columns 128*(x&1) .. of the accumulator in lane half
       // x>>1; P is read from the same lane half
-      const uint32_t o_dst = kPvIssuers == 4 ? tmem_base + (x >> 1) * kLane16 + (x & 1) * 128 : tmem_base + (x & 1) * kLane16;
-      const uint32_t p_src = tmem_base + (kPvIssuers == 4 ? (x >> 1) : (x & 1)) * kLane16 + kColS;
+      const uint32_t o_dst = n_pv == 4 ? tmem_base + (x >> 1) * kLane16 + (x & 1) * 128 : tmem_base + (x & 1) * kLane16;
+      const uint32_t p_src = tmem_base + (n_pv == 4 ? (x >> 1) : (x & 1)) * kLane16 + kColS;
       auto issue_qk = [&](int i) {
         tc::fence_after_sync();
         const uint32_t d = s_dst + (i & 1) * kSBuf;
@@ -351,8 +358,9 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
         tc::umma_commit(smem_u32(&sm.pv_done[j & 1]));
       };
       const bool does_qk = x < 2;
+      const bool wait_pv = p.qk_waits_pv != 0 || n_pv != 2;
       // Two in-order queues, "next Q K^T" (at most one tile ahead of the softmax it feeds) and "next P V".
-      int qk_next = does_qk ? 0 : n_tiles, pv_next = x < kPvIssuers ? 0 : n_tiles;
+      int qk_next = does_qk ? 0 : n_tiles, pv_next = x < n_pv ? 0 : n_tiles;
       long long t_idle = clock64();
       uint32_t spins = 0;
       while (ok && pv_next < n_tiles) {
@@ -360,7 +368,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
         if (qk_next < n_tiles && qk_next <= pv_next + 1) {
           // S buffer qk_next&1 also holds P of tile qk_next-2: it is free once that tile's P V has completed
           if (tc::mbar_test(smem_u32(&sm.k_full[qk_next % kKBufs]), (qk_next / kKBufs) & 1) &&
-              tc::mbar_test(smem_u32(&sm.pv_done[qk_next & 1]), ((qk_next >> 1) & 1) ^ 1)) {
+              (!wait_pv || tc::mbar_test(smem_u32(&sm.pv_done[qk_next & 1]), ((qk_next >> 1) & 1) ^ 1))) {
             if (x == 0 && qk_next == 0) LSA_TL(3);
             issue_qk(qk_next++);
             did = true;

@@ -52,6 +52,8 @@ struct AttnArgs {
   const int32_t* ctx_len;
   void* out;              // bf16 [n_query, H, DV]
   float* lse;             // optional [n_query, H]
+  int pv_issuers;         // tcgen05 kernel: 2 = an issuer owns a lane half (prefill), 4 = one P V issuer per 128 value dims
+  int qk_waits_pv;        // tcgen05 kernel, 2 issuers: Q K^T of tile i+1 waits for the completion barrier of P V of tile i-1
   int n_split;            // >1: partial results in part_out / part_lse, merged afterwards
   float* part_out;        // fp32 [n_query, n_split, H, DV]
   float* part_lse;        // fp32 [n_query, n_split, H]

@@ -177,6 +177,21 @@ def test_attention_on_cache_rows_with_padding(cuda_device):
     assert torch.equal(out, wl.out[0])
 
 
+def test_attention_issue_order_and_completion_barrier_give_the_same_bits(cuda_device):
+    """The tcgen05 attention kernel queues the Q K^T of a tile behind the P V that frees its accumulator (same issuing
+    thread, program order); LSA_TUNE_ATTN_PV_WAIT = 1 makes it wait for that P V's completion barrier instead.  Same
+    arithmetic in the same order either way, so the outputs must be equal bit for bit."""
+    cfg = SMALL_MLA.replace(R=1)
+    wl = PrefillWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.step()
+    fast_out, fast_lse = wl.out[0].clone(), wl.lse[0].clone()
+    wl.ctx.tune(3, 1)                 # LSA_TUNE_ATTN_PV_WAIT
+    wl.step()
+    assert wl.ctx.status() == 0
+    assert torch.equal(wl.out[0], fast_out) and torch.equal(wl.lse[0], fast_lse)
+
+
 def test_runs_are_deterministic(cuda_device):
     wl = PrefillWorkload(SMALL_FP8, cuda_device)
     wl.prepare()
