@@ -170,6 +170,13 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid == 0) LSA_TL(13);
+  // Q is requested before anything else is looked up: a block cannot start without it, and in prefill it comes from HBM.
+  if (q_tma && tid == 32 * (kSoftmaxWarps + kMmaWarps)) {
+    const uint32_t stage = smem_u32(sm.k[kKBufs - 1]);
+    tc::mbar_expect_tx(smem_u32(&sm.q_full), kH * kDQK * 2);
+    for (int a = 0; a < kAtoms; ++a)
+      tc::tma_load_2d(a < 8 ? stage + a * kAtomBytes : smem_u32(sm.q_rope), &q_map, a * 64, qi * kH, smem_u32(&sm.q_full));
+  }
 
   // ---- this query's row list (same conventions as the mma.sync kernel)
   const int64_t t = p.paged ? static_cast<int64_t>(p.ctx_len[qi]) - 1 : p.q_pos0 + qi;
@@ -211,13 +218,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       // q_full by themselves; as cp.async copies they form the first group, handed over with the first key tile.
       // Both ways leave dims 64a .. 64a+63 of the 64 rows in column block a of that buffer, 128-byte swizzled.
       const uint32_t stage = smem_u32(sm.k[kKBufs - 1]);
-      if (q_tma) {
-        if (lt == 0) {
-          tc::mbar_expect_tx(smem_u32(&sm.q_full), kH * kDQK * 2);
-          for (int a = 0; a < kAtoms; ++a)
-            tc::tma_load_2d(a < 8 ? stage + a * kAtomBytes : smem_u32(sm.q_rope), &q_map, a * 64, qi * kH, smem_u32(&sm.q_full));
-        }
-      } else {
+      if (!q_tma) {
         const uint8_t* qg = reinterpret_cast<const uint8_t*>(q_ptr) + static_cast<int64_t>(qi) * kH * kDQK * 2;
         for (int e = lt; e < kH * 8; e += 32 * kLoadWarps) {
           const int r = e >> 3, c = e & 7;
