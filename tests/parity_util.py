@@ -9,7 +9,9 @@ from oracle import reference_run as ref
 
 TOL_BF16 = dict(max_abs=2e-2, rel_l2=5e-3)
 TOL_FP8 = dict(max_abs=5e-2, rel_l2=1e-2)
-MIN_OVERLAP = 0.995
+MIN_OVERLAP = 0.995          # mean over the checked queries (the end-to-end bar)
+MIN_OVERLAP_ANY = 0.98       # no single query may fall below this (a near-tie flips a handful of its 2048 tokens at most)
+MAX_PAGE_DIFF_SHARE = 0.02   # share of checked queries whose kept page set differs from the oracle's (near-tie at rank M)
 
 
 def to_np(t: torch.Tensor) -> np.ndarray:
@@ -34,12 +36,14 @@ def boundary_queries(cfg, q_pos0, n_query, n_random, seed=0):
 class Metrics:
     def __init__(self):
         self.overlaps, self.page_diff, self.max_abs, self.num, self.den = [], 0, 0.0, 0.0, 0.0
-        self.lse_abs, self.n = 0.0, 0
+        self.lse_abs, self.n, self.n_pages = 0.0, 0, 0
 
     def add_select(self, gpu_sparse, ref_sparse, gpu_pages=None, ref_pages=None):
         self.overlaps.append(ref.overlap(gpu_sparse, ref_sparse))
-        if gpu_pages is not None and list(gpu_pages) != list(ref_pages):
-            self.page_diff += 1
+        if gpu_pages is not None:
+            self.n_pages += 1
+            if list(gpu_pages) != list(ref_pages):
+                self.page_diff += 1
         self.n += 1
 
     def add_out(self, gpu_out, ref_out, gpu_lse=None, ref_lse=None):
@@ -66,6 +70,9 @@ class Metrics:
     def assert_ok(self, tol):
         s = self.summary()
         assert s["mean_overlap"] >= MIN_OVERLAP, s
+        assert s["min_overlap"] >= MIN_OVERLAP_ANY, s
+        if self.n_pages:
+            assert self.page_diff <= max(1, int(MAX_PAGE_DIFF_SHARE * self.n_pages)), s
         assert s["max_abs"] <= tol["max_abs"] and s["rel_l2"] <= tol["rel_l2"], s
         assert s["lse_abs"] <= 1e-3, s
 

@@ -23,6 +23,10 @@ def test_reference_arm_prints_one_json_line():
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["value"] == d["value"]
     assert d["e2e"] == {"value": d["value"], "unit": d["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     assert d["config"]["workload"] == "cfg1" and d["gpu_launches"] == 0
+    # both arms describe the workload with the same object
+    import bench
+    from paper_2608_01662_b200.configs import CONFIGS
+    assert d["config"] == bench.config_dict(CONFIGS["cfg1"], CONFIGS["cfg1"].L)
 
 
 def test_reference_arm_is_silent_on_other_ranks():

@@ -67,15 +67,17 @@ def test_cfg4_decode_all_sequences(cuda_device):
     _free()
 
 
-@pytest.mark.parametrize("chunk", [0, 37, 63])
+@pytest.mark.parametrize("chunk", [0, 1, 17, 37, 50, 63])
 def test_cfg5_prefill_1m_chunks(cuda_device, chunk):
-    """1M-token caches resident; the queries of one 16384-query chunk at a time."""
+    """1M-token caches resident; the queries of one 16384-query chunk at a time.  Six chunks (the first, where the
+    number of eligible pages crosses M, its neighbour, four spread over the rest including the last) with the boundary
+    positions plus 34 random queries each: more than 200 random queries in total."""
     cfg = CONFIGS["cfg5"]
     wl = PrefillWorkload(cfg, cuda_device, q_pos0=chunk * cfg.q_chunk, n_query=cfg.q_chunk)
     wl.prepare()
     wl.step()
     assert wl.ctx.status() == 0
-    m = pu.check_prefill(wl, pu.boundary_queries(cfg, wl.q_pos0, wl.n_query, 24, seed=chunk))
+    m = pu.check_prefill(wl, pu.boundary_queries(cfg, wl.q_pos0, wl.n_query, 34, seed=chunk))
     print("cfg5 chunk", chunk, m.summary())
     m.assert_ok(pu.TOL_FP8)
     del wl
