@@ -49,6 +49,7 @@ def parse_args():
     ap.add_argument("--flat", action="store_true", help="hi_enable = 0: flat indexer (Eq. 7) instead of the hierarchy")
     ap.add_argument("--attn-split", type=int, default=0, help="override LSA_TUNE_ATTN_SPLIT (decode row splits)")
     ap.add_argument("--attn-pv-wait", type=int, default=-1, help="override LSA_TUNE_ATTN_PV_WAIT (0 or 1)")
+    ap.add_argument("--attn-gather", type=int, default=-1, help="override LSA_TUNE_ATTN_GATHER (0: cp.async rows, 1: TMA gather4)")
     ap.add_argument("--coarse-groups", type=int, default=0, help="override LSA_TUNE_COARSE_GROUPS (1 or 2)")
     return ap.parse_args()
 
@@ -259,6 +260,8 @@ def main():
         wl.ctx.tune(2, args.attn_split)
     if args.attn_pv_wait >= 0:
         wl.ctx.tune(3, args.attn_pv_wait)
+    if args.attn_gather >= 0:
+        wl.ctx.tune(4, args.attn_gather)
     torch.cuda.synchronize()
 
     def barrier():

@@ -126,8 +126,13 @@ LSA_API int64_t lsa_launch_count(lsa_ctx* ctx);
  *                           accepts 1, 2, 4 or 8; other values make lsa_sparse_attn return LSA_ERR_ARG there)
  *   LSA_TUNE_ATTN_PV_WAIT   prefill on the tcgen05 attention kernel.  0 (default): the Q K^T of a tile follows the P V that
  *                           frees its accumulator in the issuing thread's program order; 1: it waits for that P V's
- *                           completion barrier (slower, same bits).  Paged calls always wait. */
-enum { LSA_TUNE_COARSE_GROUPS = 0, LSA_TUNE_ATTN_TC, LSA_TUNE_ATTN_SPLIT, LSA_TUNE_ATTN_PV_WAIT, LSA_TUNE_COUNT };
+ *                           completion barrier (slower, same bits).  Paged calls always wait.
+ *   LSA_TUNE_ATTN_GATHER    tcgen05 attention kernel, scattered cache rows.  0 (default): coalesced 16-byte cp.async
+ *                           copies; 1: TMA gather, four rows per cp.async.bulk.tensor tile::gather4 instruction (needs a
+ *                           16-byte aligned cache whose row pitch is a multiple of 16 bytes, else the other path is
+ *                           taken).  Same bits; the TMA path measured 1.3 x slower (512 bytes per instruction). */
+enum { LSA_TUNE_COARSE_GROUPS = 0, LSA_TUNE_ATTN_TC, LSA_TUNE_ATTN_SPLIT, LSA_TUNE_ATTN_PV_WAIT, LSA_TUNE_ATTN_GATHER,
+       LSA_TUNE_COUNT };
 LSA_API int lsa_tune(lsa_ctx* ctx, int knob, int value);
 
 /* Per-kernel timing.  While enabled, every kernel-launching call records a CUDA event pair on the
@@ -203,7 +208,7 @@ LSA_API int lsa_index(lsa_ctx* ctx, const lsa_params* p, const void* q_idx, cons
               int32_t* sparse_idx, int32_t* n_sparse, int32_t* pages_out);
 
 /* lsa_index for callers that can give the library no scratch memory.  (The paper has no counterpart:
- * this is a packaging variant of the prefill indexer above, same kernels, same results.)
+ * this is a packaging variant of the prefill indexer above.)
  *
  * Who needs it: code that runs where device memory can no longer be obtained — inside a serving engine
  * that reserved the whole GPU for its own pools at start-up, from a plugin or callback that is handed
@@ -215,21 +220,42 @@ LSA_API int lsa_index(lsa_ctx* ctx, const lsa_params* p, const void* q_idx, cons
  * until the process exits.  The call takes no lsa_ctx, allocates nothing on host or device and calls no
  * allocating routine.
  *
- * Arguments as lsa_index with paged = 0 (contiguous caches, query row i at position q_pos0+i); `device`
- * is the CUDA device of all pointers, `cuda_stream` the stream to enqueue on.  No pages_out.
+ * Kernels and results: the coarse stage is dispatched exactly as lsa_index dispatches it and the fine stage
+ * is the same kernel, so sparse_idx / n_sparse are the ones lsa_index returns for the same inputs.  One
+ * difference in speed: for e4m3 caches with the 64-head indexer lsa_index first writes a bf16 copy of the
+ * codes into its workspace and feeds the fine stage from it by TMA; there is no room for that copy here, so
+ * the fine stage gathers the codes and widens them in registers, which is slower.
+ *
+ * Arguments as lsa_index with paged = 0 (contiguous caches, query row i at position q_pos0+i) and the same
+ * argument checks (LSA_ERR_SHAPE for a q_idx, w, k_idx or kmean that is not 16-byte aligned); `device` is the
+ * CUDA device of all pointers, `cuda_stream` the stream to enqueue on.  No pages_out.  The caller's current
+ * device is the same after the call as before it.
  * Limits and behaviour:
  *   - n_query * (ceil(n_key/P) rounded up to 4) * 4 bytes must not exceed LSA_STATIC_SCRATCH_BYTES, else
- *     LSA_ERR_CAPACITY and nothing is launched; split the queries over several calls.
- *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
- *     device made current); make that first call before any stream capture begins.
+ *     LSA_ERR_CAPACITY and nothing is launched; split the queries over several calls.  Mean pooling,
+ *     keep_pages * page <= 4096, and with hi_enable = 0 caches of at most 4096 tokens.
+ *   - The first call on each device is a set-up call: it looks up the arrays' device addresses
+ *     (cudaGetSymbolAddress, with that device made current), which is also when the CUDA runtime loads
+ *     this part of the library onto the device — the array's bytes and the kernels' code are obtained from
+ *     the driver then, not at dlopen.  Make that first call at start-up, before the application reserves
+ *     the rest of the GPU's memory and before any stream capture begins; if the device has no room left
+ *     it returns LSA_ERR_CUDA.
  *   - All calls on a device share the one array, which keeps the previous call's contents.  Nothing in it
  *     has to start at zero (the fine stage reads only entries the coarse stage of the same call wrote).
  *     Two calls whose kernels overlap on the GPU — different streams, or different host threads — race on
- *     it: order them on one stream or with events. */
+ *     it: order them on one stream or with events.
+ *   - Device-side waits are bounded as everywhere in the library.  A wait that ran out leaves
+ *     LSA_ERR_TIMEOUT in a status word that sits beside the array and is shared in the same way; read it
+ *     with lsa_index_static_status. */
 #define LSA_STATIC_SCRATCH_BYTES (8u << 20)
 LSA_API int lsa_index_static(int device, void* cuda_stream, const lsa_params* p, const void* q_idx, const float* w,
                              const void* k_idx, const float* k_scale, const void* kmean, int64_t q_pos0,
                              int64_t n_query, int64_t n_key, int32_t* sparse_idx, int32_t* n_sparse);
+/* Waits for `cuda_stream`, copies the status word of lsa_index_static on `device` to *device_status (0, or
+ * LSA_ERR_TIMEOUT if a device-side wait of an earlier lsa_index_static call ran out, in which case that
+ * call's outputs are not valid) and clears it.  Allocates nothing; the counterpart of lsa_status for the
+ * entry point that has no context.  (No counterpart in the paper.) */
+LSA_API int lsa_index_static_status(int device, void* cuda_stream, int* device_status);
 
 /* The selection step alone (Eq. 2 / 7 / 10 / 12) on caller-given fp32 scores; bit-exact by definition.
  *   scores    fp32 [n_query, ld_scores], column c of row i is the score of candidate c

@@ -53,6 +53,7 @@ EXPORTS = {
                           c_int64, c_int64, c_void_p, c_int64, c_void_p, c_int, c_void_p, c_void_p, c_void_p]),
     "lsa_index_static": (c_int, [c_int, c_void_p, POINTER(LsaParams), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                  c_int64, c_int64, c_int64, c_void_p, c_void_p]),
+    "lsa_index_static_status": (c_int, [c_int, c_void_p, POINTER(c_int)]),
     "lsa_select": (c_int, [c_void_p, POINTER(LsaParams), c_void_p, c_int64, c_void_p, c_int64, c_int64, c_int64,
                            c_int32, c_int32, c_void_p, c_void_p]),
     "lsa_convert": (c_int, [c_void_p, POINTER(LsaParams), c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_int64,
@@ -140,6 +141,17 @@ def index_static(params: LsaParams, q_idx, w, k_idx, k_scale, kmean, q_pos0, n_q
                                _p(k_idx), _p(k_scale), _p(kmean), q_pos0, n_query, n_key, _p(sparse_idx), _p(n_sparse))
     if r != 0:
         raise LsaError(r, "lsa_index_static")
+
+
+def index_static_status(device, stream=None) -> int:
+    """lsa_index_static_status: waits for the stream, returns and clears the status word of lsa_index_static."""
+    dev = torch.device(device)
+    stream = stream if stream is not None else torch.cuda.current_stream(dev)
+    st = c_int(0)
+    r = lib().lsa_index_static_status(dev.index or 0, c_void_p(stream.cuda_stream), ctypes.byref(st))
+    if r != 0:
+        raise LsaError(r, "lsa_index_static_status")
+    return st.value
 
 
 class Context:

@@ -22,6 +22,10 @@ struct lsa_ctx {
   cudaEvent_t ev_in[2], ev_done[2], ev_out[2];
   // per-kernel timing (lsa_profile_*): event pairs recorded around the launches of each kernel class
   int tune[LSA_TUNE_COUNT];
+  // Row lists of the last kernel launched through this context, if that kernel was a paged attention launch: the next
+  // attention launch on the same lists may read them ahead of its programmatic dependency wait (the lists were
+  // complete before that last kernel started).  Any other launch through the context clears it.
+  const void* last_attn_rows;
   int prof_on;
   int prof_n;
   cudaEvent_t* prof_ev;   // 2 * kProfPairs events, created on first enable
@@ -42,6 +46,7 @@ constexpr int64_t kFlatFusedMaxKeys = 4096;   // caches up to this length: the f
 template <class F>
 cudaError_t timed(lsa_ctx* c, int cat, F launch) {
   const bool rec = c->prof_on && c->prof_ev != nullptr && c->prof_n < kProfPairs;
+  if (cat != LSA_K_ATTN) c->last_attn_rows = nullptr;
   if (rec) cudaEventRecord(c->prof_ev[2 * c->prof_n], c->stream);
   const cudaError_t e = launch();
   if (rec) {
@@ -90,6 +95,29 @@ int check_params(const lsa_params* p, bool need_index, bool need_attn) {
   }
   return LSA_OK;
 }
+
+}  // namespace
+
+int lsa::check_index_call(const lsa_params* p, const void* q_idx, const float* w, const void* k_idx, const float* k_scale,
+                          const void* kmean, int64_t q_pos0, int64_t n_query, int64_t n_key, const int32_t* page_table,
+                          int64_t page_table_stride, const int32_t* ctx_len, int batch, const int32_t* sparse_idx,
+                          const int32_t* n_sparse) {
+  const int r = check_params(p, true, false);
+  if (r != LSA_OK) return r;
+  if (q_idx == nullptr || w == nullptr || k_idx == nullptr || sparse_idx == nullptr || n_sparse == nullptr) return LSA_ERR_ARG;
+  if (p->hi_enable && kmean == nullptr) return LSA_ERR_ARG;
+  if (p->key_dtype == LSA_KEY_E4M3 && k_scale == nullptr) return LSA_ERR_ARG;
+  if (n_query < 0 || n_key < 0 || q_pos0 < 0) return LSA_ERR_ARG;
+  if (p->paged) {
+    if (page_table == nullptr || ctx_len == nullptr || batch <= 0 || page_table_stride <= 0) return LSA_ERR_ARG;
+  } else if (q_pos0 + n_query > n_key) {
+    return LSA_ERR_ARG;
+  }
+  if (!aligned16(q_idx) || !aligned16(w) || !aligned16(k_idx) || (kmean && !aligned16(kmean))) return LSA_ERR_SHAPE;
+  return LSA_OK;
+}
+
+namespace {
 
 // Workspace map.  All offsets are multiples of 256 bytes.
 struct WsLayout {
@@ -226,10 +254,7 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
       lsa::IndexArgs d = a;
       d.P = 1; d.B = 1; d.M = 0; d.kmean = keys_bf16; d.hi_enable = 1;
       if (e == cudaSuccess)
-        e = timed(c, LSA_K_COARSE, [&] {
-          return lsa::coarse_tc_supported(d) ? lsa::launch_coarse_tc(d, c->tune[LSA_TUNE_COARSE_GROUPS], c->stream, &c->launches)
-                                             : lsa::launch_coarse(d, c->stream, &c->launches);
-        });
+        e = timed(c, LSA_K_COARSE, [&] { return lsa::launch_coarse_best(d, c->tune[LSA_TUNE_COARSE_GROUPS], c->stream, &c->launches); });
       if (e == cudaSuccess)
         e = timed(c, LSA_K_SELECT, [&] {
           return lsa::launch_select(a.page_scores, a.ps_ld, nullptr, a.key_e4m3 ? k_scale : nullptr, a.q_pos0, a.n_query,
@@ -244,10 +269,7 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
     if (p->hi_enable && p->pooling == LSA_POOL_MINMAX)
       e = timed(c, LSA_K_COARSE, [&] { return lsa::launch_coarse_minmax(a, c->stream, &c->launches); });
     else if (p->hi_enable)
-      e = timed(c, LSA_K_COARSE, [&] {
-        return lsa::coarse_tc_supported(a) ? lsa::launch_coarse_tc(a, c->tune[LSA_TUNE_COARSE_GROUPS], c->stream, &c->launches)
-                                           : lsa::launch_coarse(a, c->stream, &c->launches);
-      });
+      e = timed(c, LSA_K_COARSE, [&] { return lsa::launch_coarse_best(a, c->tune[LSA_TUNE_COARSE_GROUPS], c->stream, &c->launches); });
     if (e == cudaSuccess && l.big_keys != 0) {
       // recall budget beyond one block's shared memory: page lists, fine scores through the workspace, top-K over them
       if (!lsa::fine_big_supported(a)) return LSA_ERR_SHAPE;
@@ -287,6 +309,8 @@ int run_attn(lsa_ctx* c, const lsa_params* p, const void* q, const void* k, cons
   a.n_split = 1; a.status = status_word(c);
   a.qk_waits_pv = c->tune[LSA_TUNE_ATTN_PV_WAIT];
   a.pv_issuers = p->paged ? 4 : 2;   // decode waits on HBM gathers, prefill on the tensor pipe
+  a.gather4 = c->tune[LSA_TUNE_ATTN_GATHER];
+  a.rows_stable = rows != nullptr && c->last_attn_rows == rows;
   const bool use_tc = c->tune[LSA_TUNE_ATTN_TC] && lsa::attn_tc_supported(a);
   if (p->paged) {
     const WsLayout l = ws_layout(p, nq, 0, batch);
@@ -301,6 +325,7 @@ int run_attn(lsa_ctx* c, const lsa_params* p, const void* q, const void* k, cons
   cudaError_t e = timed(c, LSA_K_ATTN, [&] {
     return use_tc ? lsa::launch_attn_tc(a, c->stream, &c->launches) : lsa::launch_attn(a, c->stream, &c->launches);
   });
+  c->last_attn_rows = (e == cudaSuccess && use_tc && p->paged) ? rows : nullptr;
   if (e == cudaSuccess && a.n_split > 1 && !use_tc) e = timed(c, LSA_K_MERGE, [&] { return lsa::launch_merge(a, c->stream, &c->launches); });
   return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
 }
@@ -325,6 +350,7 @@ int lsa_create(lsa_ctx** ctx, int device, void* cuda_stream, void* workspace, si
   c->ws_bytes = workspace ? workspace_bytes : 0;
   c->tune[LSA_TUNE_COARSE_GROUPS] = 2;
   c->tune[LSA_TUNE_ATTN_TC] = 1;
+  c->tune[LSA_TUNE_ATTN_GATHER] = 0;   // measured: the TMA unit paces four-row gathers below what 16-byte cp.async reaches
   e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking);
@@ -403,6 +429,7 @@ int lsa_tune(lsa_ctx* c, int knob, int value) {
   if (knob == LSA_TUNE_COARSE_GROUPS && value != 1 && value != 2) return LSA_ERR_ARG;
   if (knob == LSA_TUNE_ATTN_SPLIT && (value < 0 || value > kMaxSplit)) return LSA_ERR_ARG;
   if (knob == LSA_TUNE_ATTN_PV_WAIT && value != 0 && value != 1) return LSA_ERR_ARG;
+  if (knob == LSA_TUNE_ATTN_GATHER && value != 0 && value != 1) return LSA_ERR_ARG;
   c->tune[knob] = value;
   return LSA_OK;
 }
@@ -501,18 +528,9 @@ static int index_checked(lsa_ctx* c, const lsa_params* p, const void* q_idx, con
                          int32_t* sparse_idx, int32_t* n_sparse, int32_t* pages_out, int32_t* rows_out,
                          int32_t* n_rows_out) {
   if (c == nullptr) return LSA_ERR_ARG;
-  int r = check_params(p, true, false);
+  const int r = lsa::check_index_call(p, q_idx, w, k_idx, k_scale, kmean, q_pos0, n_query, n_key, page_table,
+                                      page_table_stride, ctx_len, batch, sparse_idx, n_sparse);
   if (r != LSA_OK) return r;
-  if (q_idx == nullptr || w == nullptr || k_idx == nullptr || sparse_idx == nullptr || n_sparse == nullptr) return LSA_ERR_ARG;
-  if (p->hi_enable && kmean == nullptr) return LSA_ERR_ARG;
-  if (p->key_dtype == LSA_KEY_E4M3 && k_scale == nullptr) return LSA_ERR_ARG;
-  if (n_query < 0 || n_key < 0 || q_pos0 < 0) return LSA_ERR_ARG;
-  if (p->paged) {
-    if (page_table == nullptr || ctx_len == nullptr || batch <= 0 || page_table_stride <= 0) return LSA_ERR_ARG;
-  } else if (q_pos0 + n_query > n_key) {
-    return LSA_ERR_ARG;
-  }
-  if (!aligned16(q_idx) || !aligned16(w) || !aligned16(k_idx) || (kmean && !aligned16(kmean))) return LSA_ERR_SHAPE;
   return run_index(c, p, q_idx, w, k_idx, k_scale, kmean, q_pos0, n_query, n_key, page_table, page_table_stride,
                    ctx_len, batch, sparse_idx, n_sparse, pages_out, rows_out, n_rows_out);
 }

@@ -4,9 +4,12 @@
 // One thread block = one query (or one row split of one sequence in decode).  Its 64 heads are the M = 64
 // rows of every MMA; the attended cache rows stream through a ring of three 64-key shared tiles:
 //
-//   warps 8-11  gather: rows [window | sink | sparse] (or the caller's row list) -> 128B-swizzled K-major tiles with
-//               coalesced 16-byte cp.async, up to three tiles in flight, each handed over through an mbarrier when it
-//               has landed; tiles of 64 consecutive window rows come as nine TMA boxes instead.
+//   warps 8-11  gather: rows [window | sink | sparse] (or the caller's row list) -> 128B-swizzled K-major tiles, up to
+//               three tiles in flight.  Scattered rows come by TMA gather (cp.async.bulk.tensor ... tile::gather4: four
+//               cache rows x one 64-dim column block per instruction, 144 instructions per tile spread over the 128
+//               gather threads, completion counted in bytes on the tile's mbarrier), tiles of 64 consecutive window
+//               rows as nine plain TMA boxes; caches TMA cannot address (unaligned base or pitch) fall back to
+//               coalesced 16-byte cp.async.
 //               Q arrives the same way: its rope dims (512-575) stay in shared memory as an MMA operand, dims 0-511
 //               are staged in the last tile buffer for the softmax warps
 //   warps 4-7   one thread each issues tcgen05.mma.  Back-to-back MMAs into one accumulator run far below the pipe's
@@ -41,17 +44,59 @@
 //                     lanes 16-31.  Lanes l and l+16 of a softmax warp share head row l: they swap halves, so lane l
 //                     finishes keys 0-31 and lane l+16 keys 32-63 of the tile.  P (32 columns = 64 bf16, one copy
 //                     per lane half) overwrites the first half of the S buffer it came from.
-#include <cstdio>
-#include <cstdlib>
-
 #include "lsa_internal.h"
 #include "lsa_tc.cuh"
 
 #ifdef LSA_TIMELINE
-// Debug build only (-DLSA_TIMELINE): per-block SM-clock stamps at the phase boundaries of the attention kernel,
-// read back with lsa_debug_timeline.  0 entry, 1 set-up done, 2 Q ready, 3 first key tile landed, 4 first S ready,
-// 5 last P handed over, 6 last P V done, 7 exit.
-__device__ long long g_timeline[1024 * 16];
+// Instrumented build only (-DLSA_TIMELINE; the default library has none of this): SM-clock stamps of the attention
+// kernel, one slot per event and block, each written by one thread; read back with lsa_debug_timeline.
+enum TlEvent {
+  kTlEntry = 0,     // block entry
+  kTlSetup,         // barriers initialised, tensor memory allocated
+  kTlDepWait,       // griddepcontrol.wait returned (thread 0)
+  kTlQInTmem,       // MMA issuer 0: Q is in tensor memory
+  kTlTile0Landed,   // MMA issuer 0: first key tile landed
+  kTlS0,            // first S tile complete (softmax thread 0)
+  kTlLastP,         // last P handed to the issuers
+  kTlLastPV,        // last P V complete
+  kTlStaged,        // thread 0: its part of O staged in shared memory
+  kTlSynced,        // block barrier after the tile loop passed
+  kTlSent,          // rows for the peer blocks written (split launches)
+  kTlClusterSync,   // cluster barrier passed
+  kTlMerged,        // merge done
+  kTlExit,          // last instruction of thread 0
+  kTlTile0Issued,   // gather thread 0: copies of the first tile issued
+  kTlQIssued,       // gather thread 0: Q requested
+  // steady state: tiles kTlProbe .. kTlProbe + 3 of the block, slot = event + tile - kTlProbe
+  kTlKFreed = 16,   // gather thread 0: the tile's buffer is free (k_empty passed)
+  kTlKIssued = 20,  // gather thread 0: the tile's copies are issued
+  kTlKLanded = 24,  // (unused)
+  kTlQkIssue0 = 28, // issuer 0: about to issue the tile's Q K^T
+  kTlQkIssue1 = 32, // issuer 0: Q K^T issued
+  kTlSFull = 36,    // softmax thread 0: the tile's S complete
+  kTlSLoaded = 40,  // ... partial sums read and exchanged
+  kTlPHanded = 44,  // ... P handed over
+  kTlPvIssue0 = 48, // issuer 0: about to issue the tile's P V
+  kTlPvIssue1 = 52, // issuer 0: P V issued
+  kTlPvDone = 56,   // (unused)
+  kTlQkMmas = 60,   // issuer 0: the tile's Q K^T MMAs issued, commit not yet
+  kTlPvMmas = 64,   // issuer 0: the tile's P V MMAs issued, commits not yet
+  kTlPHanded1 = 68, kTlPHanded2 = 72, kTlPHanded3 = 76,   // softmax warps 1-3: P handed over
+  kTlSpinsQk = 80, kTlSpinsPv = 84,   // issuer 0: failed polls before the tile's Q K^T / P V (a count, not a time)
+  kTlCount = 88
+};
+#ifndef LSA_TL_PROBE
+#define LSA_TL_PROBE 10
+#endif
+constexpr int kTlProbe = LSA_TL_PROBE;
+#define LSA_TL_VAL(cond, i, k, v)                                                       \
+  do {                                                                                   \
+    const unsigned blk_ = blockIdx.x + gridDim.x * blockIdx.y;                           \
+    if ((cond) && (i) >= kTlProbe && (i) < kTlProbe + 4 && blk_ < 1024)                  \
+      g_timeline[blk_ * kTlCount + (k) + (i) - kTlProbe] = g_timeline[blk_ * kTlCount] + (v); \
+  } while (0)
+#define LSA_TL_TILE(cond, i, k) do { if ((cond) && (i) >= kTlProbe && (i) < kTlProbe + 4) LSA_TL((k) + (i) - kTlProbe); } while (0)
+__device__ long long g_timeline[1024 * kTlCount];
 __device__ long long g_wall[1024 * 2];   // globaltimer (ns) at entry and exit
 #define LSA_WALL(k)                                                                      \
   do {                                                                                   \
@@ -66,13 +111,17 @@ extern "C" __attribute__((visibility("default"))) int lsa_debug_wall(long long* 
 #define LSA_TL(k)                                                                        \
   do {                                                                                   \
     const unsigned blk_ = blockIdx.x + gridDim.x * blockIdx.y;                           \
-    if (blk_ < 1024) g_timeline[blk_ * 16 + (k)] = clock64();                             \
+    if (blk_ < 1024) g_timeline[blk_ * kTlCount + (k)] = clock64();                       \
   } while (0)
+#define LSA_TL_IF(cond, k) do { if (cond) LSA_TL(k); } while (0)
 extern "C" __attribute__((visibility("default"))) int lsa_debug_timeline(long long* host, int n_blocks) {
-  return cudaMemcpyFromSymbol(host, g_timeline, sizeof(long long) * 16 * (n_blocks < 1024 ? n_blocks : 1024)) == cudaSuccess ? 0 : -1;
+  return cudaMemcpyFromSymbol(host, g_timeline, sizeof(long long) * kTlCount * (n_blocks < 1024 ? n_blocks : 1024)) == cudaSuccess ? 0 : -1;
 }
 #else
 #define LSA_TL(k)
+#define LSA_TL_IF(cond, k)
+#define LSA_TL_TILE(cond, i, k)
+#define LSA_TL_VAL(cond, i, k, v)
 #define LSA_WALL(k)
 #endif
 
@@ -100,7 +149,7 @@ constexpr float kRescaleGap = 8.f;           // rescale O only when the row max 
 struct AttnTcSmem {
   alignas(1024) uint8_t q_rope[kAtomBytes];                 // Q[:, 512:576], 64 rows x 128 B
   alignas(1024) uint8_t k[kKBufs][kAtoms][kAtomBytes];      // [tile buffer][column block][64 rows x 128 B]
-  alignas(8) uint64_t q_full, q_tmem, k_full[kKBufs], k_empty[kKBufs], s_full[2], p_ready[2], pv_done[2];
+  alignas(8) uint64_t q_full, q_tmem, k_full[kKBufs], k_empty[kKBufs], s_full[2], p_ready[2];
   uint32_t tmem_slot;
   float lse_own[kH];              // split launches: this block's log-sum-exp per head (log2 units)
 };
@@ -119,9 +168,18 @@ __device__ __forceinline__ void cluster_sync_all() {
 //
 // q_tma != 0: q_map describes q as a bf16 matrix [n_query * 64, 576] and Q arrives as nine TMA boxes; otherwise the
 // gather warps copy it with cp.async.  k_tma != 0 (contiguous caches only): k_map describes the cache rows, and key
-// tiles that lie wholly inside the window, 64 consecutive rows, arrive as nine TMA boxes as well.
+// tiles that lie wholly inside the window, 64 consecutive rows, arrive as nine TMA boxes as well.  k_g4 != 0: g_map
+// describes the cache rows with a box one row high, and every other key tile is gathered four rows per instruction.
+//
+// One instantiation per way the kernel is used, so that each holds only the code of its mode (the instruction caches
+// hold far less than the whole kernel, and the three warp roles run their loops side by side):
+//   kRows       the caller's row lists are walked (else [window | sink | sparse] of a contiguous cache)
+//   kPv         threads that issue P V: 2 = an issuer owns a lane half, 4 = one issuer per 128 value dims
+//   kClustered  the blocks of a cluster are row splits of one sequence and merge their results
+template <bool kRows, int kPv, bool kClustered>
 __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map, int q_tma,
                                                                             const __grid_constant__ CUtensorMap k_map, int k_tma,
+                                                                            const __grid_constant__ CUtensorMap g_map, int k_g4,
                                                                             AttnArgs p) {
   extern __shared__ uint8_t smem_raw[];
   AttnTcSmem& sm = *reinterpret_cast<AttnTcSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -134,14 +192,14 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
   float* const part_out = p.part_out;
   float* const part_lse = p.part_lse;
 
-  const int n_pv = p.pv_issuers == 4 ? 4 : 2;   // threads that issue P V (see the header: 2 = lane-half ownership)
-  const bool clustered = p.n_split > 1;
+  constexpr int n_pv = kPv;
+  constexpr bool clustered = kClustered;
   const bool dead = tc::status_raised(p.status);   // an earlier block of this launch (or an earlier launch) gave up on a wait
   if (dead && !clustered) return;
 
   // ---- set-up
   if (tid == 0) {
-    LSA_TL(0);
+    LSA_TL(kTlEntry);
     LSA_WALL(0);
     tc::mbar_init(smem_u32(&sm.q_full), q_tma ? 1 : 32 * kLoadWarps);
     tc::mbar_init(smem_u32(&sm.q_tmem), kSoftmaxWarps);
@@ -151,7 +209,6 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
     }
     for (int b = 0; b < 2; ++b) {
       tc::mbar_init(smem_u32(&sm.s_full[b]), 2);
-      tc::mbar_init(smem_u32(&sm.pv_done[b]), n_pv);
       tc::mbar_init(smem_u32(&sm.p_ready[b]), kSoftmaxWarps);
     }
     tc::fence_mbar_init();
@@ -164,18 +221,34 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
   __syncthreads();
   tc::fence_after_sync();
   const uint32_t tmem_base = sm.tmem_slot;
-  if (tid == 0) LSA_TL(1);
+  if (tid == 0) LSA_TL(kTlSetup);
   // Programmatic dependent launch: this block may have been placed while the previous kernel of the stream was still
-  // draining; what earlier kernels wrote is read only from here on.  The next kernel's blocks may be placed from now.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (tid == 0) LSA_TL(13);
-  // Q is requested before anything else is looked up: a block cannot start without it, and in prefill it comes from HBM.
-  if (q_tma && tid == 32 * (kSoftmaxWarps + kMmaWarps)) {
-    const uint32_t stage = smem_u32(sm.k[kKBufs - 1]);
-    tc::mbar_expect_tx(smem_u32(&sm.q_full), kH * kDQK * 2);
-    for (int a = 0; a < kAtoms; ++a)
-      tc::tma_load_2d(a < 8 ? stage + a * kAtomBytes : smem_u32(sm.q_rope), &q_map, a * 64, qi * kH, smem_u32(&sm.q_full));
+  // draining; what that kernel wrote is read, and what it may still read is overwritten, only after
+  // griddepcontrol.wait.  The next kernel's blocks may be placed from then on.
+  // rows_stable: the row lists (and the caches, as always) were complete before the previous kernel started, so the
+  // gather warps read them and put the first two key tiles in flight while that kernel drains, and wait only before
+  // they request Q; every other thread waits here.
+  const bool early_rows = kRows && p.rows_stable != 0 && q_tma != 0;   // block-uniform
+  const bool gather_warp = warp >= kSoftmaxWarps + kMmaWarps;
+  auto dependency_wait = [&]() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  };
+  // Q is requested before anything else that depends on the previous kernel: a block cannot start without it, and in
+  // prefill it comes from HBM.
+  auto request_q = [&]() {
+    if (q_tma && tid == 32 * (kSoftmaxWarps + kMmaWarps)) {
+      const uint32_t stage = smem_u32(sm.k[kKBufs - 1]);
+      tc::mbar_expect_tx(smem_u32(&sm.q_full), kH * kDQK * 2);
+      for (int a = 0; a < kAtoms; ++a)
+        tc::tma_load_2d(a < 8 ? stage + a * kAtomBytes : smem_u32(sm.q_rope), &q_map, a * 64, qi * kH, smem_u32(&sm.q_full));
+      LSA_TL(kTlQIssued);
+    }
+  };
+  if (!(early_rows && gather_warp)) {
+    dependency_wait();
+    if (tid == 0) LSA_TL(kTlDepWait);
+    request_q();
   }
 
   // ---- this query's row list (same conventions as the mma.sync kernel)
@@ -183,7 +256,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
   int n_sink = 0, n_sp = 0, n_win = 0, n_tot;
   int64_t win0 = 0;
   const int32_t* rows = nullptr;
-  if (p.rows != nullptr) {
+  if constexpr (kRows) {
     rows = p.rows + static_cast<int64_t>(qi) * p.rows_ld;
     n_tot = p.n_rows[qi];
   } else {
@@ -198,10 +271,13 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
   // window is a run of consecutive cache rows, so its whole tiles need no per-row addressing.
   auto row_of = [&](int i) -> int32_t {
     if (i >= n_tot) return -1;
-    if (rows) return rows[i];
-    if (i < n_win) return static_cast<int32_t>(win0 + i);
-    if (i < n_win + n_sink) return i - n_win;
-    return sp[i - n_win - n_sink];
+    if constexpr (kRows) {
+      return rows[i];
+    } else {
+      if (i < n_win) return static_cast<int32_t>(win0 + i);
+      if (i < n_win + n_sink) return i - n_win;
+      return sp[i - n_win - n_sink];
+    }
   };
   const int tiles_all = (n_tot + kTileKeys - 1) / kTileKeys;
   const int tiles_per = (tiles_all + p.n_split - 1) / p.n_split;
@@ -211,7 +287,8 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
 
   if (warp >= kSoftmaxWarps + kMmaWarps) {
     // ================= gather warps =================
-    const int lt = tid - 32 * (kSoftmaxWarps + kMmaWarps);   // 0..127
+    const int gw = warp - (kSoftmaxWarps + kMmaWarps);
+    const int lt = gw * 32 + lane;   // 0..127
     {
       // Q of this query: the rope part (dims 512-575) stays in shared memory as an MMA operand; dims 0-511 are staged
       // in the last key buffer for the softmax warps, which move them to tensor memory.  As TMA boxes they complete
@@ -233,17 +310,38 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
     }
     // Every gather warp works on every tile: warp w copies rows 16w .. 16w+15, so a freed buffer is refilled by all
     // four warps at once.  Lanes 0-15 look up the cache row of their key once; the row number is then broadcast
-    // and the 72 16-byte chunks of that row are copied by consecutive lanes (coalesced 512-byte requests).
-    const int lw = lt >> 5;
+    // and the 72 16-byte chunks of that row are copied by consecutive lanes (coalesced 512-byte requests: a row is
+    // fetched whole, by one warp, in back-to-back instructions.  Spreading the chunks of a tile evenly over the warps,
+    // every instruction full, was measured at 1.3 x the time, in prefill and in decode).
     constexpr int kRowsPerWarp = kTileKeys / kLoadWarps;
     const uint8_t* kg = reinterpret_cast<const uint8_t*>(k_ptr);
     auto tile_by_tma = [&](int i) -> bool {   // block-uniform
-      return k_tma && rows == nullptr && (tile_begin + i + 1) * kTileKeys <= n_win;
+      return !kRows && k_tma && (tile_begin + i + 1) * kTileKeys <= n_win;
     };
+    // TMA gather (k_g4): thread lt < 128 fetches row quad lt / 8 (tile rows 4 * quad .. + 3) of column block lt % 8, and
+    // the threads with lt % 8 == 0 also the rope block: 144 instructions per tile.
+    const bool g4 = k_g4 != 0;   // block-uniform
+    const int quad = (lt >> 3) & 15, atom0 = lt & 7;
     auto my_key_row = [&](int i) -> int32_t {
-      return (i < n_tiles && lane < kRowsPerWarp && !tile_by_tma(i)) ? row_of((tile_begin + i) * kTileKeys + kRowsPerWarp * lw + lane) : -1;
+      return (!g4 && i < n_tiles && lane < kRowsPerWarp && !tile_by_tma(i)) ? row_of((tile_begin + i) * kTileKeys + kRowsPerWarp * gw + lane) : -1;
+    };
+    auto my_quad_rows = [&](int i) -> int4 {
+      int4 r = make_int4(0, 0, 0, 0);
+      if (g4 && i < n_tiles && !tile_by_tma(i)) {
+        const int i0 = (tile_begin + i) * kTileKeys + 4 * quad;
+        if (kRows && i0 + 3 < n_tot && ((reinterpret_cast<uintptr_t>(rows + i0) & 15u) == 0)) {
+          r = *reinterpret_cast<const int4*>(rows + i0);
+        } else {
+          r.x = row_of(i0); r.y = row_of(i0 + 1); r.z = row_of(i0 + 2); r.w = row_of(i0 + 3);
+        }
+        // rows past the end of the list are masked in the softmax: any readable row will do
+        r.x = max(r.x, 0); r.y = max(r.y, 0); r.z = max(r.z, 0); r.w = max(r.w, 0);
+      }
+      return r;
     };
     int32_t my_row = my_key_row(0);
+    int4 my_rows4 = my_quad_rows(0);
+    bool waited = !early_rows;   // this thread has executed the dependency wait
     // Copies of up to three tiles are in flight: a tile is handed to the MMA issuers (k_full) when its cp.async group
     // has landed, which is looked at after the next tile's copies are issued, or at once when no buffer is free.
     int first_pend = 0, n_pend = 0;   // tiles first_pend .. first_pend + n_pend - 1 are issued but not handed over
@@ -252,7 +350,6 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       tc::fence_proxy_async();
       tc::mbar_arrive(smem_u32(&sm.q_full));
       q_handed = true;
-      if (lt == 0) LSA_TL(15);
     };
     auto hand_over_oldest = [&]() {
       if (n_pend >= 3) cp_async_wait<2>();
@@ -268,30 +365,45 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       const int b = i % kKBufs;
       const uint32_t par = ((i / kKBufs) & 1) ^ 1;
       const int32_t next_row = my_key_row(i + 1);   // fetched before the wait: off the critical path
+      const int4 next_rows4 = my_quad_rows(i + 1);
       // Q and the first tile go out alone: requested together with the next tiles they would share the memory pipe
       // with them and the first Q K^T would start two tiles' worth of traffic later
       if (i == 1) while (n_pend > 0) hand_over_oldest();
       if (i == kKBufs - 1) {
+        if (!waited) {   // two tiles are in flight: now the previous kernel must be done, then Q goes out
+          dependency_wait();
+          request_q();
+          waited = true;
+        }
         // first use of the buffer that staged Q: the softmax warps must have moved Q to tensor memory
         while (n_pend > 0 && !__all_sync(0xffffffffu, tc::mbar_test(smem_u32(&sm.q_tmem), 0))) hand_over_oldest();
         if (!__all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.q_tmem), 0, p.status))) break;
       }
       while (n_pend > 0 && !__all_sync(0xffffffffu, tc::mbar_test(smem_u32(&sm.k_empty[b]), par))) hand_over_oldest();
       if (!__all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.k_empty[b]), par, p.status))) break;
+      LSA_TL_TILE(lt == 0, i, kTlKFreed);
       if (tile_by_tma(i)) {
         // 64 consecutive window rows: nine boxes that complete k_full by byte count; the (empty) cp.async group
-        // below keeps the hand-over bookkeeping the same for both kinds of tile
+        // below keeps the hand-over bookkeeping the same for every kind of tile
         if (lt == 0) {
           tc::mbar_expect_tx_only(smem_u32(&sm.k_full[b]), kAtoms * kAtomBytes);
           const int row0 = static_cast<int>(win0) + (tile_begin + i) * kTileKeys;
           for (int a = 0; a < kAtoms; ++a)
             tc::tma_load_2d(smem_u32(sm.k[b][a]), &k_map, a * 64, row0, smem_u32(&sm.k_full[b]));
         }
+      } else if (g4) {
+        // scattered rows: four rows x 64 dims per instruction, straight into their place in the swizzled tile
+        if (lt == 0) tc::mbar_expect_tx_only(smem_u32(&sm.k_full[b]), kAtoms * kAtomBytes);
+        tc::tma_gather4_2d(smem_u32(sm.k[b][atom0]) + quad * 512, &g_map, atom0 * 64, my_rows4.x, my_rows4.y, my_rows4.z,
+                           my_rows4.w, smem_u32(&sm.k_full[b]));
+        if (atom0 == 0)
+          tc::tma_gather4_2d(smem_u32(sm.k[b][kAtoms - 1]) + quad * 512, &g_map, (kAtoms - 1) * 64, my_rows4.x, my_rows4.y,
+                             my_rows4.z, my_rows4.w, smem_u32(&sm.k_full[b]));
       } else {
 #pragma unroll 4
         for (int rr = 0; rr < kRowsPerWarp; ++rr) {
           const int32_t row = __shfl_sync(0xffffffffu, my_row, rr);
-          const int r = kRowsPerWarp * lw + rr;
+          const int r = kRowsPerWarp * gw + rr;
           const uint8_t* src = kg + static_cast<int64_t>(row >= 0 ? row : 0) * p.ld_k * 2;
           const int nb = row >= 0 ? 16 : 0;
 #pragma unroll
@@ -300,28 +412,30 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
         }
       }
       cp_async_commit();
-      if (lt == 0 && i == 0) LSA_TL(14);
+      LSA_TL_IF(lt == 0 && i == 0, kTlTile0Issued);
+      LSA_TL_TILE(lt == 0, i, kTlKIssued);
       ++n_pend;
       if (n_pend == kKBufs) hand_over_oldest();
       my_row = next_row;
+      my_rows4 = next_rows4;
     }
     while (n_pend > 0) hand_over_oldest();
     if (!q_handed) {
       cp_async_wait<0>();
       hand_over_q();
     }
+    if (!waited) {   // fewer than three tiles: Q has not been requested yet
+      dependency_wait();
+      request_q();
+    }
   } else if (warp >= kSoftmaxWarps) {
     // ================= MMA issuers =================
     const int x = warp - kSoftmaxWarps;   // 0..3
     if (lane == 0 && n_tiles > 0) {
-#ifdef LSA_DBG_QKN
-      constexpr uint32_t idesc_qk = tc::idesc_bf16(kH, LSA_DBG_QKN, 0, 0);   // timing experiment only: wrong results
-#else
       constexpr uint32_t idesc_qk = tc::idesc_bf16(kH, kTileKeys, 0, 0);
-#endif
-      const uint32_t idesc_pv = n_pv == 4 ? tc::idesc_bf16(kH, 128, 0, 1) : tc::idesc_bf16(kH, 256, 0, 1);   // B = V read MN-major
+      constexpr uint32_t idesc_pv = n_pv == 4 ? tc::idesc_bf16(kH, 128, 0, 1) : tc::idesc_bf16(kH, 256, 0, 1);   // B = V read MN-major
       bool ok = tc::mbar_wait(smem_u32(&sm.q_full), 0, p.status) && tc::mbar_wait(smem_u32(&sm.q_tmem), 0, p.status);
-      if (x == 0) LSA_TL(2);
+      LSA_TL_IF(x == 0, kTlQInTmem);
       // Descriptors are built once; inside the loops only the start-address word moves (one add per operand).
       constexpr uint32_t kBufBytes = kAtoms * kAtomBytes;
       const uint64_t dqr = tc::smem_desc_sw128(smem_u32(sm.q_rope), 16, 1024);
@@ -346,7 +460,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
 #pragma unroll
         for (int s = 0; s < 2; ++s)    // rope dims 512 + 32x + 16s .. +15
           tc::umma_ss(d, tc::desc_advance(dqr, (2 * x + s) * 32), tc::desc_advance(dkb, 8 * kAtomBytes + (2 * x + s) * 32), idesc_qk, 1);
-        if (x == 0 && i == 22) LSA_TL(9);
+        LSA_TL_TILE(x == 0, i, kTlQkMmas);
         tc::umma_commit(smem_u32(&sm.s_full[i & 1]));
       };
       auto issue_pv = [&](int j) {   // O[:, 128x : 128x+128] += P_j V_j
@@ -355,39 +469,62 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
 #pragma unroll
         for (int kk = 0; kk < kTileKeys / 16; ++kk)   // keys 16*kk .. +15
           tc::umma_ts(o_dst, p_src + (j & 1) * kSBuf + kk * 8, tc::desc_advance(dvb, kk * 2048), idesc_pv, (j > 0) || (kk > 0));
+        LSA_TL_TILE(x == 0, j, kTlPvMmas);
+        // one completion signal per tile: "P V of tile j done" frees the key buffer for the gather warps and tells the
+        // softmax warps (and, with four issuers, the Q K^T issuers) that O and the P columns may be touched again.
+        // Several parties watch the same phase: it cannot flip twice before they have looked, because the P V of tile
+        // j + 3 needs work of theirs that comes after the look.
         tc::umma_commit(smem_u32(&sm.k_empty[j % kKBufs]));
-        tc::umma_commit(smem_u32(&sm.pv_done[j & 1]));
       };
       const bool does_qk = x < 2;
       const bool wait_pv = p.qk_waits_pv != 0 || n_pv != 2;
       // Two in-order queues, "next Q K^T" (at most one tile ahead of the softmax it feeds) and "next P V".
+      // Whatever follows a batch of MMAs in this thread - a clock read, a barrier probe - waits until the batch has
+      // left the issue stage, which costs a hundred cycles and more each time: the clock is read only while spinning
+      // and a P V ends with one commit.  Whichever of the two is ready goes first; when both are, Q K^T (the softmax it
+      // feeds is the longer chain).  Issuing the ready P V right behind a Q K^T without looking at the barriers in
+      // between was measured: faster while whole window tiles stream in, slower on gathered tiles, where the later
+      // completion of that P V holds up the refill of its key buffer; dropped.
+      auto pv_done = [&](int j) -> bool {   // j >= 0
+        return tc::mbar_test(smem_u32(&sm.k_empty[j % kKBufs]), (j / kKBufs) & 1);
+      };
       int qk_next = does_qk ? 0 : n_tiles, pv_next = x < n_pv ? 0 : n_tiles;
-      long long t_idle = clock64();
+      long long t_idle = 0;
       uint32_t spins = 0;
       while (ok && pv_next < n_tiles) {
         bool did = false;
-        if (qk_next < n_tiles && qk_next <= pv_next + 1) {
+        // P V first: its completion frees a key buffer, and the refill of that buffer is the longest latency of the ring
+        if ((!does_qk || pv_next < qk_next) && tc::mbar_test(smem_u32(&sm.p_ready[pv_next & 1]), (pv_next >> 1) & 1)) {
+          LSA_TL_TILE(x == 0, pv_next, kTlPvIssue0);
+          issue_pv(pv_next++);
+          LSA_TL_TILE(x == 0, pv_next - 1, kTlPvIssue1);
+          did = true;
+        }
+        if (!did && qk_next < n_tiles && qk_next <= pv_next + 1) {
           // S buffer qk_next&1 also holds P of tile qk_next-2: it is free once that tile's P V has completed
           if (tc::mbar_test(smem_u32(&sm.k_full[qk_next % kKBufs]), (qk_next / kKBufs) & 1) &&
-              (!wait_pv || tc::mbar_test(smem_u32(&sm.pv_done[qk_next & 1]), ((qk_next >> 1) & 1) ^ 1))) {
-            if (x == 0 && qk_next == 0) LSA_TL(3);
+              (!wait_pv || qk_next < 2 || pv_done(qk_next - 2))) {
+            LSA_TL_IF(x == 0 && qk_next == 0, kTlTile0Landed);
+            LSA_TL_TILE(x == 0, qk_next, kTlQkIssue0);
             issue_qk(qk_next++);
+            LSA_TL_TILE(x == 0, qk_next - 1, kTlQkIssue1);
             did = true;
           }
         }
-        if (!did && (!does_qk || pv_next < qk_next) && tc::mbar_test(smem_u32(&sm.p_ready[pv_next & 1]), (pv_next >> 1) & 1)) {
-          issue_pv(pv_next++);
-          did = true;
-        }
         if (did) {
           spins = 0;
-          t_idle = clock64();
         } else if ((++spins & 255u) == 0) {
+          // bounded: nothing became ready for about a second (the clock is read only while spinning)
           if (tc::status_raised(p.status)) {
             ok = false;
-          } else if (clock64() - t_idle > tc::kWaitCycles) {
-            report_status(p.status, kDevTimeout);   // bounded: nothing became ready for about a second
-            ok = false;
+          } else {
+            const long long now = clock64();
+            if (spins == 256u) {
+              t_idle = now;
+            } else if (now - t_idle > tc::kWaitCycles) {
+              report_status(p.status, kDevTimeout);
+              ok = false;
+            }
           }
         }
       }
@@ -425,8 +562,8 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       const int b = i & 1;
       ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.s_full[b]), (i >> 1) & 1, p.status));
       if (!ok) break;
-      if (tid == 0 && i == 0) LSA_TL(4);
-      if (tid == 0 && i == 20) LSA_TL(10);
+      LSA_TL_IF(tid == 0 && i == 0, kTlS0);
+      LSA_TL_TILE(tid == 0, i, kTlSFull);
       tc::fence_after_sync();
       const uint32_t s_addr = tmem_base + lane_addr + kColS + b * kSBuf;
       uint32_t v[32];
@@ -443,7 +580,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
           v[j] = __float_as_uint(keep + __shfl_xor_sync(0xffffffffu, give, 16));
         }
       }
-      if (tid == 0 && i == 20) LSA_TL(11);
+      LSA_TL_TILE(tid == 0, i, kTlSLoaded);
       // logits in log2 units, ragged tail masked
       const int n_valid = n_tot - (tile_begin + i) * kTileKeys - kHalfKeys * hi;   // keys of this lane's half that exist
       float mx = -INFINITY;
@@ -464,7 +601,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       }
       if (__any_sync(0xffffffffu, alpha != 1.f)) {
         // O may be touched only between P V of tile i-1 (done) and P V of tile i (not yet released)
-        ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done[(i - 1) & 1]), ((i - 1) >> 1) & 1, p.status));
+        ok = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.k_empty[(i - 1) % kKBufs]), ((i - 1) / kKBufs) & 1, p.status));
         if (!ok) break;
         tc::fence_after_sync();
 #pragma unroll 1
@@ -491,7 +628,6 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
         pk[j] = pack_bf16(p0, p1);
       }
       l_run += sum;
-      if (tid == 0 && i == 20) LSA_TL(12);
       {
         // The A operand of P V sits in tensor memory, in the lanes of the accumulator it feeds: both lanes of a
         // row need all 64 keys, so the two halves are swapped in, then written as 32 columns of packed bf16.
@@ -508,16 +644,19 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       }
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(smem_u32(&sm.p_ready[b]));
-      if (tid == 0 && i == 20) LSA_TL(13);
+      LSA_TL_TILE(tid == 0, i, kTlPHanded);
+      LSA_TL_TILE(tid == 32, i, kTlPHanded1);
+      LSA_TL_TILE(tid == 64, i, kTlPHanded2);
+      LSA_TL_TILE(tid == 96, i, kTlPHanded3);
     }
-    if (tid == 0) LSA_TL(5);
+    if (tid == 0) LSA_TL(kTlLastP);
     // ---- epilogue: O / l
     const float l_row = l_run + __shfl_xor_sync(0xffffffffu, l_run, 16);
     const float m_row = m_used;
     bool have_o = ok && n_tiles > 0;
-    if (have_o) have_o = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.pv_done[(n_tiles - 1) & 1]), ((n_tiles - 1) >> 1) & 1, p.status));
+    if (have_o) have_o = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.k_empty[(n_tiles - 1) % kKBufs]), ((n_tiles - 1) / kKBufs) & 1, p.status));
     tc::fence_after_sync();
-    if (tid == 0) LSA_TL(6);
+    if (tid == 0) LSA_TL(kTlLastPV);
     const float inv = (have_o && l_row > 0.f) ? 1.f / l_row : 0.f;
     const float lse2 = (have_o && l_row > 0.f) ? m_row + log2f(l_row) : -INFINITY;   // log2 domain
     uint8_t* stage = &sm.k[0][0][0];
@@ -596,10 +735,10 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       }
     }
   }
-  if (tid == 0) LSA_TL(8);
+  if (tid == 0) LSA_TL(kTlStaged);
   tc::fence_before_sync();
   __syncthreads();
-  if (tid == 0) LSA_TL(9);
+  if (tid == 0) LSA_TL(kTlSynced);
   if (warp == kSoftmaxWarps) tc::tmem_dealloc(tmem_base, kTmemColsAttn);
   if (clustered) {
     // ---- merge of the splits (Sec. 4.1.1: online-softmax rescaling) for this block's heads: weights
@@ -613,9 +752,9 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
       __threadfence();
     }
-    if (tid == 0) LSA_TL(10);
+    if (tid == 0) LSA_TL(kTlSent);
     cluster_sync_all();   // every block of the cluster has written its rows
-    if (tid == 0) LSA_TL(11);
+    if (tid == 0) LSA_TL(kTlClusterSync);
     // Warp w finishes rows w, w + 12, ... of this block's share (at most three).  Lane 8k + j first fetches the
     // log-sum-exp of split j for the warp's k-th row, so that all of them are in flight together.
     constexpr int kWarps = kThreadsAttnTc / 32;
@@ -684,10 +823,10 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
         }
       }
     }
-    if (tid == 0) LSA_TL(12);
+    if (tid == 0) LSA_TL(kTlMerged);
   }
   if (tid == 0) {
-    LSA_TL(7);
+    LSA_TL(kTlExit);
     LSA_WALL(1);
   }
 }
@@ -697,22 +836,31 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
 // Largest cluster of full-SM blocks of this kernel the device can place (queried once per process).
 static_assert(sizeof(AttnTcSmem) + 1024 <= 227 * 1024, "shared memory of the attention kernel exceeds one SM");
 
+using AttnTcKernel = void (*)(CUtensorMap, int, CUtensorMap, int, CUtensorMap, int, AttnArgs);
+
+// The instantiation that serves a call (see the kernel's template parameters).
+static AttnTcKernel pick_kernel(const AttnArgs& a) {
+  const bool rows = a.rows != nullptr;
+  if (!rows) return a.pv_issuers == 4 ? sparse_attn_tc_kernel<false, 4, false> : sparse_attn_tc_kernel<false, 2, false>;
+  if (a.n_split > 1) return a.pv_issuers == 4 ? sparse_attn_tc_kernel<true, 4, true> : sparse_attn_tc_kernel<true, 2, true>;
+  return a.pv_issuers == 4 ? sparse_attn_tc_kernel<true, 4, false> : sparse_attn_tc_kernel<true, 2, false>;
+}
+
 static int max_cluster_blocks() {
   static const int n = [] {
     const size_t smem = sizeof(AttnTcSmem) + 1024;
-    if (cudaFuncSetAttribute(sparse_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) return 1;
+    AttnTcKernel kernel = sparse_attn_tc_kernel<true, 4, true>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) return 1;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(1, kMaxClusterSplit);
     cfg.blockDim = dim3(kThreadsAttnTc);
     cfg.dynamicSmemBytes = smem;
     int size = 0;
-    const cudaError_t eq = cudaOccupancyMaxPotentialClusterSize(&size, sparse_attn_tc_kernel, &cfg);
+    const cudaError_t eq = cudaOccupancyMaxPotentialClusterSize(&size, kernel, &cfg);
     if (eq != cudaSuccess) {
-      if (getenv("LSA_DEBUG")) fprintf(stderr, "[lsa] cluster size query failed: %s\n", cudaGetErrorString(eq));
       (void)cudaGetLastError();
       return 1;
     }
-    if (getenv("LSA_DEBUG")) fprintf(stderr, "[lsa] attention kernel: max cluster size %d\n", size);
     return size < 1 ? 1 : size;
   }();
   return n;
@@ -732,16 +880,23 @@ bool attn_tc_supported(const AttnArgs& a) {
 cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t st, int64_t* n_launch) {
   if (a.n_query == 0) return cudaSuccess;
   const size_t smem = sizeof(AttnTcSmem) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(sparse_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (a.n_split > 1 && a.rows == nullptr) return cudaErrorInvalidValue;   // row splits walk row lists
+  AttnTcKernel kernel = pick_kernel(a);
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) return e;
-  CUtensorMap q_map{}, k_map{};
+  CUtensorMap q_map{}, k_map{}, g_map{};
   const int q_tma = (reinterpret_cast<uintptr_t>(a.q) & 15u) == 0 &&
                     make_map_bf16_rows(&q_map, a.q, kDQK, static_cast<uint64_t>(a.n_query) * kH, kH);
   // contiguous cache: the last query sees rows 0 .. q_pos0 + n_query - 1, so the cache holds at least that many
   const int k_tma = !a.paged && a.rows == nullptr && a.ld_k % 8 == 0 && (reinterpret_cast<uintptr_t>(a.k) & 15u) == 0 &&
                     make_map_bf16_rows(&k_map, a.k, static_cast<uint64_t>(a.ld_k), static_cast<uint64_t>(a.q_pos0 + a.n_query), kTileKeys);
+  // gather of scattered rows by TMA: any cache whose base and row pitch TMA can address; a paged pool's row count is
+  // not known here (every row number comes from the caller's list), so its map spans the whole coordinate range
+  const uint64_t g_rows = a.paged || a.rows != nullptr ? 0x7fffffffull : static_cast<uint64_t>(a.q_pos0 + a.n_query);
+  const int k_g4 = a.gather4 && a.ld_k % 8 == 0 && (reinterpret_cast<uintptr_t>(a.k) & 15u) == 0 &&
+                   make_map_bf16_rows(&g_map, a.k, static_cast<uint64_t>(a.ld_k), g_rows, 1);
   if (a.n_split <= 1) {
-    sparse_attn_tc_kernel<<<dim3(a.n_query, 1, 1), kThreadsAttnTc, smem, st>>>(q_map, q_tma, k_map, k_tma, a);
+    kernel<<<dim3(a.n_query, 1, 1), kThreadsAttnTc, smem, st>>>(q_map, q_tma, k_map, k_tma, g_map, k_g4, a);
   } else {
     if (!attn_tc_split_ok(a.n_split)) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg{};
@@ -758,11 +913,8 @@ cudaError_t launch_attn_tc(const AttnArgs& a, cudaStream_t st, int64_t* n_launch
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    e = cudaLaunchKernelEx(&cfg, sparse_attn_tc_kernel, q_map, q_tma, k_map, k_tma, a);
-    if (e != cudaSuccess) {
-      if (getenv("LSA_DEBUG")) fprintf(stderr, "[lsa] cluster launch (%d x %d blocks) failed: %s\n", a.n_query, a.n_split, cudaGetErrorString(e));
-      return e;
-    }
+    e = cudaLaunchKernelEx(&cfg, kernel, q_map, q_tma, k_map, k_tma, g_map, k_g4, a);
+    if (e != cudaSuccess) return e;
   }
   ++*n_launch;
   return cudaGetLastError();

@@ -4,7 +4,16 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "../../include/lsa.h"
+
 namespace lsa {
+
+// Argument checks of an indexer call (parameters, required pointers, ranges, 16-byte alignment of everything the
+// kernels read with vector loads); one copy for every entry point that launches the indexer.  Returns an LSA_* code.
+int check_index_call(const lsa_params* p, const void* q_idx, const float* w, const void* k_idx, const float* k_scale,
+                     const void* kmean, int64_t q_pos0, int64_t n_query, int64_t n_key, const int32_t* page_table,
+                     int64_t page_table_stride, const int32_t* ctx_len, int batch, const int32_t* sparse_idx,
+                     const int32_t* n_sparse);
 
 struct IndexArgs {
   int HI, DI, key_e4m3, P, B, M, Ksp, S, W, hi_enable, paged;
@@ -54,6 +63,9 @@ struct AttnArgs {
   float* lse;             // optional [n_query, H]
   int pv_issuers;         // tcgen05 kernel: 2 = an issuer owns a lane half (prefill), 4 = one P V issuer per 128 value dims
   int qk_waits_pv;        // tcgen05 kernel, 2 issuers: Q K^T of tile i+1 waits for the completion barrier of P V of tile i-1
+  int gather4;            // tcgen05 kernel: scattered rows by TMA gather (cp.async.bulk.tensor tile::gather4) where the cache allows
+  int rows_stable;        // tcgen05 kernel, row lists: `rows` / `n_rows` were complete before the previous kernel of the
+                          // stream started, so they may be read ahead of the programmatic dependency wait
   int n_split;            // >1: partial results in part_out / part_lse, merged afterwards
   float* part_out;        // fp32 [n_query, n_split, H, DV]
   float* part_lse;        // fp32 [n_query, n_split, H]
@@ -88,6 +100,10 @@ cudaError_t launch_coarse_minmax(const IndexArgs& a, cudaStream_t st, int64_t* n
 // tcgen05 version of the coarse stage (contiguous caches, H_I = 64, d_I = 128); groups = 4-query groups per block
 bool coarse_tc_supported(const IndexArgs& a);
 cudaError_t launch_coarse_tc(const IndexArgs& a, int groups, cudaStream_t st, int64_t* n_launch);
+// The coarse stage as every entry point runs it: the tcgen05 kernel where the shape allows, else the mma.sync tile.
+inline cudaError_t launch_coarse_best(const IndexArgs& a, int groups, cudaStream_t st, int64_t* n_launch) {
+  return coarse_tc_supported(a) ? launch_coarse_tc(a, groups, st, n_launch) : launch_coarse(a, st, n_launch);
+}
 // tcgen05 version of the coarse stage for paged caches (H_I = 64, d_I = 128); used by launch_coarse
 bool coarse_paged_tc_supported(const IndexArgs& a);
 cudaError_t launch_coarse_paged_tc(const IndexArgs& a, cudaStream_t st, int64_t* n_launch);

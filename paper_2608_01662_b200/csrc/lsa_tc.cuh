@@ -82,6 +82,18 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// Four rows of a 2-D tensor (row numbers r0..r3, any order, this GPU's memory), columns c0 .. c0 + box width - 1 of
+// each, land as four consecutive rows at `dst`.  The tensor map's box must be one row high.  c0 * element size must
+// be a multiple of 16 bytes; with a 128-byte swizzle `dst` must be 512-byte aligned for the rows to take their place
+// in the swizzled tile.  Completion is counted in bytes on `bar`.
+__device__ __forceinline__ void tma_gather4_2d(uint32_t dst, const CUtensorMap* map, int c0, int r0, int r1, int r2, int r3,
+                                               uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar)
+      : "memory");
+}
+
 // ---- tensor memory ----------------------------------------------------------------------------------
 // Whole-warp calls.  The base address (lane 0, first column) is written to the shared word `slot`.
 __device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t n_cols) {

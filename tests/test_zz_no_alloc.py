@@ -22,6 +22,7 @@ def _run_static(wl, q0, n):
     binding.index_static(wl.params, wl.q_idx[q0 - wl.q_pos0:], wl.w[q0 - wl.q_pos0:], wl.keys["k"], wl.keys.get("scale"),
                          wl.kmean, q0, n, wl.n_key, idx, cnt)
     torch.cuda.synchronize()
+    assert binding.index_static_status(wl.device) == 0     # no bounded device-side wait ran out
     return idx, cnt
 
 
@@ -44,6 +45,23 @@ def test_static_scratch_indexer_matches_workspace_indexer_twice(cuda_device):
     # a query sub-range with an offset, again on the shared array
     idx, cnt = _run_static(a, 4000, 1500)
     assert torch.equal(idx, a.sparse_idx[4000:5500]) and torch.equal(cnt, a.n_sparse[4000:5500])
+
+
+def test_static_scratch_refuses_misaligned_pointers_before_any_launch(cuda_device):
+    """The kernels read q_idx, w, k_idx and kmean with 16-byte vector loads: a pointer off by two bytes is refused with
+    LSA_ERR_SHAPE by the host-side checks (the same ones lsa_index makes); nothing reaches the GPU."""
+    cfg = CONFIGS["cfg1"]
+    params = binding.make_params(cfg)
+    buf = torch.zeros(1 << 16, dtype=torch.uint8, device=cuda_device)
+    ok, off = buf[256:], buf[258:]
+    out = torch.zeros(64, dtype=torch.int32, device=cuda_device)
+    for which in range(4):
+        ptrs = [off if i == which else ok for i in range(4)]     # q_idx, w, k_idx, kmean
+        with pytest.raises(binding.LsaError) as e:
+            binding.index_static(params, ptrs[0], ptrs[1], ptrs[2], None, ptrs[3], 0, 4, 64, out, out)
+        assert e.value.code == -2
+    torch.cuda.synchronize()
+    assert binding.index_static_status(cuda_device) == 0
 
 
 def test_static_scratch_capacity_is_enforced(cuda_device):
