@@ -150,21 +150,49 @@ struct AttnTcSmem {
   alignas(1024) uint8_t q_rope[kAtomBytes];                 // Q[:, 512:576], 64 rows x 128 B
   alignas(1024) uint8_t k[kKBufs][kAtoms][kAtomBytes];      // [tile buffer][column block][64 rows x 128 B]
   alignas(8) uint64_t q_full, q_tmem, k_full[kKBufs], k_empty[kKBufs], s_full[2], p_ready[2];
+  alignas(8) uint64_t recv_full;          // two-split launches: the peer's rows and log-sum-exps have arrived
   uint32_t tmem_slot;
-  float lse_own[kH];              // split launches: this block's log-sum-exp per head (log2 units)
+  alignas(16) float lse_own[kH];          // split launches: this block's log-sum-exp per head (log2 units)
+  alignas(16) float lse_peer[kH / 2];     // two-split launches: the peer's, for the heads this block finishes
 };
+constexpr int kPitchPart = kDV * 4 + 16;                  // staged fp32 row of a partial result, padded against bank conflicts
+constexpr int kRecvOffset = kH * kPitchPart;              // two-split launches: the peer's rows land behind the staged ones
+constexpr uint32_t kRecvBytes = (kH / 2) * kDV * 4 + (kH / 2) * 4;
+static_assert(kRecvOffset + (kH / 2) * kDV * 4 <= kKBufs * kAtoms * kAtomBytes, "staged and received rows must fit the key buffers");
 
 // ---- thread-block cluster: barrier and loads from a peer block's shared memory
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// The two halves of the cluster barrier on their own: a thread arrives when it is done with a phase and waits later,
+// where it needs every thread of the cluster to have arrived.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+// Address of this block's shared-memory location `addr` in the block of rank `rank` of the cluster.
+__device__ __forceinline__ uint32_t peer_smem(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+// Bulk copy from this block's shared memory into a peer block's (addresses from peer_smem); the bytes are counted on
+// the peer's mbarrier.  16-byte aligned addresses, size a multiple of 16.
+__device__ __forceinline__ void bulk_copy_to_peer(uint32_t dst_peer, uint32_t src, uint32_t bytes, uint32_t bar_peer) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst_peer), "r"(src), "r"(bytes), "r"(bar_peer) : "memory");
+}
 // With n_split > 1 the kernel must be launched with clusters of (1, n_split, 1) blocks: the splits of one sequence
 // are co-scheduled and merge their partial results themselves (no second kernel).  Block s finishes heads
-// [s * 64 / n_split, (s + 1) * 64 / n_split): every block stages its rows (normalised, fp32) in shared memory, keeps its
-// own share there and sends the other rows (one bulk copy per row) and all its log-sum-exps to the global scratch, where
-// they stay in L2; after one cluster barrier the owner of a row combines its own part with the others'.  (Distributed shared memory moved the
-// same rows at about a quarter of the L2 path's rate, so it carries nothing here.)
+// [s * 64 / n_split, (s + 1) * 64 / n_split): every block stages its rows (normalised, fp32) in shared memory and keeps
+// its own share there.
+//   Two splits (the decode configuration): the other 32 rows and their log-sum-exps are pushed straight into the
+//   peer's shared memory, behind its staged rows, by bulk copies that count bytes on the peer's mbarrier.  The cluster
+//   barrier is used in halves: a thread arrives when it has left the tile loop and waits before the first copy (the
+//   peer's key buffers must be out of use before they receive), and once more around the end, so that no block leaves
+//   while the other may still write into it.  Nothing goes through global memory.
+//   Four or eight splits: the other rows (one bulk copy per row) and all log-sum-exps go to the global scratch, where
+//   they stay in L2; after one cluster barrier the owner of a row combines its own part with the others'.  (Loads from
+//   a peer's shared memory moved the same rows at about a quarter of the L2 path's rate.)
 //
 // q_tma != 0: q_map describes q as a bf16 matrix [n_query * 64, 576] and Q arrives as nine TMA boxes; otherwise the
 // gather warps copy it with cp.async.  k_tma != 0 (contiguous caches only): k_map describes the cache rows, and key
@@ -194,6 +222,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
 
   constexpr int n_pv = kPv;
   constexpr bool clustered = kClustered;
+  const bool pair = kClustered && p.n_split == 2;   // two splits exchange their rows through shared memory
   const bool dead = tc::status_raised(p.status);   // an earlier block of this launch (or an earlier launch) gave up on a wait
   if (dead && !clustered) return;
 
@@ -210,6 +239,10 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
     for (int b = 0; b < 2; ++b) {
       tc::mbar_init(smem_u32(&sm.s_full[b]), 2);
       tc::mbar_init(smem_u32(&sm.p_ready[b]), kSoftmaxWarps);
+    }
+    if constexpr (kClustered) {
+      tc::mbar_init(smem_u32(&sm.recv_full), 1);
+      if (p.n_split == 2) tc::mbar_expect_tx(smem_u32(&sm.recv_full), kRecvBytes);   // armed once; used once per launch
     }
     tc::fence_mbar_init();
   }
@@ -656,6 +689,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
     bool have_o = ok && n_tiles > 0;
     if (have_o) have_o = __all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.k_empty[(n_tiles - 1) % kKBufs]), ((n_tiles - 1) / kKBufs) & 1, p.status));
     tc::fence_after_sync();
+    if (pair) cluster_arrive();   // this thread has left the tile loop, and every P V of the block has completed
     if (tid == 0) LSA_TL(kTlLastPV);
     const float inv = (have_o && l_row > 0.f) ? 1.f / l_row : 0.f;
     const float lse2 = (have_o && l_row > 0.f) ? m_row + log2f(l_row) : -INFINITY;   // log2 domain
@@ -699,7 +733,6 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       if (hi == 0 && lse_ptr != nullptr) lse_ptr[static_cast<int64_t>(qi) * kH + row] = lse2 / kLog2eTc;
     } else {
       // partial result of a split: normalised fp32 rows in the key buffers (padded against bank conflicts)
-      constexpr int kPitchPart = kDV * 4 + 16;
       uint8_t* my_stage = stage + row * kPitchPart + hi * (kDV * 2);
 #pragma unroll 1
       for (int c = 0; c < 256; c += 64) {
@@ -719,22 +752,40 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       }
       if (hi == 0) {
         sm.lse_own[row] = lse2;
-        part_lse[(static_cast<int64_t>(qi) * p.n_split + split) * kH + row] = lse2;
+        if (!pair) part_lse[(static_cast<int64_t>(qi) * p.n_split + split) * kH + row] = lse2;
       }
-      // Rows that another block of the cluster finishes go to the global scratch as soon as this warp has staged them:
-      // one bulk copy per row (2 KB), issued by the lane that holds the row's first half, while the other softmax warps
-      // are still staging.
+      // Rows that another block of the cluster finishes leave as soon as this warp has staged them: one bulk copy per
+      // row (2 KB), issued by the lane that holds the row's first half, while the other softmax warps are still staging.
       tc::fence_proxy_async();
       __syncwarp();
-      const int rows_per = kH / p.n_split;
-      if (hi == 0 && row / rows_per != split) {
-        float* dst = part_out + ((static_cast<int64_t>(qi) * p.n_split + split) * kH + row) * kDV;
-        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                     :: "l"(dst), "r"(smem_u32(stage + row * kPitchPart)), "n"(kDV * 4) : "memory");
-        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      if (pair) {
+        // into the peer's shared memory, once every thread of the peer has left its tile loop (first half of the
+        // cluster barrier: its key buffers, which receive the rows, are then out of use)
+        cluster_wait();
+        const uint32_t peer = static_cast<uint32_t>(split ^ 1);
+        const int peer_row0 = (kH / 2) * (split ^ 1);
+        if (row / (kH / 2) != split) {   // warp-uniform: a warp stages 16 consecutive rows
+          const uint32_t bar = peer_smem(smem_u32(&sm.recv_full), peer);
+          if (hi == 0)
+            bulk_copy_to_peer(peer_smem(smem_u32(stage + kRecvOffset + (row - peer_row0) * (kDV * 4)), peer),
+                              smem_u32(stage + row * kPitchPart), kDV * 4, bar);
+          if (lane == 0)
+            bulk_copy_to_peer(peer_smem(smem_u32(&sm.lse_peer[16 * quarter - peer_row0]), peer), smem_u32(&sm.lse_own[16 * quarter]),
+                              16 * 4, bar);
+        }
+      } else {
+        const int rows_per = kH / p.n_split;
+        if (hi == 0 && row / rows_per != split) {
+          float* dst = part_out + ((static_cast<int64_t>(qi) * p.n_split + split) * kH + row) * kDV;
+          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                       :: "l"(dst), "r"(smem_u32(stage + row * kPitchPart)), "n"(kDV * 4) : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
       }
     }
   }
+  // the threads of the other roles have left the tile loop too
+  if (pair && warp >= kSoftmaxWarps) cluster_arrive();
   if (tid == 0) LSA_TL(kTlStaged);
   tc::fence_before_sync();
   __syncthreads();
@@ -746,36 +797,30 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
     const int n = p.n_split;
     const int rows_per = kH / n;
     const int row0 = split * rows_per;
-    constexpr int kPitchPart = kDV * 4 + 16;
     const uint8_t* stage = &sm.k[0][0][0];
-    if (warp < kSoftmaxWarps) {   // the threads that sent rows wait until they are written (not only read out of shared memory)
-      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-      __threadfence();
+    constexpr int kWarps = kThreadsAttnTc / 32;
+    if (pair) {
+      if (warp >= kSoftmaxWarps) cluster_wait();   // (the softmax warps completed this phase before they sent)
+      // the peer's rows for this block's heads, and their log-sum-exps, are in shared memory when the byte count is met
+      (void)tc::mbar_wait(smem_u32(&sm.recv_full), 0, p.status);
+      if (tid == 0) LSA_TL(kTlClusterSync);
+    } else {
+      if (warp < kSoftmaxWarps) {   // the threads that sent rows wait until they are written (not only read out of shared memory)
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        __threadfence();
+      }
+      if (tid == 0) LSA_TL(kTlSent);
+      cluster_sync_all();   // every block of the cluster has written its rows
+      if (tid == 0) LSA_TL(kTlClusterSync);
     }
-    if (tid == 0) LSA_TL(kTlSent);
-    cluster_sync_all();   // every block of the cluster has written its rows
-    if (tid == 0) LSA_TL(kTlClusterSync);
     // Warp w finishes rows w, w + 12, ... of this block's share (at most three).  Lane 8k + j first fetches the
     // log-sum-exp of split j for the warp's k-th row, so that all of them are in flight together.
-    constexpr int kWarps = kThreadsAttnTc / 32;
-    // two splits (the usual decode case): the peer's parts of all of this warp's rows are requested before the first is used
-    float4 pre[3][4];
-    if (n == 2) {
-#pragma unroll
-      for (int k = 0; k < 3; ++k) {
-        const int rl = warp + kWarps * k;
-        if (rl < rows_per) {
-          const float4* src = reinterpret_cast<const float4*>(part_out + ((static_cast<int64_t>(qi) * 2 + (split ^ 1)) * kH + row0 + rl) * kDV);
-#pragma unroll
-          for (int u = 0; u < 4; ++u) pre[k][u] = __ldcg(src + lane + 32 * u);
-        }
-      }
-    }
     const int k_of = lane >> 3, j_of = lane & 7;
     const int rl_mine = warp + kWarps * k_of;
     float my_l = -INFINITY;
     if (k_of < 3 && rl_mine < rows_per && j_of < n)
       my_l = j_of == split ? sm.lse_own[row0 + rl_mine]
+             : pair        ? sm.lse_peer[rl_mine]
                            : __ldcg(part_lse + (static_cast<int64_t>(qi) * n + j_of) * kH + row0 + rl_mine);
     float m = my_l;
 #pragma unroll
@@ -801,9 +846,9 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
           if (j == split) {
 #pragma unroll
             for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const float4*>(stage + (row0 + rl) * kPitchPart + (lane + 32 * u) * 16);
-          } else if (n == 2) {
+          } else if (pair) {
 #pragma unroll
-            for (int u = 0; u < 4; ++u) v[u] = pre[k][u];
+            for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const float4*>(stage + kRecvOffset + rl * (kDV * 4) + (lane + 32 * u) * 16);
           } else {
             const float4* src = reinterpret_cast<const float4*>(part_out + ((static_cast<int64_t>(qi) * n + j) * kH + row0 + rl) * kDV);
 #pragma unroll
@@ -824,6 +869,12 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       }
     }
     if (tid == 0) LSA_TL(kTlMerged);
+    if (pair) {
+      // second use of the cluster barrier: a block leaves only when the peer has everything it was sent (its own
+      // arrival follows its wait for those bytes), so no copy is ever in flight towards a block that has gone
+      cluster_arrive();
+      cluster_wait();
+    }
   }
   if (tid == 0) {
     LSA_TL(kTlExit);
