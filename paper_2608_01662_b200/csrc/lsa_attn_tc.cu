@@ -156,9 +156,14 @@ struct AttnTcSmem {
   alignas(16) float lse_peer[kH / 2];     // two-split launches: the peer's, for the heads this block finishes
 };
 constexpr int kPitchPart = kDV * 4 + 16;                  // staged fp32 row of a partial result, padded against bank conflicts
-constexpr int kRecvOffset = kH * kPitchPart;              // two-split launches: the peer's rows land behind the staged ones
+// Two-split launches stage their rows unpadded, with the 16-byte chunks of row r XOR-swizzled by r % 8 (no bank
+// conflicts either way), so that the 16 rows a warp stages are one contiguous piece and leave as one bulk copy; the
+// peer's rows land behind the staged ones.
+constexpr int kPairRowBytes = kDV * 4;
+constexpr int kRecvOffset = kH * kPairRowBytes;
 constexpr uint32_t kRecvBytes = (kH / 2) * kDV * 4 + (kH / 2) * 4;
-static_assert(kRecvOffset + (kH / 2) * kDV * 4 <= kKBufs * kAtoms * kAtomBytes, "staged and received rows must fit the key buffers");
+static_assert(kRecvOffset + (kH / 2) * kPairRowBytes <= kKBufs * kAtoms * kAtomBytes, "staged and received rows must fit the key buffers");
+static_assert(kH * kPitchPart <= kKBufs * kAtoms * kAtomBytes, "staged rows must fit the key buffers");
 
 // ---- thread-block cluster: barrier and loads from a peer block's shared memory
 __device__ __forceinline__ void cluster_sync_all() {
@@ -733,7 +738,8 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       if (hi == 0 && lse_ptr != nullptr) lse_ptr[static_cast<int64_t>(qi) * kH + row] = lse2 / kLog2eTc;
     } else {
       // partial result of a split: normalised fp32 rows in the key buffers (padded against bank conflicts)
-      uint8_t* my_stage = stage + row * kPitchPart + hi * (kDV * 2);
+      uint8_t* my_row = stage + row * (pair ? kPairRowBytes : kPitchPart);
+      const int sw = pair ? (row & 7) : 0;
 #pragma unroll 1
       for (int c = 0; c < 256; c += 64) {
         uint32_t o[64];
@@ -745,8 +751,8 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
           for (int j = 0; j < 64; ++j) o[j] = 0u;
         }
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-          *reinterpret_cast<float4*>(my_stage + (c + 4 * j) * 4) =
+        for (int j = 0; j < 16; ++j)   // 16-byte chunk hi * 64 + c / 4 + j of the row
+          *reinterpret_cast<float4*>(my_row + (((hi * 64 + c / 4 + j) ^ sw) << 4)) =
               make_float4(__uint_as_float(o[4 * j]) * inv, __uint_as_float(o[4 * j + 1]) * inv,
                           __uint_as_float(o[4 * j + 2]) * inv, __uint_as_float(o[4 * j + 3]) * inv);
       }
@@ -754,8 +760,8 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
         sm.lse_own[row] = lse2;
         if (!pair) part_lse[(static_cast<int64_t>(qi) * p.n_split + split) * kH + row] = lse2;
       }
-      // Rows that another block of the cluster finishes leave as soon as this warp has staged them: one bulk copy per
-      // row (2 KB), issued by the lane that holds the row's first half, while the other softmax warps are still staging.
+      // Rows that another block of the cluster finishes leave as soon as this warp has staged them, while the other
+      // softmax warps are still staging.
       tc::fence_proxy_async();
       __syncwarp();
       if (pair) {
@@ -766,16 +772,16 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
         const int peer_row0 = (kH / 2) * (split ^ 1);
         if (row / (kH / 2) != split) {   // warp-uniform: a warp stages 16 consecutive rows
           const uint32_t bar = peer_smem(smem_u32(&sm.recv_full), peer);
-          if (hi == 0)
-            bulk_copy_to_peer(peer_smem(smem_u32(stage + kRecvOffset + (row - peer_row0) * (kDV * 4)), peer),
-                              smem_u32(stage + row * kPitchPart), kDV * 4, bar);
-          if (lane == 0)
+          if (lane == 0) {   // the warp's 16 rows are one piece of 32 KB; their log-sum-exps another of 64 bytes
+            bulk_copy_to_peer(peer_smem(smem_u32(stage + kRecvOffset + (16 * quarter - peer_row0) * kPairRowBytes), peer),
+                              smem_u32(stage + 16 * quarter * kPairRowBytes), 16 * kPairRowBytes, bar);
             bulk_copy_to_peer(peer_smem(smem_u32(&sm.lse_peer[16 * quarter - peer_row0]), peer), smem_u32(&sm.lse_own[16 * quarter]),
                               16 * 4, bar);
+          }
         }
       } else {
         const int rows_per = kH / p.n_split;
-        if (hi == 0 && row / rows_per != split) {
+        if (hi == 0 && row / rows_per != split) {   // one bulk copy per row (2 KB), issued by the lane that holds its first half
           float* dst = part_out + ((static_cast<int64_t>(qi) * p.n_split + split) * kH + row) * kDV;
           asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                        :: "l"(dst), "r"(smem_u32(stage + row * kPitchPart)), "n"(kDV * 4) : "memory");
@@ -804,6 +810,36 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       // the peer's rows for this block's heads, and their log-sum-exps, are in shared memory when the byte count is met
       (void)tc::mbar_wait(smem_u32(&sm.recv_full), 0, p.status);
       if (tid == 0) LSA_TL(kTlClusterSync);
+      __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(out_ptr) + (static_cast<int64_t>(qi) * kH + row0) * kDV;
+#pragma unroll 1
+      for (int rl = warp; rl < kH / 2; rl += kWarps) {   // a warp finishes a row: lane l the chunks l, l + 32, ...
+        const int R = row0 + rl;
+        const float l_own = sm.lse_own[R], l_peer = sm.lse_peer[rl];
+        const float m = fmaxf(l_own, l_peer);
+        float w_own = m > -INFINITY ? exp2f(l_own - m) : 0.f, w_peer = m > -INFINITY ? exp2f(l_peer - m) : 0.f;
+        const float den = w_own + w_peer;
+        const float r_den = den > 0.f ? 1.f / den : 0.f;
+        w_own *= r_den;
+        w_peer *= r_den;
+        if (lane == 0 && lse_ptr != nullptr)
+          lse_ptr[static_cast<int64_t>(qi) * kH + R] = den > 0.f ? (m + log2f(den)) / kLog2eTc : -INFINITY;
+        const uint8_t* a_row = stage + R * kPairRowBytes;
+        const uint8_t* b_row = stage + kRecvOffset + rl * kPairRowBytes;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int ch = ((lane + 32 * u) ^ (R & 7)) << 4;   // the peer staged head R with the same swizzle
+          const float4 a = *reinterpret_cast<const float4*>(a_row + ch), b = *reinterpret_cast<const float4*>(b_row + ch);
+          uint2 o;
+          o.x = pack_bf16(w_own * a.x + w_peer * b.x, w_own * a.y + w_peer * b.y);
+          o.y = pack_bf16(w_own * a.z + w_peer * b.z, w_own * a.w + w_peer * b.w);
+          *reinterpret_cast<uint2*>(out + static_cast<int64_t>(rl) * kDV + (lane + 32 * u) * 4) = o;
+        }
+      }
+      if (tid == 0) LSA_TL(kTlMerged);
+      // second use of the cluster barrier: a block leaves only when the peer has everything it was sent (its own
+      // arrival follows its wait for those bytes), so no copy is ever in flight towards a block that has gone
+      cluster_arrive();
+      cluster_wait();
     } else {
       if (warp < kSoftmaxWarps) {   // the threads that sent rows wait until they are written (not only read out of shared memory)
         asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
@@ -812,7 +848,6 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       if (tid == 0) LSA_TL(kTlSent);
       cluster_sync_all();   // every block of the cluster has written its rows
       if (tid == 0) LSA_TL(kTlClusterSync);
-    }
     // Warp w finishes rows w, w + 12, ... of this block's share (at most three).  Lane 8k + j first fetches the
     // log-sum-exp of split j for the warp's k-th row, so that all of them are in flight together.
     const int k_of = lane >> 3, j_of = lane & 7;
@@ -820,7 +855,6 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
     float my_l = -INFINITY;
     if (k_of < 3 && rl_mine < rows_per && j_of < n)
       my_l = j_of == split ? sm.lse_own[row0 + rl_mine]
-             : pair        ? sm.lse_peer[rl_mine]
                            : __ldcg(part_lse + (static_cast<int64_t>(qi) * n + j_of) * kH + row0 + rl_mine);
     float m = my_l;
 #pragma unroll
@@ -846,9 +880,6 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
           if (j == split) {
 #pragma unroll
             for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const float4*>(stage + (row0 + rl) * kPitchPart + (lane + 32 * u) * 16);
-          } else if (pair) {
-#pragma unroll
-            for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const float4*>(stage + kRecvOffset + rl * (kDV * 4) + (lane + 32 * u) * 16);
           } else {
             const float4* src = reinterpret_cast<const float4*>(part_out + ((static_cast<int64_t>(qi) * n + j) * kH + row0 + rl) * kDV);
 #pragma unroll
@@ -869,12 +900,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       }
     }
     if (tid == 0) LSA_TL(kTlMerged);
-    if (pair) {
-      // second use of the cluster barrier: a block leaves only when the peer has everything it was sent (its own
-      // arrival follows its wait for those bytes), so no copy is ever in flight towards a block that has gone
-      cluster_arrive();
-      cluster_wait();
-    }
+    }   // four or eight splits
   }
   if (tid == 0) {
     LSA_TL(kTlExit);
