@@ -146,9 +146,9 @@ WsLayout ws_layout(const lsa_params* p, int64_t n_query, int64_t n_key_max, int 
     l.fine_pages = off;
     off += align_up(static_cast<size_t>(batch) * 65 * sizeof(int32_t), 256);
   }
-  const bool flat = !p->hi_enable && !p->paged && n_key_max > kFlatFusedMaxKeys;
+  const bool flat = !p->hi_enable && n_key_max > kFlatFusedMaxKeys;
   const bool tc_fine = !p->paged && p->n_heads_idx == 64 && p->d_idx == 128;
-  if ((flat || tc_fine) && p->key_dtype == LSA_KEY_E4M3) {
+  if (!p->paged && (flat || tc_fine) && p->key_dtype == LSA_KEY_E4M3) {
     // e4m3 codes widened to bf16 once per call: dense scoring of the flat indexer, TMA source of the fine stage
     l.wide_keys = off;
     off += align_up(static_cast<size_t>(n_key_max) * p->d_idx * 2, 256);
@@ -202,7 +202,6 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
   if (nq == 0) return LSA_OK;
   const int64_t n_key_max = p->paged ? pt_stride * p->kv_page : n_key;
   const bool flat = !p->hi_enable && n_key_max > kFlatFusedMaxKeys;
-  if (flat && p->paged) return LSA_ERR_SHAPE;   // the flat indexer over long caches is built for contiguous caches only
   const int64_t chunk = (!p->paged && p->q_chunk > 0) ? p->q_chunk : nq;
   const WsLayout l = ws_layout(p, chunk < nq ? chunk : nq, n_key_max, batch);
   if (c->ws == nullptr || l.total > c->ws_bytes) return LSA_ERR_WORKSPACE;
@@ -224,7 +223,15 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
     a.n_rows_out = n_rows_out;
     a.status = status_word(c);
     a.fine_parts = 1;
-    if (p->paged) {
+    a.sm_count = c->sm_count;
+    const bool paged_tc = p->paged && lsa::paged_scores_tc_supported(a);   // token scores of cache pages on tcgen05
+    if (flat && p->paged && !paged_tc) return LSA_ERR_SHAPE;   // the flat indexer over long paged caches needs that kernel
+    if (paged_tc && (flat || c->tune[LSA_TUNE_FINE_PAGED_TC])) {
+      a.fine_paged_tc = 1;
+      a.fine_parts = 2;   // (marks the split path: the top-K kernel writes the cache rows itself)
+      a.fine_keys = reinterpret_cast<uint32_t*>(c->ws + l.fine_keys);
+      a.fine_pages = reinterpret_cast<int32_t*>(c->ws + l.fine_pages);
+    } else if (p->paged) {
       // few queries and many SMs: several blocks score each query's candidates, a second kernel selects
       int parts = 2 * c->sm_count / (batch > 0 ? batch : 1);   // two scoring blocks fit one SM
       parts = parts > 4 ? 4 : parts;
@@ -241,6 +248,26 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
       if (q0 == 0) e = timed(c, LSA_K_MEANS, [&] { return lsa::launch_widen_e4m3(k_idx, wide, n_key * p->d_idx, c->stream, &c->launches); });
       if (e != cudaSuccess) return cuda_fail(c, e);
       a.k_wide = wide;
+    }
+    if (flat && p->paged) {
+      // Eq. 7 without the hierarchy over paged caches: token scores of every page of the scoring range (per-token
+      // scale applied), the top-K_sparse of each sequence's row, then the cache rows.
+      e = timed(c, LSA_K_COARSE, [&] { return lsa::launch_paged_scores_tc(a, 1, c->sm_count, c->stream, &c->launches); });
+      if (e == cudaSuccess)
+        e = timed(c, LSA_K_SELECT, [&] {
+          return lsa::launch_select(a.page_scores, a.ps_ld, nullptr, nullptr, 0, a.n_query, n_key_max, p->k_sparse, 1, p->k_sink,
+                                    p->k_swa, a.sparse_idx, a.n_sparse, c->stream, &c->launches, ctx_len);
+        });
+      if (e == cudaSuccess && a.rows_out != nullptr)
+        e = timed(c, LSA_K_CONVERT, [&] {
+          return lsa::launch_convert(p->k_sink, p->k_swa, p->k_sparse, p->paged, p->kv_page, a.sparse_idx, a.n_sparse, a.q_pos0,
+                                     a.n_query, page_table, pt_stride, ctx_len, a.rows_out, a.n_rows_out, nullptr, c->stream,
+                                     &c->launches);
+        });
+      if (e == cudaSuccess && a.pages_out != nullptr)
+        e = cudaMemsetAsync(a.pages_out, 0xff, static_cast<size_t>(a.n_query) * p->keep_pages * sizeof(int32_t), c->stream);
+      if (e != cudaSuccess) return cuda_fail(c, e);
+      continue;
     }
     if (flat) {
       // Eq. 7 without the hierarchy: dense causal token scores (the coarse kernel with one token per "page"), then
@@ -430,6 +457,7 @@ int lsa_tune(lsa_ctx* c, int knob, int value) {
   if (knob == LSA_TUNE_ATTN_SPLIT && (value < 0 || value > kMaxSplit)) return LSA_ERR_ARG;
   if (knob == LSA_TUNE_ATTN_PV_WAIT && value != 0 && value != 1) return LSA_ERR_ARG;
   if (knob == LSA_TUNE_ATTN_GATHER && value != 0 && value != 1) return LSA_ERR_ARG;
+  if (knob == LSA_TUNE_FINE_PAGED_TC && value != 0 && value != 1) return LSA_ERR_ARG;
   c->tune[knob] = value;
   return LSA_OK;
 }

@@ -621,6 +621,53 @@ __global__ void __launch_bounds__(kThreads, 2) fine_select_kernel(IndexArgs p) {
   // template trips an internal error of nvcc 12.9)
 }
 
+// a2 for paged caches as a kernel of its own (the tcgen05 scoring kernel that follows walks ready-made page lists):
+// the pages of sequence qi that survive the coarse stage (Eq. 10), ascending, into fine_pages[qi], their count last.
+// A sequence without candidates gets its (empty) results here.
+__global__ void __launch_bounds__(kSelThreads) page_topm_paged_kernel(IndexArgs p) {
+  __shared__ uint32_t keys[kMaxSlots];
+  __shared__ int32_t pages[kMaxPages];
+  __shared__ SelectScratch sc;
+  const int qi = blockIdx.x, tid = threadIdx.x;
+  pdl_wait();
+  pdl_launch_dependents();
+  const int64_t t = static_cast<int64_t>(p.ctx_len[qi]) - 1;
+  const int64_t lo = p.S, hi = t - p.W;
+  int32_t* fp = p.fine_pages + qi * (kMaxPages + 1);
+  int32_t* out_pages = p.pages_out ? p.pages_out + static_cast<int64_t>(qi) * p.M : nullptr;
+  if (hi < lo) {
+    if (tid == 0) {
+      fp[kMaxPages] = 0;
+      p.n_sparse[qi] = 0;
+    }
+    for (int i = tid; i < p.Ksp; i += kSelThreads) p.sparse_idx[static_cast<int64_t>(qi) * p.Ksp + i] = -1;
+    if (out_pages) for (int i = tid; i < p.M; i += kSelThreads) out_pages[i] = -1;
+    emit_rows_of_query<kSelThreads>(p.rows_out, p.n_rows_out, p.sparse_idx, p.page_table, p.pt_stride, t, p.S, p.W, p.Ksp, p.paged,
+                                    p.P, qi, tid, 0);
+    return;
+  }
+  const int p0 = static_cast<int>(lo / p.P), p1 = static_cast<int>(hi / p.P);
+  const int nE = p1 - p0 + 1;
+  int nP;
+  if (p.hi_enable && nE > p.M) {
+    const float* ps = p.page_scores + static_cast<int64_t>(qi) * p.ps_ld + p0;
+    if (nE <= kMaxSlots) {
+      for (int i = tid; i < nE; i += kSelThreads) keys[i] = score_key(ps[i]);
+      __syncthreads();
+      nP = block_select_topk([&](int i) { return keys[i]; }, [&](int i) { return p0 + i; }, nE, p.M, pages, sc);
+    } else {
+      nP = block_select_topk([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M, pages, sc);
+    }
+  } else {
+    nP = nE;   // the host guarantees nE <= kMaxPages here
+    for (int i = tid; i < nP; i += kSelThreads) pages[i] = p0 + i;
+    __syncthreads();
+  }
+  for (int i = tid; i < nP; i += kSelThreads) fp[i] = pages[i];
+  if (tid == 0) fp[kMaxPages] = nP;
+  if (out_pages) for (int i = tid; i < p.M; i += kSelThreads) out_pages[i] = i < nP ? pages[i] : -1;
+}
+
 // Second half of the split fine stage: top-K_sparse over the keys the scoring blocks left in global memory.
 __global__ void __launch_bounds__(kSelThreads) fine_topk_kernel(IndexArgs p) {
   __shared__ uint32_t keys[kMaxSlots];
@@ -655,12 +702,14 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
                                                             const int32_t* __restrict__ cand_pos,
                                                             const float* __restrict__ pos_scale, int64_t q_pos0,
                                                             int64_t n_cand, int k, int apply_range, int S, int W,
-                                                            int32_t* __restrict__ idx_out, int32_t* __restrict__ n_out) {
+                                                            int32_t* __restrict__ idx_out, int32_t* __restrict__ n_out,
+                                                            const int32_t* __restrict__ ctx_len) {
   __shared__ SelectScratch sc;
   const int qi = blockIdx.x;
   const float* row = scores + qi * ld;
   const int32_t* pos = cand_pos ? cand_pos + qi * n_cand : nullptr;
-  const int64_t lo = S, hi = q_pos0 + qi - W;
+  // the query of row qi sits at q_pos0 + qi, or (paged caches: one query per sequence) at the end of its sequence
+  const int64_t lo = S, hi = (ctx_len ? static_cast<int64_t>(ctx_len[qi]) - 1 : q_pos0 + qi) - W;
   auto id = [&](int i) { return pos ? pos[i] : i; };
   auto key = [&](int i) -> uint32_t {
     const int64_t s = id(i);
@@ -1103,6 +1152,18 @@ static cudaError_t launch_fine_t(const IndexArgs& a, cudaStream_t st, int64_t* n
 
 cudaError_t launch_fine_select(const IndexArgs& a, cudaStream_t st, int64_t* n_launch) {
   if (a.n_query == 0) return cudaSuccess;
+  if (a.fine_paged_tc && a.paged && a.fine_keys != nullptr && a.fine_pages != nullptr && paged_scores_tc_supported(a)) {
+    // decode: page lists, then token scores of the listed pages on tcgen05, then the top-K_sparse with the cache rows
+    cudaError_t e = launch_pdl(page_topm_paged_kernel, dim3(a.n_query), dim3(kSelThreads), 0, st, a);
+    if (e != cudaSuccess) return e;
+    ++*n_launch;
+    e = launch_paged_scores_tc(a, 0, a.sm_count, st, n_launch);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(fine_topk_kernel, dim3(a.n_query), dim3(kSelThreads), 0, st, a);
+    if (e != cudaSuccess) return e;
+    ++*n_launch;
+    return cudaGetLastError();
+  }
   if (fine_tc_supported(a)) {
     cudaError_t e = launch_fine_select_tc(a, st, n_launch);
     if (e != cudaSuccess || a.fine_parts <= 1) return e;
@@ -1127,10 +1188,10 @@ cudaError_t launch_widen_e4m3(const void* codes, void* out_bf16, int64_t n_elems
 
 cudaError_t launch_select(const float* scores, int64_t ld, const int32_t* cand_pos, const float* pos_scale,
                           int64_t q_pos0, int n_query, int64_t n_cand, int k, int apply_range, int S, int W,
-                          int32_t* idx_out, int32_t* n_out, cudaStream_t st, int64_t* n_launch) {
+                          int32_t* idx_out, int32_t* n_out, cudaStream_t st, int64_t* n_launch, const int32_t* ctx_len) {
   if (n_query == 0) return cudaSuccess;
   select_kernel<<<n_query, kSelThreads, 0, st>>>(scores, ld, cand_pos, pos_scale, q_pos0, n_cand, k, apply_range, S, W,
-                                                 idx_out, n_out);
+                                                 idx_out, n_out, ctx_len);
   ++*n_launch;
   return cudaGetLastError();
 }

@@ -41,6 +41,8 @@ struct IndexArgs {
   int fine_parts;         // 1: fused kernel; >1: blocks per query in the scoring kernel
   uint32_t* fine_keys;    // [n_query, 4096] order-preserving keys of the candidate slots (0 = not a candidate)
   int32_t* fine_pages;    // [n_query, 65]: kept pages, then their count
+  int sm_count;           // SMs of the device (grid of the persistent paged kernels)
+  int fine_paged_tc;      // paged caches: page lists, token scores on tcgen05 (lsa_scores_paged_tc.cu), top-K, as three kernels
   int* status;
 };
 
@@ -116,9 +118,15 @@ cudaError_t launch_fine_select_tc(const IndexArgs& a, cudaStream_t st, int64_t* 
 bool fine_big_supported(const IndexArgs& a);
 cudaError_t launch_fine_big(const IndexArgs& a, int32_t* pages_ws, int32_t* n_pages_ws, uint32_t* keys, cudaStream_t st,
                             int64_t* n_launch);
+// ctx_len != NULL (paged caches): the query of row i sits at ctx_len[i] - 1 instead of q_pos0 + i
 cudaError_t launch_select(const float* scores, int64_t ld, const int32_t* cand_pos, const float* pos_scale,
                           int64_t q_pos0, int n_query, int64_t n_cand, int k, int apply_range, int S, int W,
-                          int32_t* idx_out, int32_t* n_out, cudaStream_t st, int64_t* n_launch);
+                          int32_t* idx_out, int32_t* n_out, cudaStream_t st, int64_t* n_launch,
+                          const int32_t* ctx_len = nullptr);
+// Token scores over cache pages on tcgen05 (paged caches, 64-token pages, H_I = 64, d_I = 128).  flat = 0: keys of the
+// slots of the page lists a.fine_pages -> a.fine_keys; flat = 1: scores of the whole scoring range -> a.page_scores.
+bool paged_scores_tc_supported(const IndexArgs& a);
+cudaError_t launch_paged_scores_tc(const IndexArgs& a, int flat, int sm_count, cudaStream_t st, int64_t* n_launch);
 cudaError_t launch_widen_e4m3(const void* codes, void* out_bf16, int64_t n_elems, cudaStream_t st, int64_t* n_launch);
 cudaError_t launch_convert(int S, int W, int Ksp, int paged, int kv_page, const int32_t* sparse_idx,
                            const int32_t* n_sparse, int64_t q_pos0, int n_query, const int32_t* page_table,

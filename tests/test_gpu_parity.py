@@ -213,6 +213,49 @@ def test_small_paged_decode(cuda_device):
     m.assert_ok(pu.TOL_FP8)
 
 
+@pytest.mark.parametrize("key_dtype", ["e4m3", "bf16"])
+def test_flat_indexer_on_paged_caches(cuda_device, key_dtype):
+    """hi_enable = 0 in decode (what the paper itself runs there): Eq. 7 over every cached token of each sequence, scored
+    page by page through the page table.  Contexts on both sides of the 4096-token limit of the fused kernel; a
+    sequence whose eligible pages all fit the recall budget must get the same set from the hierarchy."""
+    cfg = SMALL_DEC.replace(name="dec_flat_" + key_dtype, hi_enable=False, key_dtype=key_dtype, M=64, ctx_lo=1100, ctx_hi=9000, seed=23)
+    wl = DecodeWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.step()
+    assert wl.ctx.status() == 0
+    m = pu.check_decode(wl, range(cfg.batch))
+    print(cfg.name, m.summary())
+    m.assert_ok(pu.TOL_FP8 if key_dtype == "e4m3" else pu.TOL_BF16)
+    hier = DecodeWorkload(cfg.replace(hi_enable=True), cuda_device)
+    hier.prepare()
+    hier.index()
+    assert hier.ctx.status() == 0
+    ctx = wl.ctx_len.cpu().numpy()
+    short = [b for b in range(cfg.batch) if (int(ctx[b]) - 1 - cfg.W) // cfg.P - cfg.S // cfg.P + 1 <= cfg.M]
+    assert short, "the test wants at least one sequence whose eligible pages fit the budget"
+    for b in short:
+        assert torch.equal(hier.sparse_idx[b], wl.sparse_idx[b])
+
+
+def test_paged_fine_stage_on_tcgen05_gives_the_same_selection(cuda_device):
+    """LSA_TUNE_FINE_PAGED_TC = 1: page lists, token scores of the listed pages on tcgen05, top-K.  Same arithmetic per
+    token up to the summation order of the heads, so the sets are compared with the oracle, and with the default path."""
+    cfg = SMALL_DEC
+    ref_wl = DecodeWorkload(cfg, cuda_device)
+    ref_wl.prepare()
+    ref_wl.step()
+    wl = DecodeWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.ctx.tune(5, 1)
+    wl.step()
+    assert wl.ctx.status() == 0
+    m = pu.check_decode(wl, range(cfg.batch))
+    print(cfg.name, m.summary())
+    m.assert_ok(pu.TOL_FP8)
+    same = sum(int(torch.equal(wl.sparse_idx[b], ref_wl.sparse_idx[b])) for b in range(cfg.batch))
+    assert same >= cfg.batch - 1       # a near-tie may flip one token of one sequence
+
+
 @pytest.mark.parametrize("n_split", [1, 2, 4, 8])
 def test_paged_decode_row_splits(cuda_device, n_split):
     """Each row-split count of the decode attention (blocks of one thread-block cluster merging their parts by
