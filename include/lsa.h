@@ -112,6 +112,14 @@ LSA_API int lsa_workspace_bytes(const lsa_params* p, int64_t n_query, int64_t n_
 /* Waits for the stream, then writes the device status word (host int; 0 = fine, LSA_ERR_TIMEOUT...)
  * and clears it. */
 LSA_API int lsa_status(lsa_ctx* ctx, int* device_status);
+
+/* Failure-detection self-test.  Launches one small block whose threads wait, as every tcgen05 kernel of the library
+ * waits, on a shared-memory barrier - but one that nobody ever arrives on.  Thread 0 gives up after `budget_cycles`
+ * SM clock cycles (at most 2^31, about a second) and records LSA_ERR_TIMEOUT in the context's status word; the other
+ * threads see the word and stop; the kernel ends normally.  Afterwards lsa_status reports LSA_ERR_TIMEOUT (and
+ * clears it) and the context serves further calls as before.  Nothing faults, traps or hangs.
+ * (The paper has no counterpart: this exercises the library's own handling of a wait that runs out.) */
+LSA_API int lsa_selftest_wait(lsa_ctx* ctx, int64_t budget_cycles);
 LSA_API const char* lsa_strerror(int err);
 /* Text of the last CUDA error seen by this context (host string owned by the library). */
 LSA_API const char* lsa_last_cuda_error(lsa_ctx* ctx);

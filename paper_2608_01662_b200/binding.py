@@ -45,6 +45,7 @@ EXPORTS = {
     "lsa_last_cuda_error": (c_char_p, [c_void_p]),
     "lsa_launch_count": (c_int64, [c_void_p]),
     "lsa_tune": (c_int, [c_void_p, c_int, c_int]),
+    "lsa_selftest_wait": (c_int, [c_void_p, c_int64]),
     "lsa_profile_enable": (c_int, [c_void_p, c_int]),
     "lsa_profile_read": (c_int, [c_void_p, POINTER(ctypes.c_double), POINTER(c_int64)]),
     "lsa_block_means": (c_int, [c_void_p, POINTER(LsaParams), c_void_p, c_void_p, c_int64, c_void_p, c_int64,
@@ -188,6 +189,10 @@ class Context:
 
     def launch_count(self) -> int:
         return lib().lsa_launch_count(self.h)
+
+    def selftest_wait(self, budget_cycles: int):
+        """lsa_selftest_wait: a bounded device-side wait that runs out (status() then returns LSA_ERR_TIMEOUT)."""
+        self._chk(lib().lsa_selftest_wait(self.h, budget_cycles), "lsa_selftest_wait")
 
     def tune(self, knob: int, value: int):
         self._chk(lib().lsa_tune(self.h, knob, value), "lsa_tune")

@@ -436,6 +436,13 @@ int lsa_status(lsa_ctx* c, int* device_status) {
   return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
 }
 
+int lsa_selftest_wait(lsa_ctx* c, int64_t budget_cycles) {
+  if (c == nullptr || budget_cycles < 0 || budget_cycles > (1ll << 31)) return LSA_ERR_ARG;
+  if (c->ws == nullptr) return LSA_ERR_WORKSPACE;
+  const cudaError_t e = lsa::launch_selftest_wait(status_word(c), budget_cycles, nullptr, c->stream, &c->launches);
+  return e == cudaSuccess ? LSA_OK : cuda_fail(c, e);
+}
+
 const char* lsa_strerror(int err) {
   switch (err) {
     case LSA_OK: return "ok";

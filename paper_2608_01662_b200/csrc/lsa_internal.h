@@ -149,6 +149,10 @@ struct MergeArgs {
 };
 cudaError_t launch_merge_parts(const MergeArgs& a, cudaStream_t st, int64_t* n_launch);
 
+// One block waits on an mbarrier nobody arrives on, for at most budget_cycles (thread 0) before the status word gets
+// the time-out code; *waited_ok (optional, zeroed by the caller) counts threads whose wait claimed success.
+cudaError_t launch_selftest_wait(int* status, long long budget_cycles, int* waited_ok, cudaStream_t st, int64_t* n_launch);
+
 bool index_shape_supported(int HI, int DI);
 bool attn_shape_supported(int H, int DQK, int DV);
 

@@ -55,7 +55,8 @@ constexpr long long kWaitCycles = 1ll << 31;
 __device__ __forceinline__ bool status_raised(const int* status) {
   return status != nullptr && *reinterpret_cast<const volatile int*>(status) != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+// The wait with its cycle budget as an argument (the production kernels use kWaitCycles; the self-test a short one).
+__device__ __forceinline__ bool mbar_wait_budget(uint32_t bar, uint32_t parity, int* status, long long budget) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
 #pragma unroll 1
@@ -64,12 +65,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* st
     if ((i & 255u) == 0) {
       // once any wait anywhere in the grid has given up, everybody stops waiting
       if (status_raised(status)) return false;
-      if (clock64() - t0 > kWaitCycles) {
+      if (clock64() - t0 > budget) {
         report_status(status, kDevTimeout);
         return false;
       }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
+  return mbar_wait_budget(bar, parity, status, kWaitCycles);
 }
 
 // ---- TMA -------------------------------------------------------------------------------------------

@@ -192,6 +192,25 @@ def test_attention_issue_order_and_completion_barrier_give_the_same_bits(cuda_de
     assert torch.equal(wl.out[0], fast_out) and torch.equal(wl.lse[0], fast_lse)
 
 
+def test_group_of_three_layers(cuda_device):
+    """R = 3, the paper's MTP-style group (Sec. 3.2): one index set, three attention layers with their own caches."""
+    cfg = SMALL_MLA.replace(name="mla_r3", R=3, seed=29)
+    wl = PrefillWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.step()
+    assert wl.ctx.status() == 0
+    m = pu.check_prefill(wl, pu.boundary_queries(cfg, 0, cfg.L, 40, seed=6))
+    print(cfg.name, m.summary())
+    m.assert_ok(pu.TOL_BF16)
+    assert not torch.equal(wl.out[0], wl.out[2])
+    dcfg = SMALL_DEC.replace(name="dec_r3", R=3, seed=30)
+    dw = DecodeWorkload(dcfg, cuda_device)
+    dw.prepare()
+    dw.step()
+    assert dw.ctx.status() == 0
+    pu.check_decode(dw, range(dcfg.batch)).assert_ok(pu.TOL_FP8)
+
+
 def test_runs_are_deterministic(cuda_device):
     wl = PrefillWorkload(SMALL_FP8, cuda_device)
     wl.prepare()
