@@ -22,7 +22,7 @@ import json
 import torch
 
 from .configs import CONFIGS
-from .workload import PrefillWorkload
+from .workload import DecodeWorkload, PrefillWorkload
 
 
 def _index(cfg, dev, q_pos0, n_query, steps=3):
@@ -52,8 +52,35 @@ def _recall(idx_a, n_a, idx_ref, n_ref):
     return float(rec.mean())
 
 
+def decode_table(dev, batch=4, steps=20):
+    """Decode cost against context length (the counterpart of the paper's Table 1): `batch` sequences of equal length,
+    one query token each, one attention layer; indexer kernels and the attention kernel timed by the library's event
+    pairs, for the hierarchical indexer and for the flat one (hi_enable = 0)."""
+    for ctx in (4096, 16384, 65536, 262144, 1048576):
+        for flat in (False, True):
+            cfg = CONFIGS["cfg4"].replace(name="decode_table", batch=batch, ctx_lo=ctx, ctx_hi=ctx, R=1, hi_enable=not flat)
+            wl = DecodeWorkload(cfg, dev, with_lse=False)
+            wl.prepare()
+            for _ in range(3):
+                wl.step()
+            wl.ctx.profile_enable(True)
+            for _ in range(steps):
+                wl.step()
+            prof = wl.ctx.profile_read()
+            wl.ctx.profile_enable(False)
+            assert wl.ctx.status() == 0
+            us = {k: round(v[0] / steps * 1e3, 1) for k, v in prof.items() if v[1] > 0}
+            indexer = round(sum(v for k, v in us.items() if k != "sparse_attn"), 1)
+            print(json.dumps(dict(context=ctx, batch=batch, indexer="flat" if flat else "hierarchical", kernels_us=us,
+                                  indexer_us=indexer, attention_us=us.get("sparse_attn", 0.0))), flush=True)
+            del wl
+            torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--decode-table", action="store_true",
+                    help="decode indexer and attention time against context length, hierarchical and flat, instead of the sweep")
     ap.add_argument("--seq-len", type=int, default=32768)
     ap.add_argument("--q-tail", type=int, default=2048)
     ap.add_argument("--boost", default="0.02,4", help="share of boosted keys and their gain; '0,1' = none")
@@ -62,6 +89,9 @@ def main():
     ap.add_argument("--device", default="cuda:0")
     args = ap.parse_args()
     dev = torch.device(args.device)
+    if args.decode_table:
+        decode_table(dev)
+        return
     bp, bg = (float(x) for x in args.boost.split(","))
     base = CONFIGS["cfg3"].replace(name="sweep", L=args.seq_len, boost_prob=bp, boost_gain=bg,
                                    segment_corr=args.segment_corr)
