@@ -511,7 +511,7 @@ def run_e2e(args, cfg, wl, dev):
     d2h = sum(o.numel() * 2 for o in out_h)
 
     def step():
-        wl.ctx.layer_group_host(q_idx_h, w_h, wl.keys["k"], wl.keys.get("scale"), wl.kmean, n, wl.n_key, q_h, wl.k,
+        wl.ctx.layer_group_host(q_idx_h, w_h, wl.keys["k"], wl.keys.get("scale"), wl.kmean, wl.q_pos0, n, wl.n_key, q_h, wl.k,
                                 wl.v, out_h, sq, stage)
     step()
     torch.cuda.synchronize()

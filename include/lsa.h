@@ -337,15 +337,15 @@ LSA_API int lsa_layer_group(lsa_ctx* ctx, const lsa_params* p, const void* q_idx
                     int32_t* sparse_idx, int32_t* n_sparse);
 
 /* Same group, prefill only, with the per-query tensors in HOST memory (pinned for full speed):
- * q_idx_host, w_host, q_host[r], out_host[r] are host pointers; caches (k_idx, k_scale, kmean, k[r], v[r])
+ * q_idx_host, w_host, q_host[r], out_host[r] are host pointers (row i = the query at position q_pos0 + i); caches (k_idx, k_scale, kmean, k[r], v[r])
  * stay device-resident.  The queries are processed in passes of `stage_queries`; each pass copies its
  * slice of q_idx, w and q[r] to the device staging buffers, runs the group on it and copies out[r] back;
  * copies in, kernels and copies out of consecutive passes overlap on two internal streams (the copy-in of pass i+2
  * starts as soon as the kernels of pass i have read their inputs).
  * stage[2] are two caller-owned device staging areas of lsa_host_stage_bytes() bytes each. */
 LSA_API int lsa_layer_group_host(lsa_ctx* ctx, const lsa_params* p, const void* q_idx_host, const float* w_host,
-                         const void* k_idx, const float* k_scale, const void* kmean, int64_t n_query,
-                         int64_t n_key, const void* const* q_host, const void* const* k,
+                         const void* k_idx, const float* k_scale, const void* kmean, int64_t q_pos0,
+                         int64_t n_query, int64_t n_key, const void* const* q_host, const void* const* k,
                          const void* const* v, int64_t ld_k, int64_t ld_v, void* const* out_host,
                          int64_t stage_queries, void* const* stage, size_t stage_bytes);
 LSA_API int lsa_host_stage_bytes(const lsa_params* p, int64_t stage_queries, size_t* bytes);

@@ -71,7 +71,7 @@ EXPORTS = {
                                 POINTER(c_void_p), POINTER(c_void_p), c_int64, c_int64, POINTER(c_void_p),
                                 POINTER(c_void_p), c_void_p, c_void_p]),
     "lsa_layer_group_host": (c_int, [c_void_p, POINTER(LsaParams), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
-                                     c_int64, c_int64, POINTER(c_void_p), POINTER(c_void_p), POINTER(c_void_p),
+                                     c_int64, c_int64, c_int64, POINTER(c_void_p), POINTER(c_void_p), POINTER(c_void_p),
                                      c_int64, c_int64, POINTER(c_void_p), c_int64, POINTER(c_void_p), c_size_t]),
     "lsa_host_stage_bytes": (c_int, [POINTER(LsaParams), c_int64, POINTER(c_size_t)]),
 }
@@ -264,9 +264,9 @@ class Context:
                                         batch, _parr(q), _parr(k), _parr(v), k[0].stride(0), v[0].stride(0),
                                         _parr(out), _parr(lse), _p(sparse_idx), _p(n_sparse)), "lsa_layer_group")
 
-    def layer_group_host(self, q_idx_host, w_host, k_idx, k_scale, kmean, n_query, n_key, q_host, k, v, out_host,
+    def layer_group_host(self, q_idx_host, w_host, k_idx, k_scale, kmean, q_pos0, n_query, n_key, q_host, k, v, out_host,
                          stage_queries, stage):
         self._chk(lib().lsa_layer_group_host(self.h, ctypes.byref(self.params), _p(q_idx_host), _p(w_host), _p(k_idx),
-                                             _p(k_scale), _p(kmean), n_query, n_key, _parr(q_host), _parr(k),
+                                             _p(k_scale), _p(kmean), q_pos0, n_query, n_key, _parr(q_host), _parr(k),
                                              _parr(v), k[0].stride(0), v[0].stride(0), _parr(out_host), stage_queries,
                                              _parr(stage), stage[0].numel()), "lsa_layer_group_host")

@@ -694,15 +694,15 @@ int lsa_host_stage_bytes(const lsa_params* p, int64_t sq, size_t* bytes) {
 }
 
 int lsa_layer_group_host(lsa_ctx* c, const lsa_params* p, const void* q_idx_host, const float* w_host,
-                         const void* k_idx, const float* k_scale, const void* kmean, int64_t n_query, int64_t n_key,
-                         const void* const* q_host, const void* const* k, const void* const* v, int64_t ld_k,
+                         const void* k_idx, const float* k_scale, const void* kmean, int64_t q_pos0, int64_t n_query,
+                         int64_t n_key, const void* const* q_host, const void* const* k, const void* const* v, int64_t ld_k,
                          int64_t ld_v, void* const* out_host, int64_t sq, void* const* stage, size_t stage_bytes) {
   if (c == nullptr) return LSA_ERR_ARG;
   size_t need = 0;
   int r = lsa_host_stage_bytes(p, sq, &need);
   if (r != LSA_OK) return r;
   if (stage == nullptr || stage[0] == nullptr || stage[1] == nullptr || stage_bytes < need) return LSA_ERR_WORKSPACE;
-  if (q_idx_host == nullptr || w_host == nullptr || q_host == nullptr || out_host == nullptr || n_query < 0) return LSA_ERR_ARG;
+  if (q_idx_host == nullptr || w_host == nullptr || q_host == nullptr || out_host == nullptr || n_query < 0 || q_pos0 < 0) return LSA_ERR_ARG;
   const int R = p->n_layers;
   if (R > 16) return LSA_ERR_SHAPE;
   const size_t b_qi = static_cast<size_t>(p->n_heads_idx) * p->d_idx * 2, b_w = static_cast<size_t>(p->n_heads_idx) * 4;
@@ -735,7 +735,7 @@ int lsa_layer_group_host(lsa_ctx* c, const lsa_params* p, const void* q_idx_host
     if (e == cudaSuccess) e = cudaStreamWaitEvent(c->stream, c->ev_in[s], 0);
     if (e == cudaSuccess && i >= 2) e = cudaStreamWaitEvent(c->stream, c->ev_out[s], 0);
     if (e != cudaSuccess) break;
-    r = lsa_layer_group(c, p, d_qi, reinterpret_cast<const float*>(d_w), k_idx, k_scale, kmean, q0, n, n_key, nullptr,
+    r = lsa_layer_group(c, p, d_qi, reinterpret_cast<const float*>(d_w), k_idx, k_scale, kmean, q_pos0 + q0, n, n_key, nullptr,
                         0, nullptr, 1, d_q, k, v, ld_k, ld_v, d_o, nullptr, d_idx, d_n);
     if (r != LSA_OK) return r;
     e = cudaEventRecord(c->ev_done[s], c->stream);

@@ -390,12 +390,13 @@ def test_large_recall_budget(cuda_device, base):
 
 
 # ---------------------------------------------------------------- host-buffer entry point
-def test_layer_group_from_host_buffers_equals_device_run(cuda_device):
+@pytest.mark.parametrize("q_pos0", [0, 2100])
+def test_layer_group_from_host_buffers_equals_device_run(cuda_device, q_pos0):
     """lsa_layer_group_host (queries in pinned host memory, staged through the device in passes, copies overlapping
     kernels) returns the bytes of the device-resident run, for a pass size that leaves a ragged last pass and needs
-    every staging buffer several times."""
+    every staging buffer several times; also for a chunk of queries that starts inside the sequence."""
     cfg = SMALL_FP8.replace(name="host_small", L=5000, R=2, seed=23)
-    wl = PrefillWorkload(cfg, cuda_device, with_lse=False)
+    wl = PrefillWorkload(cfg, cuda_device, with_lse=False, q_pos0=q_pos0, n_query=cfg.L - q_pos0)
     wl.prepare()
     wl.step()
     torch.cuda.synchronize()
@@ -405,7 +406,7 @@ def test_layer_group_from_host_buffers_equals_device_run(cuda_device):
     q_h = [q.cpu().pin_memory() for q in wl.q]
     out_h = [torch.zeros(o.shape, dtype=o.dtype).pin_memory() for o in wl.out]
     for _ in range(2):   # twice: the second call reuses events and staging areas left by the first
-        wl.ctx.layer_group_host(q_idx_h, w_h, wl.keys["k"], wl.keys.get("scale"), wl.kmean, wl.n_query, wl.n_key, q_h,
+        wl.ctx.layer_group_host(q_idx_h, w_h, wl.keys["k"], wl.keys.get("scale"), wl.kmean, wl.q_pos0, wl.n_query, wl.n_key, q_h,
                                 wl.k, wl.v, out_h, sq, stage)
         torch.cuda.synchronize()
         assert wl.ctx.status() == 0
