@@ -5,13 +5,16 @@
 // rows of every MMA; the attended cache rows stream through a ring of three 64-key shared tiles:
 //
 //   warps 8-11  gather: rows [window | sink | sparse] (or the caller's row list) -> 128B-swizzled K-major tiles, up to
-//               three tiles in flight.  Scattered rows come by TMA gather (cp.async.bulk.tensor ... tile::gather4: four
-//               cache rows x one 64-dim column block per instruction, 144 instructions per tile spread over the 128
-//               gather threads, completion counted in bytes on the tile's mbarrier), tiles of 64 consecutive window
-//               rows as nine plain TMA boxes; caches TMA cannot address (unaligned base or pitch) fall back to
-//               coalesced 16-byte cp.async.
+//               three tiles in flight.  Scattered rows are copied with coalesced 16-byte cp.async (a row whole, by one
+//               warp, in back-to-back instructions), each tile handed over through an mbarrier when it has landed;
+//               tiles of 64 consecutive window rows come as nine TMA boxes instead.  A TMA gather of the scattered
+//               rows (cp.async.bulk.tensor ... tile::gather4: four cache rows x one 64-dim column block = 512 bytes
+//               per instruction, 144 per tile) is built in as well (AttnArgs::gather4) and measured 1.3 x slower: the
+//               TMA unit takes about 26 cycles per such instruction.
 //               Q arrives the same way: its rope dims (512-575) stay in shared memory as an MMA operand, dims 0-511
 //               are staged in the last tile buffer for the softmax warps
+//               With two P V issuers (prefill) warps 6-7 have no MMAs to issue and copy rows as a fifth and sixth gather
+//               warp (11 or 10 rows of a tile each instead of 16: measured 1 % faster).
 //   warps 4-7   one thread each issues tcgen05.mma.  Back-to-back MMAs into one accumulator run far below the pipe's
 //               rate at these small shapes, so each product is cut into independent accumulation chains:
 //                 S = Q K^T   issuers 0 and 1: dims 256x .. 256x+255 with Q from tensor memory (16 steps of M64 N64
@@ -22,7 +25,8 @@
 //                             2 (prefill)  issuer x: value dims 256x .. 256x+255 (M64 N256 K16 x 4 per tile), P from lane
 //                                          half x, O in lane half x: an issuer owns everything in its lane half
 //                             4 (decode)   issuer x: value dims 128x .. 128x+127 (M64 N128 K16 x 4 per tile)
-//               A thread takes whichever of "next Q K^T" / "next P V" is ready.  The S buffer of tile i+1 still holds
+//               A thread takes whichever of "next P V" / "next Q K^T" is ready, P V first (its completion frees a key
+//               buffer, and the refill of that buffer is the longest latency of the ring).  The S buffer of tile i+1 still holds
 //               P of tile i-1 in its first columns.  With four issuers Q K^T(i+1) waits for the completion barrier of
 //               P V(i-1); the P V issuers that do no Q K^T release a key buffer as early as possible, which is what a
 //               decode step, waiting on HBM gathers, needs.  With two issuers the P V that reads those columns and the
@@ -238,7 +242,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
     tc::mbar_init(smem_u32(&sm.q_full), q_tma ? 1 : 32 * kLoadWarps);
     tc::mbar_init(smem_u32(&sm.q_tmem), kSoftmaxWarps);
     for (int b = 0; b < kKBufs; ++b) {
-      tc::mbar_init(smem_u32(&sm.k_full[b]), 32 * kLoadWarps);
+      tc::mbar_init(smem_u32(&sm.k_full[b]), 32 * (kLoadWarps + (kPv == 2 ? 2 : 0)));
       tc::mbar_init(smem_u32(&sm.k_empty[b]), n_pv);
     }
     for (int b = 0; b < 2; ++b) {
@@ -267,7 +271,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
   // gather warps read them and put the first two key tiles in flight while that kernel drains, and wait only before
   // they request Q; every other thread waits here.
   const bool early_rows = kRows && p.rows_stable != 0 && q_tma != 0;   // block-uniform
-  const bool gather_warp = warp >= kSoftmaxWarps + kMmaWarps;
+  const bool gather_warp = warp >= kSoftmaxWarps + kMmaWarps - (kPv == 2 ? 2 : 0);
   auto dependency_wait = [&]() {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -323,11 +327,14 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
   int n_tiles = max(0, min(tiles_all, tile_begin + tiles_per) - tile_begin);
   if (dead) n_tiles = 0;   // the peers of this cluster still expect this block at the cluster barrier
 
-  if (warp >= kSoftmaxWarps + kMmaWarps) {
+  // With two P V issuers the other two MMA warps have nothing to issue and gather as well.
+  constexpr int kGw = kLoadWarps + (kPv == 2 ? 2 : 0);
+  if (warp >= kSoftmaxWarps + kMmaWarps - (kGw - kLoadWarps)) {
     // ================= gather warps =================
-    const int gw = warp - (kSoftmaxWarps + kMmaWarps);
-    const int lt = gw * 32 + lane;   // 0..127
-    {
+    // gw 0..3: warps 8-11 (they also fetch Q and issue the TMA loads); gw 4..5: warps 6-7
+    const int gw = warp >= kSoftmaxWarps + kMmaWarps ? warp - (kSoftmaxWarps + kMmaWarps) : kLoadWarps + warp - (kSoftmaxWarps + kMmaWarps - 2);
+    const int lt = gw * 32 + lane;
+    if (gw < kLoadWarps) {
       // Q of this query: the rope part (dims 512-575) stays in shared memory as an MMA operand; dims 0-511 are staged
       // in the last key buffer for the softmax warps, which move them to tensor memory.  As TMA boxes they complete
       // q_full by themselves; as cp.async copies they form the first group, handed over with the first key tile.
@@ -351,7 +358,9 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
     // and the 72 16-byte chunks of that row are copied by consecutive lanes (coalesced 512-byte requests: a row is
     // fetched whole, by one warp, in back-to-back instructions.  Spreading the chunks of a tile evenly over the warps,
     // every instruction full, was measured at 1.3 x the time, in prefill and in decode).
-    constexpr int kRowsPerWarp = kTileKeys / kLoadWarps;
+    // rows of a tile a warp copies: 16 each with four warps; 11, 11, 11, 11, 10, 10 with six
+    const int row_first = kGw == 4 ? 16 * gw : (gw <= 4 ? 11 * gw : 54);
+    const int n_my_rows = kGw == 4 ? 16 : (gw < 4 ? 11 : 10);
     const uint8_t* kg = reinterpret_cast<const uint8_t*>(k_ptr);
     auto tile_by_tma = [&](int i) -> bool {   // block-uniform
       return !kRows && k_tma && (tile_begin + i + 1) * kTileKeys <= n_win;
@@ -361,11 +370,11 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
     const bool g4 = k_g4 != 0;   // block-uniform
     const int quad = (lt >> 3) & 15, atom0 = lt & 7;
     auto my_key_row = [&](int i) -> int32_t {
-      return (!g4 && i < n_tiles && lane < kRowsPerWarp && !tile_by_tma(i)) ? row_of((tile_begin + i) * kTileKeys + kRowsPerWarp * gw + lane) : -1;
+      return (!g4 && i < n_tiles && lane < n_my_rows && !tile_by_tma(i)) ? row_of((tile_begin + i) * kTileKeys + row_first + lane) : -1;
     };
     auto my_quad_rows = [&](int i) -> int4 {
       int4 r = make_int4(0, 0, 0, 0);
-      if (g4 && i < n_tiles && !tile_by_tma(i)) {
+      if (g4 && gw < kLoadWarps && i < n_tiles && !tile_by_tma(i)) {
         const int i0 = (tile_begin + i) * kTileKeys + 4 * quad;
         if (kRows && i0 + 3 < n_tot && ((reinterpret_cast<uintptr_t>(rows + i0) & 15u) == 0)) {
           r = *reinterpret_cast<const int4*>(rows + i0);
@@ -383,7 +392,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
     // Copies of up to three tiles are in flight: a tile is handed to the MMA issuers (k_full) when its cp.async group
     // has landed, which is looked at after the next tile's copies are issued, or at once when no buffer is free.
     int first_pend = 0, n_pend = 0;   // tiles first_pend .. first_pend + n_pend - 1 are issued but not handed over
-    bool q_handed = q_tma != 0;       // TMA completes q_full by itself
+    bool q_handed = q_tma != 0 || gw >= kLoadWarps;   // TMA completes q_full by itself; the extra warps fetch no Q
     auto hand_over_q = [&]() {        // call after a wait that covers the first group
       tc::fence_proxy_async();
       tc::mbar_arrive(smem_u32(&sm.q_full));
@@ -432,16 +441,17 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       } else if (g4) {
         // scattered rows: four rows x 64 dims per instruction, straight into their place in the swizzled tile
         if (lt == 0) tc::mbar_expect_tx_only(smem_u32(&sm.k_full[b]), kAtoms * kAtomBytes);
-        tc::tma_gather4_2d(smem_u32(sm.k[b][atom0]) + quad * 512, &g_map, atom0 * 64, my_rows4.x, my_rows4.y, my_rows4.z,
-                           my_rows4.w, smem_u32(&sm.k_full[b]));
-        if (atom0 == 0)
+        if (gw < kLoadWarps)
+          tc::tma_gather4_2d(smem_u32(sm.k[b][atom0]) + quad * 512, &g_map, atom0 * 64, my_rows4.x, my_rows4.y, my_rows4.z,
+                             my_rows4.w, smem_u32(&sm.k_full[b]));
+        if (gw < kLoadWarps && atom0 == 0)
           tc::tma_gather4_2d(smem_u32(sm.k[b][kAtoms - 1]) + quad * 512, &g_map, (kAtoms - 1) * 64, my_rows4.x, my_rows4.y,
                              my_rows4.z, my_rows4.w, smem_u32(&sm.k_full[b]));
       } else {
 #pragma unroll 4
-        for (int rr = 0; rr < kRowsPerWarp; ++rr) {
+        for (int rr = 0; rr < n_my_rows; ++rr) {
           const int32_t row = __shfl_sync(0xffffffffu, my_row, rr);
-          const int r = kRowsPerWarp * gw + rr;
+          const int r = row_first + rr;
           const uint8_t* src = kg + static_cast<int64_t>(row >= 0 ? row : 0) * p.ld_k * 2;
           const int nb = row >= 0 ? 16 : 0;
 #pragma unroll
