@@ -160,9 +160,11 @@ struct AttnTcSmem {
   alignas(16) float lse_peer[kH / 2];     // two-split launches: the peer's, for the heads this block finishes
 };
 constexpr int kPitchPart = kDV * 4 + 16;                  // staged fp32 row of a partial result, padded against bank conflicts
-// Two-split launches stage their rows unpadded, with the 16-byte chunks of row r XOR-swizzled by r % 8 (no bank
-// conflicts either way), so that the 16 rows a warp stages are one contiguous piece and leave as one bulk copy; the
-// peer's rows land behind the staged ones.
+// Two-split launches stage their rows in the order the softmax warps read them out of tensor memory: per warp (16
+// rows) four column steps, each [value-dim half][row][64 floats] = 8 KB, the 16-byte chunks of a row's 256-byte piece
+// XOR-swizzled by the row (no bank conflicts either way).  A step's 8 KB is contiguous, so the rows the peer finishes
+// leave step by step, one bulk copy each, while the rest is still being read out; the peer's rows land behind the
+// staged ones in the same layout.
 constexpr int kPairRowBytes = kDV * 4;
 constexpr int kRecvOffset = kH * kPairRowBytes;
 constexpr uint32_t kRecvBytes = (kH / 2) * kDV * 4 + (kH / 2) * 4;
@@ -747,9 +749,20 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       }
       if (hi == 0 && lse_ptr != nullptr) lse_ptr[static_cast<int64_t>(qi) * kH + row] = lse2 / kLog2eTc;
     } else {
-      // partial result of a split: normalised fp32 rows in the key buffers (padded against bank conflicts)
-      uint8_t* my_row = stage + row * (pair ? kPairRowBytes : kPitchPart);
-      const int sw = pair ? (row & 7) : 0;
+      // partial result of a split: normalised fp32 rows in the key buffers
+      const bool foreign = pair && row / (kH / 2) != split;   // warp-uniform: a warp stages 16 consecutive rows
+      const uint32_t peer = static_cast<uint32_t>(split ^ 1);
+      const int peer_row0 = (kH / 2) * (split ^ 1);
+      uint32_t bar_peer = 0, dst_peer = 0;
+      if (foreign) {
+        // into the peer's shared memory, once every thread of the peer has left its tile loop (first half of the
+        // cluster barrier: its key buffers, which receive the rows, are then out of use)
+        cluster_wait();
+        bar_peer = peer_smem(smem_u32(&sm.recv_full), peer);
+        dst_peer = peer_smem(smem_u32(stage + kRecvOffset + (16 * quarter - peer_row0) * kPairRowBytes), peer);
+      }
+      uint8_t* my_row = stage + row * kPitchPart;                        // (four or eight splits: padded rows)
+      uint8_t* my_warp = stage + 16 * quarter * kPairRowBytes;           // (two splits: this warp's 32 KB)
 #pragma unroll 1
       for (int c = 0; c < 256; c += 64) {
         uint32_t o[64];
@@ -760,11 +773,26 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
 #pragma unroll
           for (int j = 0; j < 64; ++j) o[j] = 0u;
         }
+        if (pair) {
+          uint8_t* piece = my_warp + (c / 64) * 8192 + hi * 4096 + r16 * 256;
 #pragma unroll
-        for (int j = 0; j < 16; ++j)   // 16-byte chunk hi * 64 + c / 4 + j of the row
-          *reinterpret_cast<float4*>(my_row + (((hi * 64 + c / 4 + j) ^ sw) << 4)) =
-              make_float4(__uint_as_float(o[4 * j]) * inv, __uint_as_float(o[4 * j + 1]) * inv,
-                          __uint_as_float(o[4 * j + 2]) * inv, __uint_as_float(o[4 * j + 3]) * inv);
+          for (int j = 0; j < 16; ++j)
+            *reinterpret_cast<float4*>(piece + ((j ^ r16) << 4)) =
+                make_float4(__uint_as_float(o[4 * j]) * inv, __uint_as_float(o[4 * j + 1]) * inv,
+                            __uint_as_float(o[4 * j + 2]) * inv, __uint_as_float(o[4 * j + 3]) * inv);
+          if (foreign) {
+            tc::fence_proxy_async();
+            __syncwarp();
+            if (lane == 0)
+              bulk_copy_to_peer(dst_peer + (c / 64) * 8192, smem_u32(my_warp + (c / 64) * 8192), 8192, bar_peer);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)   // 16-byte chunk hi * 64 + c / 4 + j of the row
+            *reinterpret_cast<float4*>(my_row + ((hi * 64 + c / 4 + j) << 4)) =
+                make_float4(__uint_as_float(o[4 * j]) * inv, __uint_as_float(o[4 * j + 1]) * inv,
+                            __uint_as_float(o[4 * j + 2]) * inv, __uint_as_float(o[4 * j + 3]) * inv);
+        }
       }
       if (hi == 0) {
         sm.lse_own[row] = lse2;
@@ -775,19 +803,12 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       tc::fence_proxy_async();
       __syncwarp();
       if (pair) {
-        // into the peer's shared memory, once every thread of the peer has left its tile loop (first half of the
-        // cluster barrier: its key buffers, which receive the rows, are then out of use)
-        cluster_wait();
-        const uint32_t peer = static_cast<uint32_t>(split ^ 1);
-        const int peer_row0 = (kH / 2) * (split ^ 1);
-        if (row / (kH / 2) != split) {   // warp-uniform: a warp stages 16 consecutive rows
-          const uint32_t bar = peer_smem(smem_u32(&sm.recv_full), peer);
-          if (lane == 0) {   // the warp's 16 rows are one piece of 32 KB; their log-sum-exps another of 64 bytes
-            bulk_copy_to_peer(peer_smem(smem_u32(stage + kRecvOffset + (16 * quarter - peer_row0) * kPairRowBytes), peer),
-                              smem_u32(stage + 16 * quarter * kPairRowBytes), 16 * kPairRowBytes, bar);
+        if (foreign) {
+          if (lane == 0)   // the log-sum-exps of the warp's 16 rows
             bulk_copy_to_peer(peer_smem(smem_u32(&sm.lse_peer[16 * quarter - peer_row0]), peer), smem_u32(&sm.lse_own[16 * quarter]),
-                              16 * 4, bar);
-          }
+                              16 * 4, bar_peer);
+        } else {
+          cluster_wait();   // (every thread passes the first half of the barrier once)
         }
       } else {
         const int rows_per = kH / p.n_split;
@@ -833,12 +854,15 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
         w_peer *= r_den;
         if (lane == 0 && lse_ptr != nullptr)
           lse_ptr[static_cast<int64_t>(qi) * kH + R] = den > 0.f ? (m + log2f(den)) / kLog2eTc : -INFINITY;
-        const uint8_t* a_row = stage + R * kPairRowBytes;
-        const uint8_t* b_row = stage + kRecvOffset + rl * kPairRowBytes;
+        // row R = row R % 16 of staging warp R / 16 (here and in the peer, whose warp 2 * split + rl / 16 sent it)
+        const uint8_t* a_warp = stage + (R >> 4) * (16 * kPairRowBytes);
+        const uint8_t* b_warp = stage + kRecvOffset + (rl >> 4) * (16 * kPairRowBytes);
+        const int r16m = R & 15;
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          const int ch = ((lane + 32 * u) ^ (R & 7)) << 4;   // the peer staged head R with the same swizzle
-          const float4 a = *reinterpret_cast<const float4*>(a_row + ch), b = *reinterpret_cast<const float4*>(b_row + ch);
+          const int chunk = lane + 32 * u;   // 16-byte chunk of the row: value-dim half chunk / 64, step (chunk % 64) / 16
+          const int ch = (chunk >> 6) * 4096 + ((chunk & 63) >> 4) * 8192 + r16m * 256 + (((chunk & 15) ^ r16m) << 4);
+          const float4 a = *reinterpret_cast<const float4*>(a_warp + ch), b = *reinterpret_cast<const float4*>(b_warp + ch);
           uint2 o;
           o.x = pack_bf16(w_own * a.x + w_peer * b.x, w_own * a.y + w_peer * b.y);
           o.y = pack_bf16(w_own * a.z + w_peer * b.z, w_own * a.w + w_peer * b.w);
