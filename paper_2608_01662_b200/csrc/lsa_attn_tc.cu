@@ -841,8 +841,12 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       // the peer's rows for this block's heads, and their log-sum-exps, are in shared memory when the byte count is met
       (void)tc::mbar_wait(smem_u32(&sm.recv_full), 0, p.status);
       if (tid == 0) LSA_TL(kTlClusterSync);
+      // Second use of the cluster barrier: a block may leave once the peer has everything it was sent (until then the
+      // copies still read this block's shared memory).  A thread arrives as soon as it has seen this block's own
+      // bytes complete and waits at the very end, by when the peer has normally long arrived.
+      cluster_arrive();
       __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(out_ptr) + (static_cast<int64_t>(qi) * kH + row0) * kDV;
-#pragma unroll 1
+#pragma unroll
       for (int rl = warp; rl < kH / 2; rl += kWarps) {   // a warp finishes a row: lane l the chunks l, l + 32, ...
         const int R = row0 + rl;
         const float l_own = sm.lse_own[R], l_peer = sm.lse_peer[rl];
@@ -870,10 +874,7 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
         }
       }
       if (tid == 0) LSA_TL(kTlMerged);
-      // second use of the cluster barrier: a block leaves only when the peer has everything it was sent (its own
-      // arrival follows its wait for those bytes), so no copy is ever in flight towards a block that has gone
-      cluster_arrive();
-      cluster_wait();
+      cluster_wait();   // (see the arrival above)
     } else {
       if (warp < kSoftmaxWarps) {   // the threads that sent rows wait until they are written (not only read out of shared memory)
         asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
