@@ -192,6 +192,29 @@ def test_attention_issue_order_and_completion_barrier_give_the_same_bits(cuda_de
     assert torch.equal(wl.out[0], fast_out) and torch.equal(wl.lse[0], fast_lse)
 
 
+def test_rows_gathered_by_tma_gather4_give_the_same_bits(cuda_device):
+    """LSA_TUNE_ATTN_GATHER = 1 fetches the scattered cache rows with tile::gather4 TMA copies instead of 16-byte
+    cp.async: the same bytes land in the same places of the key tile, so prefill and decode outputs are unchanged."""
+    cfg = SMALL_MLA.replace(R=1)
+    wl = PrefillWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.step()
+    out0, lse0 = wl.out[0].clone(), wl.lse[0].clone()
+    wl.ctx.tune(4, 1)                 # LSA_TUNE_ATTN_GATHER
+    wl.step()
+    assert wl.ctx.status() == 0
+    assert torch.equal(wl.out[0], out0) and torch.equal(wl.lse[0], lse0)
+    dw = DecodeWorkload(SMALL_DEC, cuda_device)
+    dw.prepare()
+    dw.step()
+    dec0 = [o.clone() for o in dw.out]
+    dw.ctx.tune(4, 1)
+    dw.step()
+    assert dw.ctx.status() == 0
+    for a, b in zip(dw.out, dec0):
+        assert torch.equal(a, b)
+
+
 def test_group_of_three_layers(cuda_device):
     """R = 3, the paper's MTP-style group (Sec. 3.2): one index set, three attention layers with their own caches."""
     cfg = SMALL_MLA.replace(name="mla_r3", R=3, seed=29)
