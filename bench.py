@@ -50,7 +50,7 @@ def parse_args():
     ap.add_argument("--attn-split", type=int, default=0, help="override LSA_TUNE_ATTN_SPLIT (decode row splits)")
     ap.add_argument("--attn-pv-wait", type=int, default=-1, help="override LSA_TUNE_ATTN_PV_WAIT (0 or 1)")
     ap.add_argument("--attn-gather", type=int, default=-1, help="override LSA_TUNE_ATTN_GATHER (0: cp.async rows, 1: TMA gather4)")
-    ap.add_argument("--fine-paged-tc", type=int, default=-1, help="override LSA_TUNE_FINE_PAGED_TC (0 or 1)")
+    ap.add_argument("--fine-paged-tc", type=int, default=-1, help="override LSA_TUNE_FINE_PAGED_TC (0, 1 or 2)")
     ap.add_argument("--coarse-groups", type=int, default=0, help="override LSA_TUNE_COARSE_GROUPS (1 or 2)")
     return ap.parse_args()
 

@@ -139,10 +139,12 @@ LSA_API int64_t lsa_launch_count(lsa_ctx* ctx);
  *                           copies; 1: TMA gather, four rows per cp.async.bulk.tensor tile::gather4 instruction (needs a
  *                           16-byte aligned cache whose row pitch is a multiple of 16 bytes, else the other path is
  *                           taken).  Same bits; the TMA path measured 1.3 x slower (512 bytes per instruction).
- *   LSA_TUNE_FINE_PAGED_TC  hierarchical indexer on paged caches, fine stage.  0 (default): page top-M and token scores in
- *                           one mma.sync kernel, several blocks per sequence; 1: page lists, then token scores of the
- *                           listed pages on tcgen05 (the kernel the flat paged indexer always uses), then the top-K.
- *                           Same selection; measured slower at 64 sequences (three launches of dependent phases). */
+ *   LSA_TUNE_FINE_PAGED_TC  hierarchical indexer on paged caches, fine stage (64-head indexer, 64-token pages; other
+ *                           shapes always take form 2).  0 (default): one kernel, a thread-block cluster per sequence:
+ *                           page top-M, token scores of the kept pages on tcgen05, top-K and cache rows; 1: the same
+ *                           steps as three kernels (page lists, the scoring kernel the flat paged indexer uses,
+ *                           top-K); 2: page top-M and token scores in one mma.sync kernel, several blocks per
+ *                           sequence, then a top-K kernel.  Same selection.  cfg4: 39 / 72 / 58 us per decode step. */
 enum { LSA_TUNE_COARSE_GROUPS = 0, LSA_TUNE_ATTN_TC, LSA_TUNE_ATTN_SPLIT, LSA_TUNE_ATTN_PV_WAIT, LSA_TUNE_ATTN_GATHER,
        LSA_TUNE_FINE_PAGED_TC, LSA_TUNE_COUNT };
 LSA_API int lsa_tune(lsa_ctx* ctx, int knob, int value);

@@ -10,7 +10,7 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "liblsa.so")
 SOURCES = ["lsa_api.cu", "lsa_index.cu", "lsa_attn.cu", "lsa_static.cu", "lsa_coarse_tc.cu", "lsa_attn_tc.cu", "lsa_fine_tc.cu",
-           "lsa_coarse_paged_tc.cu", "lsa_fine_big_tc.cu", "lsa_scores_paged_tc.cu", "lsa_selftest.cu"]
+           "lsa_coarse_paged_tc.cu", "lsa_fine_big_tc.cu", "lsa_scores_paged_tc.cu", "lsa_fine_paged_tc.cu", "lsa_selftest.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

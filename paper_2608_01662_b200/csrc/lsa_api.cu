@@ -226,7 +226,10 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
     a.sm_count = c->sm_count;
     const bool paged_tc = p->paged && lsa::paged_scores_tc_supported(a);   // token scores of cache pages on tcgen05
     if (flat && p->paged && !paged_tc) return LSA_ERR_SHAPE;   // the flat indexer over long paged caches needs that kernel
-    if (paged_tc && (flat || c->tune[LSA_TUNE_FINE_PAGED_TC])) {
+    if (p->paged && !flat && c->tune[LSA_TUNE_FINE_PAGED_TC] == 0 && lsa::fine_paged_tc_supported(a)) {
+      a.fine_cluster = 1;
+      a.fine_parts = 2;   // (the kernel writes the cache rows itself)
+    } else if (paged_tc && (flat || c->tune[LSA_TUNE_FINE_PAGED_TC] == 1)) {
       a.fine_paged_tc = 1;
       a.fine_parts = 2;   // (marks the split path: the top-K kernel writes the cache rows itself)
       a.fine_keys = reinterpret_cast<uint32_t*>(c->ws + l.fine_keys);
@@ -464,7 +467,7 @@ int lsa_tune(lsa_ctx* c, int knob, int value) {
   if (knob == LSA_TUNE_ATTN_SPLIT && (value < 0 || value > kMaxSplit)) return LSA_ERR_ARG;
   if (knob == LSA_TUNE_ATTN_PV_WAIT && value != 0 && value != 1) return LSA_ERR_ARG;
   if (knob == LSA_TUNE_ATTN_GATHER && value != 0 && value != 1) return LSA_ERR_ARG;
-  if (knob == LSA_TUNE_FINE_PAGED_TC && value != 0 && value != 1) return LSA_ERR_ARG;
+  if (knob == LSA_TUNE_FINE_PAGED_TC && (value < 0 || value > 2)) return LSA_ERR_ARG;
   c->tune[knob] = value;
   return LSA_OK;
 }

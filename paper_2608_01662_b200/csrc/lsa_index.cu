@@ -11,6 +11,7 @@
 // thread quad and one number per key leaves the tile.
 #include "lsa_internal.h"
 #include "lsa_select.cuh"
+#include "lsa_rows.cuh"
 
 #ifdef LSA_TIMELINE
 // Debug build only: SM-clock stamps of the fine kernel's phases per block, read back with lsa_debug_timeline_fine.
@@ -347,68 +348,6 @@ __global__ void __launch_bounds__(kThreads, 2) coarse_score_paged_kernel(IndexAr
 // ------------------------------------------------------------------------------------------------
 // a2-a4: per query: top-M pages, fine scores on their tokens, top-K_sparse.
 // ------------------------------------------------------------------------------------------------
-// a5 for one query: cache rows [sink run | sparse ascending | window run] (paged: through the page table), padded
-// with -1 to S + Ksp + W entries.  `sparse` may be global memory this block has just written (after a barrier).
-// Returns this thread's count of run starts (a row that does not follow its predecessor).
-struct RowMap {   // position i of [sink | sparse | window] -> cache row
-  int n_sink, n_sp, paged, kv_shift, kv_mask;
-  int64_t win0;
-  const int32_t* sparse;
-  const int32_t* pt;
-  __device__ __forceinline__ int32_t operator()(int i) const {
-    int64_t pos;
-    if (i < n_sink) pos = i;
-    else if (i < n_sink + n_sp) pos = sparse[i - n_sink];
-    else pos = win0 + (i - n_sink - n_sp);
-    return static_cast<int32_t>(paged ? (static_cast<int64_t>(pt[pos >> kv_shift]) << kv_shift) + (pos & kv_mask) : pos);
-  }
-};
-
-template <int THREADS>
-__device__ __forceinline__ int emit_rows(int tid, int S, int W, int Ksp, int paged, int kv_page, const int32_t* sparse,
-                                         int n_sp, int64_t t, const int32_t* pt, int32_t* out, bool count_runs) {
-  RowMap row_of;
-  row_of.n_sink = static_cast<int>(min64(S, t + 1));
-  row_of.n_sp = n_sp;
-  row_of.paged = paged;
-  row_of.kv_shift = paged ? 31 - __clz(kv_page) : 0;   // kv_page is a power of two
-  row_of.kv_mask = kv_page - 1;
-  row_of.win0 = max64(S, t - W + 1);
-  row_of.sparse = sparse;
-  row_of.pt = pt;
-  const int n_win = static_cast<int>(max64(0, t - row_of.win0 + 1));
-  const int n_tot = row_of.n_sink + n_sp + n_win;
-  const int ld = S + Ksp + W;
-  int breaks = 0;
-#pragma unroll 4
-  for (int i = tid; i < ld; i += THREADS) {
-    int32_t r = -1;
-    if (i < n_tot) {
-      r = row_of(i);
-      if (count_runs && (i == 0 || row_of(i - 1) + 1 != r)) ++breaks;
-    }
-    out[i] = r;
-  }
-  return breaks;
-}
-
-// Fused a5 at the end of the indexer (paged caches, when the caller asked for it): the rows of query qi from the
-// sparse list this block has just written.  In the indexer a cache page is a selection page (kv_page = P).
-template <int THREADS>
-__device__ __forceinline__ void emit_rows_of_query(int32_t* rows_out, int32_t* n_rows_out, const int32_t* sparse_idx,
-                                                   const int32_t* page_table, int64_t pt_stride, int64_t t, int S, int W,
-                                                   int Ksp, int paged, int P, int qi, int tid, int n_sel) {
-  if (rows_out == nullptr) return;
-  const int ld = S + Ksp + W;
-  emit_rows<THREADS>(tid, S, W, Ksp, paged, P, sparse_idx + static_cast<int64_t>(qi) * Ksp, n_sel, t,
-                     paged ? page_table + qi * pt_stride : nullptr, rows_out + static_cast<int64_t>(qi) * ld, false);
-  if (tid == 0) {
-    const int n_sink = static_cast<int>(min64(S, t + 1));
-    const int64_t win0 = max64(S, t - W + 1);
-    n_rows_out[qi] = n_sink + n_sel + static_cast<int>(max64(0, t - win0 + 1));
-  }
-}
-
 constexpr int kMaxSlots = 4096;  // keep_pages * page
 constexpr int kMaxPages = 64;    // keep_pages
 
@@ -1152,6 +1091,7 @@ static cudaError_t launch_fine_t(const IndexArgs& a, cudaStream_t st, int64_t* n
 
 cudaError_t launch_fine_select(const IndexArgs& a, cudaStream_t st, int64_t* n_launch) {
   if (a.n_query == 0) return cudaSuccess;
+  if (a.fine_cluster && fine_paged_tc_supported(a)) return launch_fine_paged_tc(a, a.sm_count, st, n_launch);
   if (a.fine_paged_tc && a.paged && a.fine_keys != nullptr && a.fine_pages != nullptr && paged_scores_tc_supported(a)) {
     // decode: page lists, then token scores of the listed pages on tcgen05, then the top-K_sparse with the cache rows
     cudaError_t e = launch_pdl(page_topm_paged_kernel, dim3(a.n_query), dim3(kSelThreads), 0, st, a);

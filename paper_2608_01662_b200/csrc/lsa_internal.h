@@ -42,6 +42,7 @@ struct IndexArgs {
   uint32_t* fine_keys;    // [n_query, 4096] order-preserving keys of the candidate slots (0 = not a candidate)
   int32_t* fine_pages;    // [n_query, 65]: kept pages, then their count
   int sm_count;           // SMs of the device (grid of the persistent paged kernels)
+  int fine_cluster;       // paged caches: the whole fine stage as one clustered tcgen05 kernel (lsa_fine_paged_tc.cu)
   int fine_paged_tc;      // paged caches: page lists, token scores on tcgen05 (lsa_scores_paged_tc.cu), top-K, as three kernels
   int* status;
 };
@@ -107,6 +108,8 @@ inline cudaError_t launch_coarse_best(const IndexArgs& a, int groups, cudaStream
   return coarse_tc_supported(a) ? launch_coarse_tc(a, groups, st, n_launch) : launch_coarse(a, st, n_launch);
 }
 // tcgen05 version of the coarse stage for paged caches (H_I = 64, d_I = 128); used by launch_coarse
+bool fine_paged_tc_supported(const IndexArgs& a);
+cudaError_t launch_fine_paged_tc(const IndexArgs& a, int sm_count, cudaStream_t st, int64_t* n_launch);
 bool coarse_paged_tc_supported(const IndexArgs& a);
 cudaError_t launch_coarse_paged_tc(const IndexArgs& a, cudaStream_t st, int64_t* n_launch);
 cudaError_t launch_fine_select(const IndexArgs& a, cudaStream_t st, int64_t* n_launch);

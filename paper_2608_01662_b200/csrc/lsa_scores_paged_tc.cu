@@ -163,10 +163,10 @@ paged_scores_tc_kernel(const __grid_constant__ CUtensorMap map_q, IndexArgs p, i
   if (tid == 0) {
     for (int s = 0; s < kRawSlots; ++s) {
       tc::mbar_init(smem_u32(&sm.raw_full[s]), 1);
-      tc::mbar_init(smem_u32(&sm.raw_empty[s]), kWidenThreads);
+      tc::mbar_init(smem_u32(&sm.raw_empty[s]), kWidenThreads / 32);
     }
     for (int b = 0; b < 2; ++b) {
-      tc::mbar_init(smem_u32(&sm.a_full[b]), kWidenThreads);
+      tc::mbar_init(smem_u32(&sm.a_full[b]), kWidenThreads / 32);
       tc::mbar_init(smem_u32(&sm.a_empty[b]), 1);
       tc::mbar_init(smem_u32(&sm.acc_full[b]), 1);
       tc::mbar_init(smem_u32(&sm.acc_empty[b]), 4);
@@ -319,8 +319,11 @@ paged_scores_tc_kernel(const __grid_constant__ CUtensorMap map_q, IndexArgs p, i
         }
       }
       tc::fence_proxy_async();
-      tc::mbar_arrive(smem_u32(&sm.a_full[b]));
-      tc::mbar_arrive(smem_u32(&sm.raw_empty[s]));
+      __syncwarp();
+      if (lane == 0) {   // one arrival per warp: 256 arrivals on one barrier are 256 serialised shared-memory operations
+        tc::mbar_arrive(smem_u32(&sm.a_full[b]));
+        tc::mbar_arrive(smem_u32(&sm.raw_empty[s]));
+      }
     }
   } else if (warp >= 4) {
     // ================= epilogue warps =================

@@ -279,16 +279,19 @@ def test_flat_indexer_on_paged_caches(cuda_device, key_dtype):
         assert torch.equal(hier.sparse_idx[b], wl.sparse_idx[b])
 
 
-def test_paged_fine_stage_on_tcgen05_gives_the_same_selection(cuda_device):
-    """LSA_TUNE_FINE_PAGED_TC = 1: page lists, token scores of the listed pages on tcgen05, top-K.  Same arithmetic per
-    token up to the summation order of the heads, so the sets are compared with the oracle, and with the default path."""
+@pytest.mark.parametrize("mode", [1, 2])
+def test_paged_fine_stage_on_tcgen05_gives_the_same_selection(cuda_device, mode):
+    """The fine stage over cache pages has three forms (LSA_TUNE_FINE_PAGED_TC): 0, the default, one kernel with a
+    thread-block cluster per sequence (page top-M, token scores on tcgen05, top-K, cache rows); 1: the same steps as
+    three kernels; 2: the mma.sync kernels.  Same arithmetic per token up to the summation order of the heads, so the
+    sets of forms 1 and 2 are compared with the oracle, and with the default form."""
     cfg = SMALL_DEC
     ref_wl = DecodeWorkload(cfg, cuda_device)
     ref_wl.prepare()
     ref_wl.step()
     wl = DecodeWorkload(cfg, cuda_device)
     wl.prepare()
-    wl.ctx.tune(5, 1)
+    wl.ctx.tune(5, mode)
     wl.step()
     assert wl.ctx.status() == 0
     m = pu.check_decode(wl, range(cfg.batch))
