@@ -275,7 +275,8 @@ def main():
     for _ in range(max(3, args.warmup)):
         wl.step()
     barrier()
-    assert wl.ctx.status() == 0
+    st = wl.ctx.status()
+    assert st == 0, f"device status {st}"
 
     stream = torch.cuda.current_stream(dev)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -449,7 +450,8 @@ def measure_decode(cfg, dev, peaks, steps=50, warmup=10):
     for _ in range(warmup):
         wl.step()
     torch.cuda.synchronize()
-    assert wl.ctx.status() == 0
+    st = wl.ctx.status()
+    assert st == 0, f"device status {st}"
     stream = torch.cuda.current_stream(dev)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     n0 = wl.ctx.launch_count()
@@ -480,7 +482,8 @@ def measure_decode(cfg, dev, peaks, steps=50, warmup=10):
     torch.cuda.synchronize()
     loop_prof = wl.ctx.profile_read()
     wl.ctx.profile_enable(False)
-    assert wl.ctx.status() == 0
+    st = wl.ctx.status()
+    assert st == 0, f"device status {st}"
     running = {"steps": grow, "us_per_step_with_event_pairs": ev0.elapsed_time(ev1) / grow * 1e3,
                "append_us": loop_prof["block_means"][0] / grow * 1e3,
                "what": "lsa_append (key quantised, sub-block mean updated, R latent rows stored) + lsa_layer_group, "

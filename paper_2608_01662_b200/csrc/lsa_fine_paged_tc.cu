@@ -9,15 +9,26 @@
 // of the cluster's first block (remote stores of 4 bytes per token), which takes the top-K and writes the results.
 // The scores never leave the SMs.
 //
-// Inside a block, after the page selection (threads 0-255):
-//   warp 0       producer: one bulk copy per page (a page is one contiguous piece of the key pool) and one for its
-//                per-token scales (e4m3 caches) into a ring of raw tiles
-//   warps 8-15   widen: a landed raw tile -> the 128B-swizzled K-major bf16 operand (e4m3 -> bf16 is exact)
-//   warps 1, 2   one thread of each issues 8 x tcgen05.mma (M128 N64 K16) per tile, warp 1 for the even tiles and
-//                warp 2 for the odd ones, each into its own TMEM accumulator
-//   warps 4-7    epilogue: one thread = one token: sum_j w_j relu(acc_j), times the token's scale, as an
-//                order-preserving key into the first block's candidate array
-// The query heads arrive by TMA before the dependency wait (they are an input of the call, not a product of the
+// Key tiles go from the pool to the tensor cores untouched: a page is one TMA box (64 rows), which lands in the
+// 128-byte-swizzled K-major layout the MMA reads.
+//   bf16 cache: kind::f16 MMAs against the bf16 query heads (8 x M128 N64 K16 per tile).
+//   e4m3 cache: the codes are the A operand of kind::f8f6f4 MMAs as they are.  The bf16 query heads become the B
+//     operand as three e5m2 planes: head j is scaled by a power of two 2^S_j that puts its largest element in
+//     [2^14, 2^15), then q 2^S = p1 + p2 + p3 with p1 = e5m2(q 2^S), p2 = e5m2(rest), p3 = e5m2(rest of that), each
+//     rest exact: a bf16 value has 8 significant bits, a plane takes 3, and an element only loses bits below 2^-23 of
+//     its head's largest (below the rounding of the fp32 accumulator).  The three planes accumulate into the same
+//     accumulator (12 x M128 N64 K32 per tile), so the tensor core sums them, every product exact, and the epilogue
+//     is the same as for bf16 with w_j 2^-S_j in place of w_j (relu commutes with a positive factor).  Nothing is
+//     widened and no 16-bit copy of the keys exists anywhere.
+//
+// Inside a block (12 warps), after the page selection (threads 0-255):
+//   warp 0       producer: TMA boxes of the pages into a ring of tiles
+//   warps 1-3    one thread of each issues the MMAs of every third tile, alternating between two TMEM accumulators of
+//                its own (one thread issues an MMA about every 95 cycles, the pipe needs 48: three issuers keep it
+//                busy, and nobody waits for the epilogue of a recent tile)
+//   warps 4-7 / 8-11   epilogue of the even / odd tiles: one thread = one token: sum_j w_j relu(acc_j), times the
+//                token's scale, as an order-preserving key into the first block's candidate array
+// The query heads are fetched before the dependency wait (they are an input of the call, not a product of the
 // coarse kernel that precedes this one in the stream).
 #include "lsa_internal.h"
 #include "lsa_select.cuh"
@@ -30,35 +41,43 @@ namespace {
 constexpr int kHI = 64, kDI = 128;
 constexpr int kTile = 128;                  // tokens per tile: two cache pages
 constexpr int kPageTok = 64;
-constexpr int kAtomA = kTile * 128;         // one 64-dim column block of a tile
-constexpr int kAtomQ = kHI * 128;
-constexpr int kThreadsFp = 512;
-constexpr int kWidenThreads = 256;          // warps 8-15
+constexpr int kThreadsFp = 384;
 constexpr int kMaxPagesFp = 64;
 constexpr int kMaxSlotsFp = kMaxPagesFp * kPageTok;
-constexpr uint32_t kTmemColsFp = 128;       // two accumulators of 64 columns
+constexpr uint32_t kTmemColsFp = 512;       // six accumulators of 64 columns (the allocation is a power of two)
+constexpr int kIssuers = 3;                 // MMA-issuing warps 1..3
+// Tile i is issued by warp 1 + i % 3 into accumulator (i % 3) + 3 * ((i / 3) % 2): an accumulator belongs to one
+// issuer, which alternates between its two.  (A barrier wait names the phase by its parity only: a thread that could
+// run two phases ahead of a barrier shared with other issuers would take an old phase for the one it waits for.)
+__device__ __forceinline__ int acc_of_tile(int i) { return i % kIssuers + kIssuers * ((i / kIssuers) & 1); }
+__device__ __forceinline__ uint32_t acc_use_parity(int i) { return static_cast<uint32_t>(i / (2 * kIssuers)) & 1u; }
 constexpr int kSelBar = 1;                  // named barrier of threads 0-255 (the selections)
 
 template <bool E4M3>
 struct FpSmem {
-  static constexpr int kRawTileBytes = E4M3 ? kTile * kDI : kTile * kDI * 2;
-  static constexpr int kRawSlots = E4M3 ? 6 : 3;
-  alignas(1024) uint8_t a[2][2][kAtomA];      // operand: [buffer][64-dim half][128 rows x 128 B]
-  alignas(1024) uint8_t q[2][kAtomQ];         // query heads: [64-dim half][64 rows x 128 B]
-  // ring of raw tiles; before the first copy it holds the keys of the page scores (up to kMaxSlotsFp of them)
-  alignas(128) uint8_t raw[kRawSlots][kRawTileBytes];
-  alignas(16) float raw_scale[kRawSlots][kTile];
-  float scale[4][kTile];   // four deep: the epilogue reads a tile's scales after its operand buffer is free again
+  static constexpr int kRowBytes = E4M3 ? kDI : kDI * 2;         // a token's key
+  static constexpr int kTileBytes = kTile * kRowBytes;
+  // ring slots: a multiple of the number of MMA issuers, so that a slot is always consumed by the same issuer (see
+  // acc_of_tile); 144 KB (e4m3) / 96 KB (bf16) of key tiles in flight
+  static constexpr int kSlots = E4M3 ? 9 : 3;
+  static constexpr int kQBytes = E4M3 ? 3 * kHI * kDI : kHI * kDI * 2;
+  // ring of key tiles.  e4m3: [128 rows x 128 B]; bf16: [64-dim half][128 rows x 128 B].  Before the first copy it
+  // holds the keys of the page scores (up to kMaxSlotsFp of them).
+  alignas(1024) uint8_t k[kSlots][kTileBytes];
+  // query heads.  e4m3 cache: three e5m2 planes [plane][64 heads x 128 B]; bf16: [64-dim half][64 heads x 128 B]
+  alignas(1024) uint8_t q[kQBytes];
+  float k_scale[E4M3 ? kMaxPagesFp / 2 : 1][kTile];   // per-token scales of the block's tiles (e4m3); a thread reads what it wrote
   float w[kHI];
   uint32_t keys[kMaxSlotsFp];   // candidate keys of the whole cluster (used in the first block only)
   int32_t pages[kMaxPagesFp];   // kept pages, ascending
   int32_t phys[kMaxPagesFp];    // their places in the pool
   SelectScratch sel;
-  alignas(8) uint64_t raw_full[6], raw_empty[6], a_full[2], acc_full[2], acc_empty[2], q_full;
+  alignas(8) uint64_t k_full[9], k_empty[9], acc_full[2 * kIssuers], acc_empty[2 * kIssuers], q_full;
   uint32_t tmem_slot;
 };
 static_assert(sizeof(FpSmem<true>) + 1024 <= 227 * 1024 && sizeof(FpSmem<false>) + 1024 <= 227 * 1024, "shared memory");
-static_assert(FpSmem<true>::kRawSlots * FpSmem<true>::kRawTileBytes >= kMaxSlotsFp * 4, "page keys fit the ring");
+static_assert(FpSmem<true>::kSlots * FpSmem<true>::kTileBytes >= kMaxSlotsFp * 4, "page keys fit the ring");
+static_assert(FpSmem<true>::kSlots % kIssuers == 0 && FpSmem<false>::kSlots % kIssuers == 0, "a ring slot has one consumer");
 
 __device__ __forceinline__ uint32_t cluster_rank() {
   uint32_t r;
@@ -81,12 +100,6 @@ __device__ __forceinline__ uint32_t smem_of_rank(uint32_t addr, uint32_t rank) {
 __device__ __forceinline__ void store_cluster_u32(uint32_t addr, uint32_t v) {
   asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
-// global -> shared bulk copy; completion is counted in bytes on `bar`.  Both addresses 16-byte aligned, size a multiple of 16.
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-
 // a4 + a5 for one sequence (all threads of the cluster's first block): top-K_sparse of the candidate keys by threads
 // 0-255, ascending positions, written both as positions (sparse_idx) and as the cache rows the attention kernels read
 // (the pages' places in the pool are at hand: no page-table look-up per row); then the sink and window rows and the
@@ -136,13 +149,40 @@ __device__ __forceinline__ void finish_sequence(const IndexArgs& p, const uint32
   if (tid == 0) p.n_rows_out[qi] = n_sink + n_sel + n_win;
 }
 
+// 16 consecutive elements of a query head, scaled, as three e5m2 planes (16 bytes each): x = p1 + p2 + p3.
+__device__ __forceinline__ void split_e5m2x16(const float (&x)[16], uint4& p1, uint4& p2, uint4& p3) {
+  uint32_t out[3][4];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    float2 r = make_float2(x[2 * j], x[2 * j + 1]);
+    uint32_t c[3];
+#pragma unroll
+    for (int pl = 0; pl < 3; ++pl) {
+      const __nv_fp8x2_storage_t v = __nv_cvt_float2_to_fp8x2(r, __NV_SATFINITE, __NV_E5M2);   // .x in the low byte
+      const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2(v, __NV_E5M2);
+      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h));
+      r.x -= f.x;   // exact: the rest has fewer significant bits than the value
+      r.y -= f.y;
+      c[pl] = v;
+    }
+#pragma unroll
+    for (int pl = 0; pl < 3; ++pl) {
+      if ((j & 1) == 0) out[pl][j >> 1] = c[pl];
+      else out[pl][j >> 1] |= c[pl] << 16;
+    }
+  }
+  p1 = make_uint4(out[0][0], out[0][1], out[0][2], out[0][3]);
+  p2 = make_uint4(out[1][0], out[1][1], out[1][2], out[1][3]);
+  p3 = make_uint4(out[2][0], out[2][1], out[2][2], out[2][3]);
+}
+
 template <bool E4M3>
 __global__ void __launch_bounds__(kThreadsFp, 1)
-fine_paged_tc_kernel(const __grid_constant__ CUtensorMap map_q, IndexArgs p) {
+fine_paged_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, IndexArgs p) {
   using Smem = FpSmem<E4M3>;
-  constexpr int kRawSlots = Smem::kRawSlots;
-  constexpr int kRowBytes = E4M3 ? kDI : kDI * 2;            // a token's key in the pool
-  constexpr int kPageBytes = kPageTok * kRowBytes;
+  constexpr int kSlots = Smem::kSlots;
+  constexpr int kAtom = kTile * 128;        // 128 rows x 128 B
+  constexpr int kAtomQ = kHI * 128;
   extern __shared__ uint8_t smem_raw[];
   Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -153,28 +193,62 @@ fine_paged_tc_kernel(const __grid_constant__ CUtensorMap map_q, IndexArgs p) {
   const bool live = !tc::status_raised(p.status);
 
   if (tid == 0) {
-    for (int s = 0; s < kRawSlots; ++s) {
-      tc::mbar_init(smem_u32(&sm.raw_full[s]), 1);
-      tc::mbar_init(smem_u32(&sm.raw_empty[s]), kWidenThreads / 32);
+    for (int s = 0; s < kSlots; ++s) {
+      tc::mbar_init(smem_u32(&sm.k_full[s]), 1);
+      tc::mbar_init(smem_u32(&sm.k_empty[s]), 1);   // the MMAs' commit
     }
-    for (int b = 0; b < 2; ++b) {
-      tc::mbar_init(smem_u32(&sm.a_full[b]), kWidenThreads / 32);
+    for (int b = 0; b < 2 * kIssuers; ++b) {
       tc::mbar_init(smem_u32(&sm.acc_full[b]), 1);
       tc::mbar_init(smem_u32(&sm.acc_empty[b]), 4);
     }
     tc::mbar_init(smem_u32(&sm.q_full), 1);
     tc::fence_mbar_init();
-    if (live) {
+    if (!E4M3 && live) {
       tc::mbar_expect_tx(smem_u32(&sm.q_full), 2 * kAtomQ);
-      tc::tma_load_2d(smem_u32(sm.q[0]), &map_q, 0, qi * kHI, smem_u32(&sm.q_full));
-      tc::tma_load_2d(smem_u32(sm.q[1]), &map_q, 64, qi * kHI, smem_u32(&sm.q_full));
+      tc::tma_load_2d(smem_u32(sm.q), &map_q, 0, qi * kHI, smem_u32(&sm.q_full));
+      tc::tma_load_2d(smem_u32(sm.q) + kAtomQ, &map_q, 64, qi * kHI, smem_u32(&sm.q_full));
     }
   }
   if (warp == 1) {
     tc::tmem_alloc(smem_u32(&sm.tmem_slot), kTmemColsFp);
     tc::tmem_relinquish();
   }
-  if (tid < kHI) sm.w[tid] = p.w[static_cast<int64_t>(qi) * kHI + tid];
+  if constexpr (E4M3) {
+    // query heads -> three e5m2 planes in the swizzled K-major layout; head weights take the inverse of the head's scale
+    for (int u = tid; u < kHI * 8; u += kThreadsFp) {   // 8 threads per head, 16 dims each (a warp never straddles a head group)
+      const int h = u >> 3, sub = u & 7;
+      const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(p.q_idx) +
+                                                        (static_cast<int64_t>(qi) * kHI + h) * kDI * 2 + sub * 32);
+      const uint4 v0 = src[0], v1 = src[1];
+      const uint32_t wv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+      float x[16];
+      float m = 0.f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        x[2 * j] = __uint_as_float(wv[j] << 16);
+        x[2 * j + 1] = __uint_as_float(wv[j] & 0xffff0000u);
+        m = fmaxf(m, fmaxf(fabsf(x[2 * j]), fabsf(x[2 * j + 1])));
+      }
+      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 4));
+      int S = 0;
+      if (m > 0.f) S = min(100, max(-100, 14 - (static_cast<int>((__float_as_uint(m) >> 23) & 0xffu) - 127)));
+      const float up = __uint_as_float(static_cast<uint32_t>(S + 127) << 23);
+#pragma unroll
+      for (int j = 0; j < 16; ++j) x[j] *= up;   // exact
+      uint4 p1, p2, p3;
+      split_e5m2x16(x, p1, p2, p3);
+      const int chunk = (sub ^ (h & 7)) << 4;    // rows of all three planes share h & 7 (a plane is 64 rows)
+      *reinterpret_cast<uint4*>(sm.q + 0 * kAtomQ + h * 128 + chunk) = p1;
+      *reinterpret_cast<uint4*>(sm.q + 1 * kAtomQ + h * 128 + chunk) = p2;
+      *reinterpret_cast<uint4*>(sm.q + 2 * kAtomQ + h * 128 + chunk) = p3;
+      if (sub == 0) sm.w[h] = p.w[static_cast<int64_t>(qi) * kHI + h] * __uint_as_float(static_cast<uint32_t>(127 - S) << 23);
+    }
+    tc::fence_proxy_async();   // the planes are read by the tensor core
+  } else {
+    if (tid < kHI) sm.w[tid] = p.w[static_cast<int64_t>(qi) * kHI + tid];
+  }
   pdl_wait();                 // the page scores come from the coarse kernel
   pdl_launch_dependents();
 
@@ -190,7 +264,7 @@ fine_paged_tc_kernel(const __grid_constant__ CUtensorMap map_q, IndexArgs p) {
       if (p.hi_enable && nE > p.M) {
         const float* ps = p.page_scores + static_cast<int64_t>(qi) * p.ps_ld + p0;
         if (nE <= kMaxSlotsFp) {
-          uint32_t* pk = reinterpret_cast<uint32_t*>(sm.raw);
+          uint32_t* pk = reinterpret_cast<uint32_t*>(sm.k);
           for (int i0 = tid; i0 < nE; i0 += 8 * kSelThreads) {   // eight loads in flight per thread
             float v[8];
 #pragma unroll
@@ -201,7 +275,7 @@ fine_paged_tc_kernel(const __grid_constant__ CUtensorMap map_q, IndexArgs p) {
           }
           select_sync<kSelBar>();
           nP = block_select_topk<kSelBar>([&](int i) { return pk[i]; }, [&](int i) { return p0 + i; }, nE, p.M, sm.pages, sm.sel);
-          tc::fence_proxy_async();   // the ring is handed to the bulk copies
+          tc::fence_proxy_async();   // the ring is handed to the TMA copies
         } else {
           nP = block_select_topk<kSelBar>([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M,
                                           sm.pages, sm.sel);
@@ -215,7 +289,7 @@ fine_paged_tc_kernel(const __grid_constant__ CUtensorMap map_q, IndexArgs p) {
     }
     if (rank == 0 && p.pages_out != nullptr)
       for (int i = tid; i < p.M; i += kSelThreads) p.pages_out[static_cast<int64_t>(qi) * p.M + i] = i < nP ? sm.pages[i] : -1;
-    if (tid == 0) sm.sel.n_valid = static_cast<uint32_t>(nP);   // for the other half of the block
+    if (tid == 0) sm.sel.n_valid = static_cast<uint32_t>(nP);   // for the other warps of the block
   }
   tc::fence_before_sync();
   __syncthreads();
@@ -232,106 +306,110 @@ fine_paged_tc_kernel(const __grid_constant__ CUtensorMap map_q, IndexArgs p) {
   if (warp == 0) {
     // ================= producer =================
     if (lane == 0) {
-      const uint8_t* kbase = reinterpret_cast<const uint8_t*>(p.k_idx);
+      constexpr uint32_t kPageBytes = kPageTok * Smem::kRowBytes;
       for (int i = 0; i < n_tiles; ++i) {
         const int tl = tile0 + i;
         const int f0 = sm.phys[2 * tl];
         const int f1 = 2 * tl + 1 < nP ? sm.phys[2 * tl + 1] : -1;
-        const int s = i % kRawSlots;
-        if (!tc::mbar_wait(smem_u32(&sm.raw_empty[s]), ((i / kRawSlots) & 1) ^ 1, p.status)) break;
-        const uint32_t bar = smem_u32(&sm.raw_full[s]);
-        const uint32_t per_page = kPageBytes + (E4M3 ? kPageTok * 4 : 0);
-        tc::mbar_expect_tx(bar, f1 >= 0 ? 2 * per_page : per_page);
-        bulk_load(smem_u32(sm.raw[s]), kbase + static_cast<int64_t>(f0) * kPageBytes, kPageBytes, bar);
-        if (E4M3) bulk_load(smem_u32(sm.raw_scale[s]), p.k_scale + static_cast<int64_t>(f0) * kPageTok, kPageTok * 4, bar);
-        if (f1 >= 0) {
-          bulk_load(smem_u32(sm.raw[s]) + kPageBytes, kbase + static_cast<int64_t>(f1) * kPageBytes, kPageBytes, bar);
-          if (E4M3)
-            bulk_load(smem_u32(&sm.raw_scale[s][kPageTok]), p.k_scale + static_cast<int64_t>(f1) * kPageTok, kPageTok * 4, bar);
+        const int s = i % kSlots;
+        if (!tc::mbar_wait(smem_u32(&sm.k_empty[s]), ((i / kSlots) & 1) ^ 1, p.status)) break;
+        const uint32_t bar = smem_u32(&sm.k_full[s]);
+        tc::mbar_expect_tx(bar, f1 >= 0 ? 2 * kPageBytes : kPageBytes);
+        const uint32_t dst = smem_u32(sm.k[s]);
+        if constexpr (E4M3) {
+          tc::tma_load_2d(dst, &map_k, 0, f0 * kPageTok, bar);
+          if (f1 >= 0) tc::tma_load_2d(dst + kPageBytes, &map_k, 0, f1 * kPageTok, bar);
+        } else {
+          // a page = rows 0-63 (or 64-127) of the tile's two 64-dim column blocks
+          tc::tma_load_2d(dst, &map_k, 0, f0 * kPageTok, bar);
+          tc::tma_load_2d(dst + kAtom, &map_k, 64, f0 * kPageTok, bar);
+          if (f1 >= 0) {
+            tc::tma_load_2d(dst + kPageTok * 128, &map_k, 0, f1 * kPageTok, bar);
+            tc::tma_load_2d(dst + kAtom + kPageTok * 128, &map_k, 64, f1 * kPageTok, bar);
+          }
         }
       }
     }
-  } else if (warp == 1 || warp == 2) {
-    // ================= MMA issuers: warp 1 takes the even tiles (operand buffer and accumulator 0), warp 2 the odd
-    // ones; one thread issues an MMA every 55-90 cycles, two keep the pipe busy =================
+  } else if (warp <= kIssuers) {
+    // ================= MMA issuers: warps 1-3 take every third tile each, alternating between two accumulators of
+    // their own, so that nobody waits for the epilogue of a recent tile.  One thread issues an MMA about every 95
+    // cycles here and the pipe needs 48 for one (both operands from shared memory): three issuers keep it busy ====
     const int b = warp - 1;
     if (lane == 0 && n_tiles > b) {
-      constexpr uint32_t idesc = tc::idesc_bf16(kTile, kHI, 0, 0);
-      const uint64_t da0 = tc::smem_desc_sw128(smem_u32(sm.a[b]), 16, 1024);
+      constexpr int kSteps = E4M3 ? 12 : 8;
+      constexpr uint32_t idesc = E4M3 ? tc::idesc_e4m3_e5m2(kTile, kHI) : tc::idesc_bf16(kTile, kHI, 0, 0);
+      const uint64_t da0 = tc::smem_desc_sw128(smem_u32(sm.k), 16, 1024);
       const uint64_t dq0 = tc::smem_desc_sw128(smem_u32(sm.q), 16, 1024);
-      uint64_t da[8], dq[8];
+      uint32_t a_off[kSteps];
+      uint64_t dq[kSteps];
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {   // 16-dim step: column block ks/4, 32-byte slice ks%4
-        da[ks] = tc::desc_advance(da0, (ks >> 2) * kAtomA + (ks & 3) * 32);
-        dq[ks] = tc::desc_advance(dq0, (ks >> 2) * kAtomQ + (ks & 3) * 32);
+      for (int j = 0; j < kSteps; ++j) {
+        if constexpr (E4M3) {   // plane j / 4, 32-element step j % 4 of the 128-byte rows
+          a_off[j] = (j & 3) * 32;
+          dq[j] = tc::desc_advance(dq0, (j >> 2) * kAtomQ + (j & 3) * 32);
+        } else {                // 64-dim column block j / 4, 16-element step j % 4
+          a_off[j] = (j >> 2) * kAtom + (j & 3) * 32;
+          dq[j] = tc::desc_advance(dq0, (j >> 2) * kAtomQ + (j & 3) * 32);
+        }
       }
-      const uint32_t d = tmem_base + b * kHI;
-      bool ok = tc::mbar_wait(smem_u32(&sm.q_full), 0, p.status);
-      for (int i = b; i < n_tiles && ok; i += 2) {
-        if (!tc::mbar_wait(smem_u32(&sm.a_full[b]), (i >> 1) & 1, p.status) ||
-            !tc::mbar_wait(smem_u32(&sm.acc_empty[b]), ((i >> 1) & 1) ^ 1, p.status))
+      bool ok = E4M3 ? true : tc::mbar_wait(smem_u32(&sm.q_full), 0, p.status);
+      for (int i = b; i < n_tiles && ok; i += kIssuers) {
+        const int s = i % kSlots;
+        const int acc = acc_of_tile(i);
+        if (!tc::mbar_wait(smem_u32(&sm.k_full[s]), (i / kSlots) & 1, p.status) ||
+            !tc::mbar_wait(smem_u32(&sm.acc_empty[acc]), acc_use_parity(i) ^ 1u, p.status))
           break;
         tc::fence_after_sync();
+        const uint32_t d = tmem_base + acc * kHI;
+        const uint64_t da = tc::desc_advance(da0, s * Smem::kTileBytes);
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) tc::umma_ss(d, da[ks], dq[ks], idesc, ks != 0);
-        tc::umma_commit(smem_u32(&sm.acc_full[b]));   // accumulator ready = operand buffer free again
-      }
-    }
-  } else if (warp >= 8) {
-    // ================= widen warps =================
-    const int wt = tid - 256;   // 0..255
-    for (int i = 0; i < n_tiles; ++i) {
-      const int s = i % kRawSlots, b = i & 1;
-      if (!tc::mbar_wait(smem_u32(&sm.raw_full[s]), (i / kRawSlots) & 1, p.status) ||
-          !tc::mbar_wait(smem_u32(&sm.acc_full[b]), ((i >> 1) & 1) ^ 1, p.status))   // MMAs of tile i - 2 complete
-        break;
-      if constexpr (E4M3) {
-        if (wt < kTile) sm.scale[i & 3][wt] = sm.raw_scale[s][wt];
-#pragma unroll
-        for (int j = 0; j < kTile * 8 / kWidenThreads; ++j) {   // 16 codes -> dims 16u .. 16u+15 = 16-byte chunks 2u, 2u+1 of the row
-          const int e = wt + j * kWidenThreads, r = e >> 3, u = e & 7;
-          const uint4 c = *reinterpret_cast<const uint4*>(sm.raw[s] + e * 16);
-          uint4 lo16, hi16;
-          e4m3x16_to_bf16(c, lo16, hi16);
-          uint8_t* dst = sm.a[b][u >> 2] + r * 128;
-          *reinterpret_cast<uint4*>(dst + ((((2 * u) & 7) ^ (r & 7)) << 4)) = lo16;
-          *reinterpret_cast<uint4*>(dst + ((((2 * u + 1) & 7) ^ (r & 7)) << 4)) = hi16;
+        for (int j = 0; j < kSteps; ++j) {
+          if constexpr (E4M3) tc::umma_ss_f8(d, tc::desc_advance(da, a_off[j]), dq[j], idesc, j != 0);
+          else tc::umma_ss(d, tc::desc_advance(da, a_off[j]), dq[j], idesc, j != 0);
         }
-      } else {
-#pragma unroll
-        for (int j = 0; j < kTile * 16 / kWidenThreads; ++j) {
-          const int e = wt + j * kWidenThreads, r = e >> 4, u = e & 15;
-          *reinterpret_cast<uint4*>(sm.a[b][u >> 3] + r * 128 + (((u & 7) ^ (r & 7)) << 4)) =
-              *reinterpret_cast<const uint4*>(sm.raw[s] + e * 16);
-        }
-      }
-      tc::fence_proxy_async();
-      __syncwarp();
-      if (lane == 0) {   // one arrival per warp: 256 arrivals on one barrier are 256 serialised shared-memory operations
-        tc::mbar_arrive(smem_u32(&sm.a_full[b]));
-        tc::mbar_arrive(smem_u32(&sm.raw_empty[s]));
+        tc::umma_commit(smem_u32(&sm.k_empty[s]));
+        tc::umma_commit(smem_u32(&sm.acc_full[acc]));
       }
     }
   } else if (warp >= 4) {
-    // ================= epilogue warps =================
-    const int quarter = warp & 3;          // warps 4-7 own TMEM lanes 32*quarter .. +31
+    // ================= epilogue: warps 4-7 the even tiles, warps 8-11 the odd ones =================
+    const int b = (warp >> 2) - 1;
+    const int quarter = warp & 3;          // TMEM lanes 32*quarter .. +31
     const int r = 32 * quarter + lane;     // token row of the tile
     const uint32_t keys0 = smem_of_rank(smem_u32(sm.keys), 0);
-    for (int i = 0; i < n_tiles; ++i) {
-      const int b = i & 1;
+    if constexpr (E4M3) {
+      // the scales of this thread's tokens, straight from the pool (an issued TMA or bulk copy costs its thread some
+      // 200 cycles, so the producer issues nothing but the key boxes); the loads of all tiles are in flight together
+      for (int i0 = b; i0 < n_tiles; i0 += 16) {
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {   // eight loads in flight
+          const int i = i0 + 2 * u;
+          const int c = (tile0 + i) * kTile + r;
+          v[u] = (i < n_tiles && c < n_slots) ? p.k_scale[static_cast<int64_t>(sm.phys[c >> 6]) * kPageTok + (c & (kPageTok - 1))] : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          if (i0 + 2 * u < n_tiles) sm.k_scale[i0 + 2 * u][r] = v[u];
+      }
+    }
+    for (int i = b; i < n_tiles; i += 2) {
+      const int acc = acc_of_tile(i);
       const int c = (tile0 + i) * kTile + r;   // candidate slot
       int64_t pos = -1;
       if (c < n_slots) pos = static_cast<int64_t>(sm.pages[c >> 6]) * kPageTok + (c & (kPageTok - 1));
       const bool cand = pos >= lo && pos <= hi;
-      if (!__all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.acc_full[b]), (i >> 1) & 1, p.status))) break;
+      if (!__all_sync(0xffffffffu, tc::mbar_wait(smem_u32(&sm.acc_full[acc]), acc_use_parity(i), p.status))) break;
       tc::fence_after_sync();
       uint32_t v[64];
-      tc::tmem_ld64(tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + b * kHI, v);
+      tc::tmem_ld64(tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + acc * kHI, v);
       tc::tmem_ld_wait();
-      const float sc = E4M3 ? sm.scale[i & 3][r] : 1.f;   // read before the accumulator is handed back
+      const float sc = E4M3 ? sm.k_scale[i][r] : 1.f;
       tc::fence_before_sync();
       __syncwarp();
-      if (lane == 0) tc::mbar_arrive(smem_u32(&sm.acc_empty[b]));
+      if (lane == 0) {
+        tc::mbar_arrive(smem_u32(&sm.acc_empty[acc]));
+      }
       float a0 = 0.f, a1 = 0.f;
       const float4* w4 = reinterpret_cast<const float4*>(sm.w);
 #pragma unroll
@@ -367,8 +445,12 @@ bool fine_paged_tc_supported(const IndexArgs& a) {
 // One cluster per sequence: two blocks while all clusters are resident at once, else one.
 cudaError_t launch_fine_paged_tc(const IndexArgs& a, int sm_count, cudaStream_t st, int64_t* n_launch) {
   if (a.n_query == 0) return cudaSuccess;
-  CUtensorMap map_q;
-  if (!make_map_bf16_128(&map_q, a.q_idx, static_cast<uint64_t>(a.n_query) * kHI, kHI)) return cudaErrorInvalidValue;
+  // The key pool belongs to the caller and its size is not part of the call: the map spans the largest row range a
+  // page-table entry can address; only boxes of mapped pages are ever requested.
+  CUtensorMap map_q, map_k;
+  if (!make_map_bf16_128(&map_q, a.q_idx, static_cast<uint64_t>(a.n_query) * kHI, kHI) ||
+      !(a.key_e4m3 ? make_map_u8_128(&map_k, a.k_idx, 1ull << 31, kPageTok) : make_map_bf16_128(&map_k, a.k_idx, 1ull << 31, kPageTok)))
+    return cudaErrorInvalidValue;
   const int sms = sm_count > 0 ? sm_count : 148;
   const unsigned n_rank = 2 * a.n_query <= sms ? 2u : 1u;
   cudaLaunchConfig_t cfg{};
@@ -390,13 +472,13 @@ cudaError_t launch_fine_paged_tc(const IndexArgs& a, int sm_count, cudaStream_t 
     e = cudaFuncSetAttribute(fine_paged_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(cfg.dynamicSmemBytes));
     if (e != cudaSuccess) return e;
-    e = cudaLaunchKernelEx(&cfg, fine_paged_tc_kernel<true>, map_q, a);
+    e = cudaLaunchKernelEx(&cfg, fine_paged_tc_kernel<true>, map_q, map_k, a);
   } else {
     cfg.dynamicSmemBytes = sizeof(FpSmem<false>) + 1024;
     e = cudaFuncSetAttribute(fine_paged_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(cfg.dynamicSmemBytes));
     if (e != cudaSuccess) return e;
-    e = cudaLaunchKernelEx(&cfg, fine_paged_tc_kernel<false>, map_q, a);
+    e = cudaLaunchKernelEx(&cfg, fine_paged_tc_kernel<false>, map_q, map_k, a);
   }
   ++*n_launch;
   return e;

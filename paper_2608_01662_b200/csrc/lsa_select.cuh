@@ -155,18 +155,26 @@ __device__ int block_select_topk_emit(KeyF key, EmitF emit, AbsentF absent, int 
   int out_run = gt_before + min(eq_before, need_eq);
   int eq_run = eq_before;
   const uint32_t lt_mask = (1u << lane) - 1u;
-  for (int base = begin; base < end; base += 32) {
-    const int i = base + lane;
-    const uint32_t kk = i < end ? key(i) : 0u;
-    const bool is_gt = kk > T;
-    const bool is_eq = (kk == T) && (kk != 0u);
-    const uint32_t eq_mask = __ballot_sync(0xffffffffu, is_eq);
-    const int my_eq_rank = eq_run + __popc(eq_mask & lt_mask);
-    const bool sel = is_gt || (is_eq && my_eq_rank < need_eq);
-    const uint32_t sel_mask = __ballot_sync(0xffffffffu, sel);
-    if (sel) emit(out_run + __popc(sel_mask & lt_mask), i);
-    out_run += __popc(sel_mask);
-    eq_run += __popc(eq_mask);
+  // four rows of 32 keys per step: their loads and the ballots of the threshold ties do not wait for one another
+#pragma unroll 1
+  for (int base = begin; base < end; base += 4 * 32) {
+    uint32_t kk[4], eq_mask[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = base + 32 * u + lane;
+      kk[u] = i < end ? key(i) : 0u;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) eq_mask[u] = __ballot_sync(0xffffffffu, (kk[u] == T) && (kk[u] != 0u));
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const bool is_eq = (kk[u] == T) && (kk[u] != 0u);
+      const bool sel = kk[u] > T || (is_eq && eq_run + __popc(eq_mask[u] & lt_mask) < need_eq);
+      const uint32_t sel_mask = __ballot_sync(0xffffffffu, sel);
+      if (sel) emit(out_run + __popc(sel_mask & lt_mask), base + 32 * u + lane);
+      out_run += __popc(sel_mask);
+      eq_run += __popc(eq_mask[u]);
+    }
   }
   const int written = min(k, n_valid);
   for (int i = written + tid; i < k; i += kSelThreads) absent(i);

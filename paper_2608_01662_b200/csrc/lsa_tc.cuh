@@ -206,6 +206,21 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N, int a_mn, int b_
          (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
 }
 
+// Instruction descriptor for 8-bit floating-point operands (kind::f8f6f4): A in e4m3, B in e5m2, fp32 accumulator, both
+// K-major.  One instruction covers K = 32 elements (32 bytes of a row).
+__host__ __device__ constexpr uint32_t idesc_e4m3_e5m2(int M, int N) {
+  return (1u << 4) | (0u << 7) | (1u << 10) | (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
+}
+// D[tmem] (+)= A[smem] * B[smem] with 8-bit floating-point operands.
+__device__ __forceinline__ void umma_ss_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
 // D[tmem] (+)= A[smem] * B[smem]; one thread issues.
 __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
@@ -238,6 +253,8 @@ bool tma_available();
 // Tensor map of a bf16 matrix [rows, 128] row-major: box = 64 columns x box_rows rows, 128-byte swizzle, zero fill
 // outside.  `base` must be 16-byte aligned.
 bool make_map_bf16_128(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows);
+// bytes [rows, 128] row-major (e4m3 codes of a 128-dim key per row), box = the whole row x box_rows rows, 128-byte swizzle.
+bool make_map_u8_128(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows);
 bool make_map_bf16_rows(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint32_t box_rows);
 
 }  // namespace lsa
