@@ -244,15 +244,18 @@ def test_runs_are_deterministic(cuda_device):
         assert torch.equal(idx0, wl.sparse_idx) and torch.equal(out0, wl.out[1])
 
 
-def test_small_paged_decode(cuda_device):
-    cfg = SMALL_DEC
+@pytest.mark.parametrize("key_dtype", ["e4m3", "bf16"])
+def test_small_paged_decode(cuda_device, key_dtype):
+    """e4m3 caches: the fine stage feeds the codes to FP8 MMAs against the query heads split into three e5m2 planes;
+    bf16 caches: bf16 MMAs.  Both against the fp64 oracle."""
+    cfg = SMALL_DEC.replace(name="dec_small_" + key_dtype, key_dtype=key_dtype)
     wl = DecodeWorkload(cfg, cuda_device)
     wl.prepare()
     wl.step()
     assert wl.ctx.status() == 0
     m = pu.check_decode(wl, range(cfg.batch))
     print(cfg.name, m.summary())
-    m.assert_ok(pu.TOL_FP8)
+    m.assert_ok(pu.TOL_FP8 if key_dtype == "e4m3" else pu.TOL_BF16)
 
 
 @pytest.mark.parametrize("key_dtype", ["e4m3", "bf16"])
@@ -317,8 +320,9 @@ def test_paged_decode_row_splits(cuda_device, n_split):
 
 
 def test_paged_decode_large_batch(cuda_device):
-    """More sequences than twice the SM count: the fine stage runs unsplit (one block per sequence selects by itself)
-    and the cache rows come from the separate conversion kernel."""
+    """More sequences than half the SM count: the fine stage gives each sequence one block instead of a cluster of two
+    (the block scores every kept page itself).  Short contexts: some sequences have fewer eligible pages than the
+    budget, and an odd number of them (a tile with one page)."""
     cfg = SMALL_DEC.replace(name="dec_wide", batch=320, ctx_lo=700, ctx_hi=1600, M=8, Ksp=256, R=1, seed=19)
     wl = DecodeWorkload(cfg, cuda_device)
     wl.prepare()
