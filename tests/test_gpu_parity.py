@@ -319,6 +319,24 @@ def test_paged_decode_row_splits(cuda_device, n_split):
     m.assert_ok(pu.TOL_FP8)
 
 
+def test_paged_decode_tiny_contexts(cuda_device):
+    """Contexts from one token up: sequences with nothing outside sink and window (no candidate page, no tile, an empty
+    selection), with a window that is not yet full, and with a handful of candidate pages."""
+    cfg = SMALL_DEC.replace(name="dec_tiny", batch=24, ctx_lo=1, ctx_hi=700, M=8, Ksp=256, R=1, seed=41)
+    wl = DecodeWorkload(cfg, cuda_device)
+    wl.prepare()
+    wl.step()
+    assert wl.ctx.status() == 0
+    ctx = wl.ctx_len.cpu().numpy()
+    assert (ctx <= cfg.S + cfg.W).any() and (ctx > cfg.S + cfg.W + cfg.P).any()
+    m = pu.check_decode(wl, range(cfg.batch))
+    print(cfg.name, m.summary())
+    m.assert_ok(pu.TOL_FP8)
+    n_sp = wl.n_sparse.cpu().numpy()
+    for b in range(cfg.batch):
+        assert n_sp[b] == max(0, min(cfg.Ksp, int(ctx[b]) - cfg.S - cfg.W))
+
+
 def test_paged_decode_large_batch(cuda_device):
     """More sequences than half the SM count: the fine stage gives each sequence one block instead of a cluster of two
     (the block scores every kept page itself).  Short contexts: some sequences have fewer eligible pages than the
