@@ -90,6 +90,44 @@ __device__ __forceinline__ void e4m3x16_to_bf16(const uint4& c, uint4& lo, uint4
   hi.w = e4m3x2_to_bf16x2(static_cast<uint16_t>(c.w >> 16));
 }
 
+// ---- bf16 query heads as e5m2 planes (B operand of FP8 MMAs against e4m3 key codes) -------------------
+// A head is scaled by 2^S so that its largest element lies in [2^14, 2^15); then x = p1 + p2 + p3 with p1 = e5m2(x),
+// p2 = e5m2(x - p1), p3 = e5m2(x - p1 - p2), every difference exact: a bf16 value has 8 significant bits, a plane
+// takes 3; only an element below 2^-23 of its head's largest loses bits, and what it loses is below 2^-30 of that
+// largest element (less than the rounding of the fp32 accumulator).
+__device__ __forceinline__ int e5m2_head_shift(float head_max_abs) {
+  if (!(head_max_abs > 0.f)) return 0;
+  const int e = static_cast<int>((__float_as_uint(head_max_abs) >> 23) & 0xffu) - 127;
+  const int s = 14 - e;
+  return s > 100 ? 100 : (s < -100 ? -100 : s);
+}
+// 16 consecutive elements of a query head, scaled, as three e5m2 planes (16 bytes each): x = p1 + p2 + p3.
+__device__ __forceinline__ void split_e5m2x16(const float (&x)[16], uint4& p1, uint4& p2, uint4& p3) {
+  uint32_t out[3][4];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    float2 r = make_float2(x[2 * j], x[2 * j + 1]);
+    uint32_t c[3];
+#pragma unroll
+    for (int pl = 0; pl < 3; ++pl) {
+      const __nv_fp8x2_storage_t v = __nv_cvt_float2_to_fp8x2(r, __NV_SATFINITE, __NV_E5M2);   // .x in the low byte
+      const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2(v, __NV_E5M2);
+      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h));
+      r.x -= f.x;   // exact: the rest has fewer significant bits than the value
+      r.y -= f.y;
+      c[pl] = v;
+    }
+#pragma unroll
+    for (int pl = 0; pl < 3; ++pl) {
+      if ((j & 1) == 0) out[pl][j >> 1] = c[pl];
+      else out[pl][j >> 1] |= c[pl] << 16;
+    }
+  }
+  p1 = make_uint4(out[0][0], out[0][1], out[0][2], out[0][3]);
+  p2 = make_uint4(out[1][0], out[1][1], out[1][2], out[1][3]);
+  p3 = make_uint4(out[2][0], out[2][1], out[2][2], out[2][3]);
+}
+
 // ---- order-preserving key of an fp32 score --------------------------------------------------------
 // Larger score <-> larger key; -0 is folded onto +0; key 0 is never produced by a finite score and
 // marks "absent".

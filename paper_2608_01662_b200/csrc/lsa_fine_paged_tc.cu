@@ -149,33 +149,6 @@ __device__ __forceinline__ void finish_sequence(const IndexArgs& p, const uint32
   if (tid == 0) p.n_rows_out[qi] = n_sink + n_sel + n_win;
 }
 
-// 16 consecutive elements of a query head, scaled, as three e5m2 planes (16 bytes each): x = p1 + p2 + p3.
-__device__ __forceinline__ void split_e5m2x16(const float (&x)[16], uint4& p1, uint4& p2, uint4& p3) {
-  uint32_t out[3][4];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    float2 r = make_float2(x[2 * j], x[2 * j + 1]);
-    uint32_t c[3];
-#pragma unroll
-    for (int pl = 0; pl < 3; ++pl) {
-      const __nv_fp8x2_storage_t v = __nv_cvt_float2_to_fp8x2(r, __NV_SATFINITE, __NV_E5M2);   // .x in the low byte
-      const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2(v, __NV_E5M2);
-      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h));
-      r.x -= f.x;   // exact: the rest has fewer significant bits than the value
-      r.y -= f.y;
-      c[pl] = v;
-    }
-#pragma unroll
-    for (int pl = 0; pl < 3; ++pl) {
-      if ((j & 1) == 0) out[pl][j >> 1] = c[pl];
-      else out[pl][j >> 1] |= c[pl] << 16;
-    }
-  }
-  p1 = make_uint4(out[0][0], out[0][1], out[0][2], out[0][3]);
-  p2 = make_uint4(out[1][0], out[1][1], out[1][2], out[1][3]);
-  p3 = make_uint4(out[2][0], out[2][1], out[2][2], out[2][3]);
-}
-
 template <bool E4M3>
 __global__ void __launch_bounds__(kThreadsFp, 1)
 fine_paged_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, IndexArgs p) {
@@ -232,8 +205,7 @@ fine_paged_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
       m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
       m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 4));
-      int S = 0;
-      if (m > 0.f) S = min(100, max(-100, 14 - (static_cast<int>((__float_as_uint(m) >> 23) & 0xffu) - 127)));
+      const int S = e5m2_head_shift(m);
       const float up = __uint_as_float(static_cast<uint32_t>(S + 127) << 23);
 #pragma unroll
       for (int j = 0; j < 16; ++j) x[j] *= up;   // exact
