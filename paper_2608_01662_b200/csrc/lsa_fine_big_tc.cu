@@ -43,7 +43,7 @@ __global__ void __launch_bounds__(kSelThreads) page_topm_kernel(IndexArgs p, int
     const int nE = p1 - p0 + 1;
     if (p.hi_enable && nE > p.M) {
       const float* ps = p.page_scores + static_cast<int64_t>(qi) * p.ps_ld + p0;
-      nP = block_select_topk([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M, out, sc);
+      nP = block_select_topk<0, true>([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M, out, sc);
     } else {
       nP = nE;   // the host sized M so that every eligible page fits the list when the hierarchy is off
       for (int i = tid; i < p.M; i += kSelThreads) out[i] = i < nP ? p0 + i : -1;

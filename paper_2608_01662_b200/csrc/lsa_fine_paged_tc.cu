@@ -249,7 +249,7 @@ fine_paged_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           nP = block_select_topk<kSelBar>([&](int i) { return pk[i]; }, [&](int i) { return p0 + i; }, nE, p.M, sm.pages, sm.sel);
           tc::fence_proxy_async();   // the ring is handed to the TMA copies
         } else {
-          nP = block_select_topk<kSelBar>([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M,
+          nP = block_select_topk<kSelBar, true>([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M,
                                           sm.pages, sm.sel);
         }
       } else {

@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(kFineThreads, 2) fine_select_tc_kernel(const _
       __syncthreads();
       nP = block_select_topk([&](int i) { return sm.keys[i]; }, [&](int i) { return p0 + i; }, nE, p.M, sm.pages, sm.sel);
     } else {
-      nP = block_select_topk([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M, sm.pages,
+      nP = block_select_topk<0, true>([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M, sm.pages,
                              sm.sel);
     }
   } else {

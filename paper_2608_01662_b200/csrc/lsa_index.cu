@@ -11,6 +11,7 @@
 // thread quad and one number per key leaves the tile.
 #include "lsa_internal.h"
 #include "lsa_select.cuh"
+#include "lsa_select_cluster.cuh"
 #include "lsa_rows.cuh"
 
 #ifdef LSA_TIMELINE
@@ -348,6 +349,8 @@ __global__ void __launch_bounds__(kThreads, 2) coarse_score_paged_kernel(IndexAr
 // ------------------------------------------------------------------------------------------------
 // a2-a4: per query: top-M pages, fine scores on their tokens, top-K_sparse.
 // ------------------------------------------------------------------------------------------------
+constexpr int kClusterRowsMax = 256;    // rows: up to this many, a row of kClusterMinRow scores or more gets a cluster of blocks
+constexpr int kClusterMinRow = 16384;
 constexpr int kMaxSlots = 4096;  // keep_pages * page
 constexpr int kMaxPages = 64;    // keep_pages
 
@@ -410,7 +413,7 @@ __global__ void __launch_bounds__(kThreads, 2) fine_select_kernel(IndexArgs p) {
       LSA_TLF(7);
       nP = block_select_topk([&](int i) { return sm.keys[i]; }, [&](int i) { return p0 + i; }, nE, p.M, sm.pages, sm.sel);
     } else {
-      nP = block_select_topk([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M,
+      nP = block_select_topk<0, true>([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M,
                              sm.pages, sm.sel);
     }
   } else {
@@ -595,7 +598,7 @@ __global__ void __launch_bounds__(kSelThreads) page_topm_paged_kernel(IndexArgs 
       __syncthreads();
       nP = block_select_topk([&](int i) { return keys[i]; }, [&](int i) { return p0 + i; }, nE, p.M, pages, sc);
     } else {
-      nP = block_select_topk([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M, pages, sc);
+      nP = block_select_topk<0, true>([&](int i) { return score_key(ps[i]); }, [&](int i) { return p0 + i; }, nE, p.M, pages, sc);
     }
   } else {
     nP = nE;   // the host guarantees nE <= kMaxPages here
@@ -650,18 +653,47 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
   // the query of row qi sits at q_pos0 + qi, or (paged caches: one query per sequence) at the end of its sequence
   const int64_t lo = S, hi = (ctx_len ? static_cast<int64_t>(ctx_len[qi]) - 1 : q_pos0 + qi) - W;
   auto id = [&](int i) { return pos ? pos[i] : i; };
+  // (no branch between the loads and the test: the caller evaluates several keys per step and wants their loads in
+  // flight together)
   auto key = [&](int i) -> uint32_t {
     const int64_t s = id(i);
-    if (s < 0) return 0u;
-    if (apply_range && (s < lo || s > hi)) return 0u;
+    const bool ok = s >= 0 && (!apply_range || (s >= lo && s <= hi));
+    float v = row[i];
     // pos_scale: per-position factor of the score (the fp32 scale of an e4m3 key), applied before the comparison
-    return score_key(pos_scale ? row[i] * pos_scale[s] : row[i]);
+    if (pos_scale) v *= pos_scale[s < 0 ? 0 : s];
+    return ok ? score_key(v) : 0u;
   };
   // columns that are positions: nothing beyond the range can take part, so it is not even scanned
   int n = static_cast<int>(n_cand);
   if (pos == nullptr && apply_range) n = static_cast<int>(max64(0, min64(n_cand, hi + 1)));
-  const int n_sel = block_select_topk(key, id, n, k, idx_out + static_cast<int64_t>(qi) * k, sc);
+  const int n_sel = block_select_topk<0, true>(key, id, n, k, idx_out + static_cast<int64_t>(qi) * k, sc);
   if (threadIdx.x == 0) n_out[qi] = n_sel;
+}
+
+// The same selection with a cluster of kClusterSel blocks per row (few long rows: the flat indexer in decode).
+__global__ void __launch_bounds__(kSelThreads) select_cluster_kernel(const float* __restrict__ scores, int64_t ld,
+                                                                    const int32_t* __restrict__ cand_pos,
+                                                                    const float* __restrict__ pos_scale, int64_t q_pos0,
+                                                                    int64_t n_cand, int k, int apply_range, int S, int W,
+                                                                    int32_t* __restrict__ idx_out, int32_t* __restrict__ n_out,
+                                                                    const int32_t* __restrict__ ctx_len) {
+  __shared__ ClusterSelScratch sc;
+  const int qi = blockIdx.y;
+  const float* row = scores + qi * ld;
+  const int32_t* pos = cand_pos ? cand_pos + qi * n_cand : nullptr;
+  const int64_t lo = S, hi = (ctx_len ? static_cast<int64_t>(ctx_len[qi]) - 1 : q_pos0 + qi) - W;
+  auto id = [&](int i) { return pos ? pos[i] : i; };
+  auto key = [&](int i) -> uint32_t {   // branch-free, as in select_kernel
+    const int64_t s = id(i);
+    const bool ok = s >= 0 && (!apply_range || (s >= lo && s <= hi));
+    float v = row[i];
+    if (pos_scale) v *= pos_scale[s < 0 ? 0 : s];
+    return ok ? score_key(v) : 0u;
+  };
+  int n = static_cast<int>(n_cand);
+  if (pos == nullptr && apply_range) n = static_cast<int>(max64(0, min64(n_cand, hi + 1)));
+  const int n_sel = cluster_select_topk(key, id, n, k, idx_out + static_cast<int64_t>(qi) * k, sc);
+  if (threadIdx.x == 0 && blockIdx.x == 0) n_out[qi] = n_sel;
 }
 
 // e4m3 codes -> the same values as bf16 (exact), for the dense scoring of the flat indexer
@@ -1130,6 +1162,24 @@ cudaError_t launch_select(const float* scores, int64_t ld, const int32_t* cand_p
                           int64_t q_pos0, int n_query, int64_t n_cand, int k, int apply_range, int S, int W,
                           int32_t* idx_out, int32_t* n_out, cudaStream_t st, int64_t* n_launch, const int32_t* ctx_len) {
   if (n_query == 0) return cudaSuccess;
+  if (n_query <= kClusterRowsMax && n_cand >= kClusterMinRow) {
+    // few long rows: a cluster of blocks per row
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(kClusterSel, static_cast<unsigned>(n_query), 1);
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = kClusterSel;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, select_cluster_kernel, scores, ld, cand_pos, pos_scale, q_pos0, n_cand, k,
+                                             apply_range, S, W, idx_out, n_out, ctx_len);
+    ++*n_launch;
+    return e;
+  }
   select_kernel<<<n_query, kSelThreads, 0, st>>>(scores, ld, cand_pos, pos_scale, q_pos0, n_cand, k, apply_range, S, W,
                                                  idx_out, n_out, ctx_len);
   ++*n_launch;

@@ -39,7 +39,20 @@ __device__ __forceinline__ void select_sync() {
 // (ascending i).   AbsentF: void operator()(int r): there is no r-th item (r in [written, k)).
 // Every thread of the 256-thread block must call this (BAR != 0: threads 0-255 of a larger block, all of them).
 // Returns the number of items selected (min(k, #present)).
-template <int BAR = 0, class KeyF, class EmitF, class AbsentF>
+// Key of item i of [0, n), 0 beyond.  UNCOND: the functor is called for every i (on the last item beyond the range),
+// so that the global-memory loads inside it are not control-dependent and the loads of one step are issued together
+// (a functor that reads a long row from L2 runs 2.5 x faster that way; for keys in shared memory it does not pay).
+template <bool UNCOND, class KeyF>
+__device__ __forceinline__ uint32_t select_key(KeyF& key, int i, int n) {
+  if constexpr (UNCOND) {
+    const uint32_t v = key(min(i, n - 1));
+    return i < n ? v : 0u;
+  } else {
+    return i < n ? key(i) : 0u;
+  }
+}
+
+template <int BAR = 0, bool UNCOND = false, class KeyF, class EmitF, class AbsentF>
 __device__ int block_select_topk_emit(KeyF key, EmitF emit, AbsentF absent, int n, int k, SelectScratch& sc) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -66,7 +79,7 @@ __device__ int block_select_topk_emit(KeyF key, EmitF emit, AbsentF absent, int 
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const int i = i0 + u * kSelThreads;
-          kk[u] = i < n ? key(i) : 0u;
+          kk[u] = select_key<UNCOND>(key, i, n);
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u)
@@ -132,7 +145,7 @@ __device__ int block_select_topk_emit(KeyF key, EmitF emit, AbsentF absent, int 
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int i = i0 + 32 * u;
-      kk[u] = i < end ? key(i) : 0u;
+      kk[u] = select_key<UNCOND>(key, i, end);
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
@@ -162,7 +175,7 @@ __device__ int block_select_topk_emit(KeyF key, EmitF emit, AbsentF absent, int 
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int i = base + 32 * u + lane;
-      kk[u] = i < end ? key(i) : 0u;
+      kk[u] = select_key<UNCOND>(key, i, end);
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) eq_mask[u] = __ballot_sync(0xffffffffu, (kk[u] == T) && (kk[u] != 0u));
@@ -184,8 +197,8 @@ __device__ int block_select_topk_emit(KeyF key, EmitF emit, AbsentF absent, int 
 
 // The common form: out[r] = id(i) for the selected items in ascending i, out[written..k) = -1.
 // IdF: int operator()(int i).
-template <int BAR = 0, class KeyF, class IdF>
+template <int BAR = 0, bool UNCOND = false, class KeyF, class IdF>
 __device__ int block_select_topk(KeyF key, IdF id, int n, int k, int* out, SelectScratch& sc) {
-  return block_select_topk_emit<BAR>(key, [&](int r, int i) { out[r] = id(i); }, [&](int r) { out[r] = -1; }, n, k, sc);
+  return block_select_topk_emit<BAR, UNCOND>(key, [&](int r, int i) { out[r] = id(i); }, [&](int r) { out[r] = -1; }, n, k, sc);
 }
 }  // namespace lsa

@@ -24,7 +24,8 @@ def _sel_params(S=0, W=0):
 
 
 # ---------------------------------------------------------------- selection alone: bit exact
-@pytest.mark.parametrize("n_cand,k", [(1, 1), (37, 8), (1000, 256), (4096, 2048), (5000, 5000), (70000, 2048), (300, 512)])
+@pytest.mark.parametrize("n_cand,k", [(1, 1), (37, 8), (1000, 256), (4096, 2048), (5000, 5000), (70000, 2048), (300, 512),
+                                      (20000, 5000), (333333, 2048)])
 def test_select_is_bit_exact_on_given_scores(cuda_device, n_cand, k):
     g = torch.Generator(device="cpu").manual_seed(n_cand * 7 + k)
     n_query = 9
