@@ -144,7 +144,7 @@ LSA_API int64_t lsa_launch_count(lsa_ctx* ctx);
  *                           page top-M, token scores of the kept pages on tcgen05, top-K and cache rows; 1: the same
  *                           steps as three kernels (page lists, the scoring kernel the flat paged indexer uses,
  *                           top-K); 2: page top-M and token scores in one mma.sync kernel, several blocks per
- *                           sequence, then a top-K kernel.  Same selection.  cfg4: 39 / 72 / 58 us per decode step. */
+ *                           sequence, then a top-K kernel.  Same selection.  cfg4: 33 / 72 / 58 us per decode step. */
 enum { LSA_TUNE_COARSE_GROUPS = 0, LSA_TUNE_ATTN_TC, LSA_TUNE_ATTN_SPLIT, LSA_TUNE_ATTN_PV_WAIT, LSA_TUNE_ATTN_GATHER,
        LSA_TUNE_FINE_PAGED_TC, LSA_TUNE_COUNT };
 LSA_API int lsa_tune(lsa_ctx* ctx, int knob, int value);
