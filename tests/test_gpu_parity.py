@@ -73,6 +73,35 @@ def test_select_with_positions_range_and_leading_dimension(cuda_device):
     assert ctx.status() == 0
 
 
+def test_select_of_long_rows_with_positions_and_range(cuda_device):
+    """Rows long enough for the cluster selection (eight blocks per row): the scoring range cuts the row, explicit
+    candidate positions have holes, many scores tie, and a row has fewer candidates than k."""
+    rng = np.random.default_rng(8)
+    n_query, n_cand, k, S, W, q_pos0 = 5, 40000, 3000, 4, 300, 39000
+    scores = torch.from_numpy(np.round(rng.standard_normal((n_query, n_cand)), 2).astype(np.float32))
+    params = _sel_params(S, W)
+    ctx = binding.Context(params, n_query, n_cand, device=cuda_device)
+    idx = torch.empty((n_query, k), dtype=torch.int32, device=cuda_device)
+    cnt = torch.empty((n_query,), dtype=torch.int32, device=cuda_device)
+    d_sc = scores.to(cuda_device)
+    ctx.select(d_sc, None, q_pos0, k, True, idx, cnt)              # columns are positions; query i sits at q_pos0 + i
+    for i in range(n_query):
+        want = orc.select_fp32(scores[i].numpy(), None, q_pos0 + i, k, apply_range=True, S=S, W=W)
+        assert cnt[i] == len(want)
+        assert np.array_equal(idx[i, :int(cnt[i])].cpu().numpy(), want)
+    pos = np.stack([np.sort(rng.permutation(300000)[:n_cand]) for _ in range(n_query)]).astype(np.int32)
+    pos[:, ::7] = -1
+    pos[4, 2000:] = -1                                             # 2000 columns, of which 1714 are present: fewer than k
+    d_pos = torch.from_numpy(pos).to(cuda_device)
+    ctx.select(d_sc, d_pos, 0, k, False, idx, cnt)
+    for i in range(n_query):
+        want = orc.select_fp32(scores[i].numpy(), pos[i], 0, k, apply_range=False)
+        assert cnt[i] == len(want)
+        got = idx[i].cpu().numpy()
+        assert np.array_equal(got[:len(want)], want) and (got[len(want):] == -1).all()
+    assert ctx.status() == 0
+
+
 # ---------------------------------------------------------------- mean cache
 @pytest.mark.parametrize("cfg", [CONFIGS["cfg1"], SMALL_FP8], ids=lambda c: c.name)
 def test_block_means_match_oracle(cuda_device, cfg):
