@@ -281,12 +281,16 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
   // Q is requested before anything else that depends on the previous kernel: a block cannot start without it, and in
   // prefill it comes from HBM.
   auto request_q = [&]() {
-    if (q_tma && tid == 32 * (kSoftmaxWarps + kMmaWarps)) {
+    // nine boxes, dealt to lane 0 of the four gather warps (an issued TMA copy costs its thread 200-300 cycles); the
+    // first of them arrives on the barrier with the byte count of all nine (a box that completes before that only
+    // makes the count negative for a moment: the phase cannot end before the arrival)
+    const int qw = warp - (kSoftmaxWarps + kMmaWarps);
+    if (q_tma && lane == 0 && qw >= 0) {
       const uint32_t stage = smem_u32(sm.k[kKBufs - 1]);
-      tc::mbar_expect_tx(smem_u32(&sm.q_full), kH * kDQK * 2);
-      for (int a = 0; a < kAtoms; ++a)
+      if (qw == 0) tc::mbar_expect_tx(smem_u32(&sm.q_full), kH * kDQK * 2);
+      for (int a = qw; a < kAtoms; a += kLoadWarps)
         tc::tma_load_2d(a < 8 ? stage + a * kAtomBytes : smem_u32(sm.q_rope), &q_map, a * 64, qi * kH, smem_u32(&sm.q_full));
-      LSA_TL(kTlQIssued);
+      if (qw == 0) LSA_TL(kTlQIssued);
     }
   };
   if (!(early_rows && gather_warp)) {
@@ -433,11 +437,13 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
       LSA_TL_TILE(lt == 0, i, kTlKFreed);
       if (tile_by_tma(i)) {
         // 64 consecutive window rows: nine boxes that complete k_full by byte count; the (empty) cp.async group
-        // below keeps the hand-over bookkeeping the same for every kind of tile
-        if (lt == 0) {
-          tc::mbar_expect_tx_only(smem_u32(&sm.k_full[b]), kAtoms * kAtomBytes);
+        // below keeps the hand-over bookkeeping the same for every kind of tile.  An issued TMA copy costs its thread
+        // 200-300 cycles, so the nine boxes are dealt to the gather warps (each announces the bytes of its own)
+        if (lane == 0 && gw < kAtoms) {
+          const int n_mine = (kAtoms - gw + kGw - 1) / kGw;
+          tc::mbar_expect_tx_only(smem_u32(&sm.k_full[b]), n_mine * kAtomBytes);
           const int row0 = static_cast<int>(win0) + (tile_begin + i) * kTileKeys;
-          for (int a = 0; a < kAtoms; ++a)
+          for (int a = gw; a < kAtoms; a += kGw)
             tc::tma_load_2d(smem_u32(sm.k[b][a]), &k_map, a * 64, row0, smem_u32(&sm.k_full[b]));
         }
       } else if (g4) {

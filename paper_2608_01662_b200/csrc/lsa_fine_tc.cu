@@ -145,20 +145,22 @@ __global__ void __launch_bounds__(kFineThreads, 2) fine_select_tc_kernel(const _
   };
 
   if (TMA && warp < 3) {
-    // ================= TMA producer =================
-    if (tid == 0) {
+    // ================= TMA producers: lane 0 of warps 0 and 1 takes the boxes of one 64-row half of every tile each
+    // (an issued TMA copy costs its thread 200-300 cycles: four boxes per tile from one thread were a good part of a
+    // tile's time).  Warp 0 arrives on the barrier with the byte count of the whole tile; a box of warp 1 that completes
+    // before that only makes the count negative for a moment =================
+    if (lane == 0 && warp < 2) {
+      const int h = warp;
       for (int i = 0; i < n_tiles; ++i) {
         const int b = i & 1;
         if (!tc::mbar_wait(smem_u32(&sm.k_empty[b]), ((i >> 1) & 1) ^ 1, p.status)) break;
-        tc::mbar_expect_tx(smem_u32(&sm.k_full[b]), 2 * kAtomA);
+        if (h == 0) tc::mbar_expect_tx(smem_u32(&sm.k_full[b]), 2 * kAtomA);
+        // 64 consecutive slots lie in one page; rows past the cache read as zero
+        const int c = (tile0 + i) * kTile + 64 * h;
+        const int row = c < n_slots ? static_cast<int>(slot_pos(c)) : static_cast<int>(n_key);
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {   // 64 consecutive slots lie in one page; rows past the cache read as zero
-          const int c = (tile0 + i) * kTile + 64 * h;
-          const int row = c < n_slots ? static_cast<int>(slot_pos(c)) : static_cast<int>(n_key);
-#pragma unroll
-          for (int cb = 0; cb < 2; ++cb)
-            tc::tma_load_2d(smem_u32(sm.a[b][cb]) + h * 64 * 128, &map, cb * 64, row, smem_u32(&sm.k_full[b]));
-        }
+        for (int cb = 0; cb < 2; ++cb)
+          tc::tma_load_2d(smem_u32(sm.a[b][cb]) + h * 64 * 128, &map, cb * 64, row, smem_u32(&sm.k_full[b]));
       }
     }
   } else if (warp < 3) {
