@@ -133,12 +133,12 @@ def attn_bytes_per_launch(cfg, positions):
 
 
 # DRAM traffic of one attention launch, from the ncu capture of the same kernel on cfg3 cut to 16384 queries
-# (profiles/sparse_attn_tc_cfg3_16k.md: dram__bytes_read.sum 1.347529 GB + dram__bytes_write.sum 1.049575 GB).
+# (profiles/sparse_attn_tc_cfg3_16k.md: dram__bytes_read.sum 1.344671 GB + dram__bytes_write.sum 1.047908 GB).
 # Traffic there is q + out (the KV latent stays in L2), so it scales with the number of queries of a launch.
-NCU_ATTN_DRAM_BYTES_PER_QUERY = (1.347529e9 + 1.049575e9) / 16384
+NCU_ATTN_DRAM_BYTES_PER_QUERY = (1.344671e9 + 1.047908e9) / 16384
 # Decode: DRAM bytes of one attention launch per sequence, from the ncu capture at batch 16
-# (profiles/sparse_attn_tc_cfg4_decode_batch16.md: dram__bytes_read.sum 43.95 MB + dram__bytes_write.sum 0.57 MB).
-NCU_DECODE_ATTN_DRAM_BYTES_PER_SEQ = (43948544 + 574720) / 16
+# (profiles/sparse_attn_tc_cfg4_decode_batch16.md: dram__bytes_read.sum 43.95 MB + dram__bytes_write.sum 0.47 MB).
+NCU_DECODE_ATTN_DRAM_BYTES_PER_SEQ = (43949568 + 472832) / 16
 
 
 def measured_peaks():
