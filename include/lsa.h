@@ -60,7 +60,12 @@ typedef enum {
   LSA_ERR_WORKSPACE = -3,  /* workspace missing or smaller than lsa_workspace_bytes says */
   LSA_ERR_CUDA = -4,       /* a CUDA runtime call failed (see lsa_last_cuda_error) */
   LSA_ERR_TIMEOUT = -5,    /* a bounded device-side wait expired (reported through lsa_status) */
-  LSA_ERR_CAPACITY = -6    /* the call needs more scratch than a fixed-capacity entry point owns */
+  LSA_ERR_CAPACITY = -6,   /* the call needs more scratch than a fixed-capacity entry point owns */
+  LSA_ERR_INDEX = -7       /* checking build only (library compiled with -DLSA_CHECK, `python -m
+                              paper_2608_01662_b200.build --check`): an attention kernel met a cache row number
+                              outside [0, n_key) in a caller-given sparse list or row list; the row was skipped (it
+                              contributes nothing) and the code is reported through lsa_status.  The normal build
+                              trusts these lists, as it trusts its pointers */
 } lsa_error;
 
 enum { LSA_KEY_BF16 = 0, LSA_KEY_E4M3 = 1 };

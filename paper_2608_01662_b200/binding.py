@@ -15,7 +15,8 @@ import torch
 from .configs import LsaConfig
 
 _LIB = None
-LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblsa.so")
+# LSA_LIBRARY selects another build of the same library (the checking build liblsa_check.so, see build.py)
+LIB_PATH = os.environ.get("LSA_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblsa.so")
 
 LSA_KEY_BF16, LSA_KEY_E4M3 = 0, 1
 LSA_POOL_MEAN, LSA_POOL_MINMAX = 0, 1

@@ -326,7 +326,7 @@ int run_index(lsa_ctx* c, const lsa_params* p, const void* q_idx, const float* w
 int run_attn(lsa_ctx* c, const lsa_params* p, const void* q, const void* k, const void* v, int64_t ld_k,
              int64_t ld_v, const int32_t* sparse_idx, const int32_t* n_sparse, const int32_t* rows,
              const int32_t* n_rows, int64_t q_pos0, int64_t n_query, const int32_t* ctx_len, int batch,
-             void* out, float* lse) {
+             void* out, float* lse, int64_t n_key = 0) {
   const int64_t nq = p->paged ? batch : n_query;
   if (nq == 0) return LSA_OK;
   lsa::AttnArgs a{};
@@ -335,6 +335,7 @@ int run_attn(lsa_ctx* c, const lsa_params* p, const void* q, const void* k, cons
   a.q = q; a.k = k; a.v = v; a.ld_k = ld_k; a.ld_v = ld_v;
   a.sparse_idx = sparse_idx; a.n_sparse = n_sparse; a.rows = rows; a.n_rows = n_rows;
   a.rows_ld = p->k_sink + p->k_sparse + p->k_swa;
+  a.n_key = p->paged ? 0 : n_key;   // (the checking build validates caller-given row numbers against it)
   a.q_pos0 = q_pos0; a.n_query = static_cast<int>(nq); a.ctx_len = ctx_len; a.out = out; a.lse = lse;
   a.n_split = 1; a.status = status_word(c);
   a.qk_waits_pv = c->tune[LSA_TUNE_ATTN_PV_WAIT];
@@ -455,6 +456,7 @@ const char* lsa_strerror(int err) {
     case LSA_ERR_CUDA: return "CUDA runtime error";
     case LSA_ERR_TIMEOUT: return "device-side wait timed out";
     case LSA_ERR_CAPACITY: return "request exceeds the fixed scratch capacity of this entry point";
+    case LSA_ERR_INDEX: return "cache row number outside the cache (checking build)";
     default: return "unknown error";
   }
 }
@@ -626,7 +628,7 @@ int lsa_sparse_attn(lsa_ctx* c, const lsa_params* p, const void* q, const void* 
   if (n_query < 0 || q_pos0 < 0 || n_key < 0) return LSA_ERR_ARG;
   if (ld_k < p->d_qk || ld_v < p->d_v || (ld_k % 8) || (ld_v % 8)) return LSA_ERR_SHAPE;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return LSA_ERR_SHAPE;
-  return run_attn(c, p, q, k, v, ld_k, ld_v, sparse_idx, n_sparse, rows, n_rows, q_pos0, n_query, ctx_len, batch, out, lse);
+  return run_attn(c, p, q, k, v, ld_k, ld_v, sparse_idx, n_sparse, rows, n_rows, q_pos0, n_query, ctx_len, batch, out, lse, n_key);
 }
 
 int lsa_merge(lsa_ctx* c, const lsa_params* p, int n_parts, const void* const* outs, const float* const* lses,

@@ -63,9 +63,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) sparse_attn_kernel(AttnArgs p
   const int32_t* sp = p.sparse_idx ? p.sparse_idx + static_cast<int64_t>(qi) * p.Ksp : nullptr;
   auto row_of = [&](int i) -> int32_t {
     if (i >= n_tot) return -1;
-    if (rows) return rows[i];
+    if (rows) return checked_row(rows[i], p.n_key, p.status);
     if (i < n_sink) return i;
-    if (i < n_sink + n_sp) return sp[i - n_sink];
+    if (i < n_sink + n_sp) return checked_row(sp[i - n_sink], p.n_key, p.status);
     return static_cast<int32_t>(win0 + (i - n_sink - n_sp));
   };
   // slots of this split: whole tiles

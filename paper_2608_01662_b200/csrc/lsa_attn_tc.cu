@@ -320,11 +320,11 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
   auto row_of = [&](int i) -> int32_t {
     if (i >= n_tot) return -1;
     if constexpr (kRows) {
-      return rows[i];
+      return checked_row(rows[i], p.n_key, p.status);
     } else {
       if (i < n_win) return static_cast<int32_t>(win0 + i);
       if (i < n_win + n_sink) return i - n_win;
-      return sp[i - n_win - n_sink];
+      return checked_row(sp[i - n_win - n_sink], p.n_key, p.status);
     }
   };
   const int tiles_all = (n_tot + kTileKeys - 1) / kTileKeys;

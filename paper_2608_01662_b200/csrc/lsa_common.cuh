@@ -11,10 +11,23 @@ namespace lsa {
 
 // ---- device status word -----------------------------------------------------------------------
 // Slot 0 of the workspace: 0 = fine, otherwise the first problem a kernel recorded.
-enum : int { kDevOk = 0, kDevTimeout = -5 };
+enum : int { kDevOk = 0, kDevTimeout = -5, kDevBadIndex = -7 };
 
 __device__ __forceinline__ void report_status(int* status, int code) {
   if (status != nullptr) atomicCAS(status, 0, code);
+}
+
+// A cache row number taken from a caller-given list.  Checking build (-DLSA_CHECK): a number outside [0, limit)
+// other than the padding value -1 is recorded in the status word and treated as padding (the row is skipped);
+// limit <= 0 = the cache's size is not known to the call (paged pools).  Normal build: the number as it is.
+__device__ __forceinline__ int32_t checked_row(int32_t row, int64_t limit, int* status) {
+#ifdef LSA_CHECK
+  if (row < -1 || (limit > 0 && row >= limit)) {
+    report_status(status, kDevBadIndex);
+    return -1;
+  }
+#endif
+  return row;
 }
 
 __host__ __device__ __forceinline__ int64_t min64(int64_t a, int64_t b) { return a < b ? a : b; }

@@ -59,6 +59,7 @@ struct AttnArgs {
   const int32_t* rows;    // optional [n_query, rows_ld]
   const int32_t* n_rows;
   int rows_ld;
+  int64_t n_key;          // rows of a contiguous cache (0: paged pool, size unknown); read by the checking build only
   int64_t q_pos0;
   int n_query;
   const int32_t* ctx_len;
