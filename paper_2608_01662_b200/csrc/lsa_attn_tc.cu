@@ -720,8 +720,8 @@ __global__ void __launch_bounds__(kThreadsAttnTc, 1) sparse_attn_tc_kernel(const
     if (!clustered) {
       // The block's output is one contiguous piece of memory (64 rows of 512 bf16).  A thread owns half a row, so
       // direct stores would scatter 16-byte pieces over 32 rows per instruction; instead each warp lays its 16 rows
-      // out in the (now idle) key buffers, with a 16-byte pad per row against bank conflicts, and copies them out
-      // with consecutive lanes on consecutive 16-byte chunks.
+      // out in the (now idle) key buffers, with a 16-byte pad per row against bank conflicts, and every row leaves
+      // as one bulk copy.
       constexpr int kRowBytes = kDV * 2, kPitch = kRowBytes + 16;
       uint8_t* my_stage = stage + row * kPitch + hi * (kRowBytes / 2);
 #pragma unroll 1
